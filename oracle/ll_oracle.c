@@ -1,0 +1,400 @@
+/*
+ * CPU fp64 oracle for sink+window attention over a rolling KV cache.
+ *
+ * TEST INFRASTRUCTURE ONLY.  This file is the slow, plain definition the CUDA
+ * library is checked against.  It shares no code, header, table or constant
+ * with the CUDA path, and nothing in the product may call it.
+ *
+ * What it follows (paper sections):
+ *   - Frame sink, Sec. 3.3 "Frame Sink": the first frame chunk's tokens stay in
+ *     the cache for ever and are concatenated to every attention block's K/V;
+ *     the rest of the cache is a short rolling window, evicted normally.
+ *   - Short-window attention, Sec. 3.3: attention restricted to a fixed
+ *     temporal window of W latent frames.
+ *   - KV-recache, Sec. 3.1 and Sec. 3.3 (last paragraph): at a prompt switch the
+ *     cache is rebuilt from the most recent W generated frames only.
+ *   - Algorithm 2 (interactive inference): every denoising pass of a chunk
+ *     attends over the cache; the final clean pass commits the chunk's K/V.
+ *
+ * Readings where the paper is silent (the benchmark definition fixes them):
+ *   - W counts the current chunk ("9 local + 3 sink = effective window 12").
+ *   - Attention is bidirectional inside a chunk and causal across chunks.
+ *   - The sink is S whole frames, S a multiple of the chunk size; recache never
+ *     touches it.
+ *   - 3-D RoPE (the paper does not define one): the D/2 rotation pairs are
+ *     split t|h|w with n_h = n_w = floor(D/6) pairs and n_t = D/2 - 2*n_h pairs;
+ *     pair j holds elements (2j, 2j+1); pair i of an axis with n_a pairs turns by
+ *     pos_axis * theta^(-i/n_a).  Positions are absolute (t = frame index since
+ *     the stream began).  K is cached after the rotation.
+ *   - Softmax scale 1/sqrt(D); any q/k normalisation is upstream.
+ *
+ * Storage here is [layer][slot][token][head][dim] in double.  The slot rule
+ * (frame f -> slot f if f < S, else S + (f - S) mod W) is the bit-exact
+ * contract for the cache state.
+ *
+ * Every function states which step it is.  No blocking, fusion or reordering
+ * beyond the definition; OpenMP only parallelises over independent query rows.
+ */
+#include <math.h>
+#include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+
+#define LLO_OK 0
+#define LLO_ERR_ARG (-1)
+#define LLO_ERR_POSITION (-2)
+#define LLO_ERR_NOT_RESIDENT (-3)
+
+typedef struct llo {
+    int L, H, D, P, C, S, W;
+    int faithful;          /* 1: round roped Q/K to bf16 like the stored cache does */
+    int64_t *end;          /* [L] frames appended so far */
+    int32_t *slot_frame;   /* [L][S+W] absolute frame in each slot, -1 = empty */
+    int64_t *evictions;    /* [L] frames overwritten by a newer frame */
+    double *K, *V;         /* [L][S+W][P][H][D] */
+} llo;
+
+/* ---- helpers that are not part of the method ---------------------------- */
+
+static size_t slots(const llo *o) { return (size_t)(o->S + o->W); }
+static size_t row_elems(const llo *o) { return (size_t)o->H * o->D; }
+static size_t layer_elems(const llo *o) { return slots(o) * o->P * row_elems(o); }
+
+/* Round a double to the nearest bfloat16 value (8 significant bits, ties to
+ * even) and return it as a double.  Used only in storage-faithful mode. */
+double llo_round_bf16(double x)
+{
+    if (x == 0.0 || !isfinite(x)) return x;
+    int e;
+    double m = frexp(x, &e);              /* x = m * 2^e, 0.5 <= |m| < 1 */
+    double q = nearbyint(m * 256.0);      /* default rounding mode: ties to even */
+    return ldexp(q, e - 8);
+}
+
+/* ---- lifetime ------------------------------------------------------------ */
+
+llo *llo_create(int L, int H, int D, int P, int C, int S, int W, int faithful)
+{
+    if (L <= 0 || H <= 0 || D <= 0 || (D & 1) || P <= 0 || C <= 0 || S < 0 || W <= 0)
+        return NULL;
+    llo *o = (llo *)calloc(1, sizeof(llo));
+    if (!o) return NULL;
+    o->L = L; o->H = H; o->D = D; o->P = P; o->C = C; o->S = S; o->W = W;
+    o->faithful = faithful;
+    o->end = (int64_t *)calloc((size_t)L, sizeof(int64_t));
+    o->evictions = (int64_t *)calloc((size_t)L, sizeof(int64_t));
+    o->slot_frame = (int32_t *)malloc((size_t)L * slots(o) * sizeof(int32_t));
+    o->K = (double *)calloc((size_t)L * layer_elems(o), sizeof(double));
+    o->V = (double *)calloc((size_t)L * layer_elems(o), sizeof(double));
+    if (!o->end || !o->evictions || !o->slot_frame || !o->K || !o->V) return NULL;
+    for (size_t i = 0; i < (size_t)L * slots(o); ++i) o->slot_frame[i] = -1;
+    return o;
+}
+
+void llo_destroy(llo *o)
+{
+    if (!o) return;
+    free(o->end); free(o->evictions); free(o->slot_frame); free(o->K); free(o->V);
+    free(o);
+}
+
+/* Reset (Algorithm 2, "initialise KV cache C <- []"): every layer forgets
+ * everything; stored bytes need not be cleared. */
+int llo_reset(llo *o)
+{
+    if (!o) return LLO_ERR_ARG;
+    for (int l = 0; l < o->L; ++l) { o->end[l] = 0; o->evictions[l] = 0; }
+    for (size_t i = 0; i < (size_t)o->L * slots(o); ++i) o->slot_frame[i] = -1;
+    return LLO_OK;
+}
+
+int llo_get_state(const llo *o, int layer, int64_t *end, int32_t *slot_frame,
+                  int64_t *evictions)
+{
+    if (!o || layer < 0 || layer >= o->L) return LLO_ERR_ARG;
+    *end = o->end[layer];
+    if (evictions) *evictions = o->evictions[layer];
+    memcpy(slot_frame, o->slot_frame + (size_t)layer * slots(o), slots(o) * sizeof(int32_t));
+    return LLO_OK;
+}
+
+/* ---- step: slot rule ------------------------------------------------------ */
+
+/* Sink frames keep slot f for ever; later frames roll through W ring slots. */
+int llo_slot_of(const llo *o, int64_t f)
+{
+    if (f < o->S) return (int)f;
+    return o->S + (int)((f - o->S) % o->W);
+}
+
+/* ---- step: 3-D RoPE ------------------------------------------------------- */
+
+void llo_rope_split(int D, int *n_t, int *n_h, int *n_w)
+{
+    *n_h = D / 6;
+    *n_w = D / 6;
+    *n_t = D / 2 - 2 * (D / 6);
+}
+
+/* Rotate one head row of D values sitting at grid position (t, y, x). */
+static void rope_row(const double *in, double *out, int D, double theta,
+                     int64_t t, int y, int x, int round_bf16)
+{
+    int n_t, n_h, n_w;
+    llo_rope_split(D, &n_t, &n_h, &n_w);
+    for (int j = 0; j < D / 2; ++j) {
+        double pos; int i, n_a;
+        if (j < n_t)            { pos = (double)t; i = j;             n_a = n_t; }
+        else if (j < n_t + n_h) { pos = (double)y; i = j - n_t;       n_a = n_h; }
+        else                    { pos = (double)x; i = j - n_t - n_h; n_a = n_w; }
+        double ang = pos * pow(theta, -(double)i / (double)n_a);
+        double c = cos(ang), s = sin(ang);
+        double a = in[2 * j], b = in[2 * j + 1];
+        double r0 = a * c - b * s;
+        double r1 = a * s + b * c;
+        out[2 * j]     = round_bf16 ? llo_round_bf16(r0) : r0;
+        out[2 * j + 1] = round_bf16 ? llo_round_bf16(r1) : r1;
+    }
+}
+
+/* RoPE over a token-major tensor [n_frames*gh*gw, H, D]; token n of a frame is
+ * (y, x) = (n / gw, n % gw); frame index = frame_start + token / (gh*gw). */
+int llo_rope(const double *in, double *out, int64_t n_tokens, int H, int D,
+             int64_t frame_start, int gh, int gw, double theta, int round_bf16)
+{
+    if (!in || !out || gh <= 0 || gw <= 0 || (D & 1)) return LLO_ERR_ARG;
+    int64_t P = (int64_t)gh * gw;
+    for (int64_t n = 0; n < n_tokens; ++n) {
+        int64_t t = frame_start + n / P;
+        int y = (int)((n % P) / gw), x = (int)((n % P) % gw);
+        for (int h = 0; h < H; ++h) {
+            size_t off = ((size_t)n * H + h) * D;
+            rope_row(in + off, out + off, D, theta, t, y, x, round_bf16);
+        }
+    }
+    return LLO_OK;
+}
+
+/* ---- step: append (Algorithm 2, cache write; Sec. 3.3 rolling window) ----- */
+
+/* Accepts frame_start == end (a new chunk: may evict, end += C) or
+ * frame_start == end - C (overwrite the newest chunk: state unchanged). */
+int llo_append(llo *o, int layer, const double *k, const double *v,
+               int64_t frame_start, int n_frames, int gh, int gw, double theta)
+{
+    if (!o || layer < 0 || layer >= o->L || !k || !v) return LLO_ERR_ARG;
+    if (n_frames != o->C || gh * gw != o->P) return LLO_ERR_ARG;
+    int64_t end = o->end[layer];
+    int is_new = (frame_start == end);
+    int is_over = (end >= o->C && frame_start == end - o->C);
+    if (!is_new && !is_over) return LLO_ERR_POSITION;
+
+    int32_t *sf = o->slot_frame + (size_t)layer * slots(o);
+    double *K = o->K + (size_t)layer * layer_elems(o);
+    double *V = o->V + (size_t)layer * layer_elems(o);
+    size_t re = row_elems(o);
+    for (int i = 0; i < n_frames; ++i) {
+        int64_t f = frame_start + i;
+        int slot = llo_slot_of(o, f);
+        if (sf[slot] >= 0 && sf[slot] != f) o->evictions[layer] += 1;
+        sf[slot] = (int32_t)f;
+        for (int n = 0; n < o->P; ++n) {
+            int y = n / gw, x = n % gw;
+            size_t src = ((size_t)i * o->P + n) * re;
+            size_t dst = ((size_t)slot * o->P + n) * re;
+            for (int h = 0; h < o->H; ++h)
+                rope_row(k + src + (size_t)h * o->D, K + dst + (size_t)h * o->D,
+                         o->D, theta, f, y, x, o->faithful);
+            memcpy(V + dst, v + src, re * sizeof(double));
+        }
+    }
+    if (is_new) o->end[layer] = end + o->C;
+    return LLO_OK;
+}
+
+/* ---- step: visible set ---------------------------------------------------- */
+
+/* Frame fk is visible to a query in frame fq iff it is not in a later chunk
+ * and it is either a sink frame or inside the W-frame window that ends with the
+ * query's chunk.  lo_floor additionally hides non-sink frames older than it
+ * (recache: frames that no longer exist). */
+int llo_visible(const llo *o, int64_t fq, int64_t fk, int64_t lo_floor)
+{
+    int64_t hi = (fq / o->C + 1) * o->C;      /* one past the query's chunk */
+    if (fk < 0 || fk >= hi) return 0;
+    if (fk < o->S) return 1;
+    return fk >= hi - o->W && fk >= lo_floor;
+}
+
+/* ---- step: attention ------------------------------------------------------ */
+
+/* Softmax attention of selected query rows over their visible keys.
+ *   q_roped [n_q_frames*P, H, D] : queries after RoPE
+ *   rows[n_rows]                 : query row indices to evaluate (NULL = all)
+ *   out [n_rows, H, D], lse [n_rows, H] (natural log of the softmax denominator)
+ * Per row and head: s_j = q.k_j / sqrt(D), p = softmax(s), o = sum p_j v_j. */
+int llo_attn(const llo *o, int layer, const double *q_roped, int64_t q_frame_start,
+             int n_q_frames, int64_t lo_floor, const int64_t *rows, int64_t n_rows,
+             double *out, double *lse)
+{
+    if (!o || layer < 0 || layer >= o->L || !q_roped || !out) return LLO_ERR_ARG;
+    int64_t nq = (int64_t)n_q_frames * o->P;
+    if (!rows) n_rows = nq;
+    const int32_t *sf = o->slot_frame + (size_t)layer * slots(o);
+    const double *K = o->K + (size_t)layer * layer_elems(o);
+    const double *V = o->V + (size_t)layer * layer_elems(o);
+    const int H = o->H, D = o->D, P = o->P;
+    const double scale = 1.0 / sqrt((double)D);
+    int status = LLO_OK;
+
+#pragma omp parallel for schedule(dynamic, 1)
+    for (int64_t ri = 0; ri < n_rows; ++ri) {
+        int64_t r = rows ? rows[ri] : ri;
+        if (r < 0 || r >= nq) { status = LLO_ERR_ARG; continue; }
+        int64_t fq = q_frame_start + r / P;
+        int64_t hi = (fq / o->C + 1) * o->C;
+        /* visible frames -> slots; every visible frame must be resident */
+        int nvis = 0;
+        int *vslot = (int *)malloc(sizeof(int) * (size_t)(o->S + o->W));
+        for (int64_t fk = 0; fk < hi; ++fk) {
+            if (!llo_visible(o, fq, fk, lo_floor)) continue;
+            int slot = llo_slot_of(o, fk);
+            if (sf[slot] != (int32_t)fk || nvis >= o->S + o->W) { status = LLO_ERR_NOT_RESIDENT; nvis = -1; break; }
+            vslot[nvis++] = slot;
+        }
+        if (nvis <= 0) { free(vslot); if (nvis == 0) status = LLO_ERR_NOT_RESIDENT; continue; }
+        int64_t nk = (int64_t)nvis * P;
+        double *s = (double *)malloc(sizeof(double) * (size_t)nk);
+        for (int h = 0; h < H; ++h) {
+            const double *qv = q_roped + ((size_t)r * H + h) * D;
+            double m = -INFINITY;
+            for (int a = 0; a < nvis; ++a)
+                for (int n = 0; n < P; ++n) {
+                    const double *kv = K + (((size_t)vslot[a] * P + n) * H + h) * D;
+                    double dot = 0.0;
+                    for (int d = 0; d < D; ++d) dot += qv[d] * kv[d];
+                    dot *= scale;
+                    s[(size_t)a * P + n] = dot;
+                    if (dot > m) m = dot;
+                }
+            double denom = 0.0;
+            for (int64_t j = 0; j < nk; ++j) { s[j] = exp(s[j] - m); denom += s[j]; }
+            double *ov = out + ((size_t)ri * H + h) * D;
+            for (int d = 0; d < D; ++d) ov[d] = 0.0;
+            for (int a = 0; a < nvis; ++a)
+                for (int n = 0; n < P; ++n) {
+                    double p = s[(size_t)a * P + n] / denom;
+                    const double *vv = V + (((size_t)vslot[a] * P + n) * H + h) * D;
+                    for (int d = 0; d < D; ++d) ov[d] += p * vv[d];
+                }
+            if (lse) lse[(size_t)ri * H + h] = m + log(denom);
+        }
+        free(s); free(vslot);
+    }
+    return status;
+}
+
+/* Softmax probabilities of one (row, head) and the cache rows they belong to;
+ * for tiny cases (checks that rows sum to one, and which keys are seen).
+ * key_rows[j] = slot*P + token.  Returns the number of visible keys or <0. */
+int64_t llo_attn_probs(const llo *o, int layer, const double *q_roped, int64_t q_frame_start,
+                       int64_t lo_floor, int64_t row, int head, double *probs,
+                       int64_t *key_rows, int64_t cap)
+{
+    if (!o || layer < 0 || layer >= o->L) return LLO_ERR_ARG;
+    const int32_t *sf = o->slot_frame + (size_t)layer * slots(o);
+    const double *K = o->K + (size_t)layer * layer_elems(o);
+    const int H = o->H, D = o->D, P = o->P;
+    int64_t fq = q_frame_start + row / P;
+    int64_t hi = (fq / o->C + 1) * o->C;
+    int64_t nk = 0;
+    const double *qv = q_roped + ((size_t)row * H + head) * D;
+    double m = -INFINITY;
+    for (int64_t fk = 0; fk < hi; ++fk) {
+        if (!llo_visible(o, fq, fk, lo_floor)) continue;
+        int slot = llo_slot_of(o, fk);
+        if (sf[slot] != (int32_t)fk) return LLO_ERR_NOT_RESIDENT;
+        for (int n = 0; n < P; ++n) {
+            if (nk >= cap) return LLO_ERR_ARG;
+            const double *kv = K + (((size_t)slot * P + n) * H + head) * D;
+            double dot = 0.0;
+            for (int d = 0; d < D; ++d) dot += qv[d] * kv[d];
+            probs[nk] = dot / sqrt((double)D);
+            key_rows[nk] = (int64_t)slot * P + n;
+            if (probs[nk] > m) m = probs[nk];
+            ++nk;
+        }
+    }
+    double denom = 0.0;
+    for (int64_t j = 0; j < nk; ++j) { probs[j] = exp(probs[j] - m); denom += probs[j]; }
+    for (int64_t j = 0; j < nk; ++j) probs[j] /= denom;
+    return nk;
+}
+
+/* ---- step: recache (Sec. 3.1; Sec. 3.3 last paragraph) --------------------- */
+
+/* Rebuild the ring from fresh K/V of the resident window frames
+ * [r0, end), r0 = max(S, end - W): re-rope and overwrite their rows (slot table,
+ * end and sink untouched), then attend all those frames' queries under the
+ * block-causal visible set.  q_roped_out (nullable) receives the roped queries.
+ * n_frames must equal end - r0 (0 when only sink frames exist: no work). */
+int llo_recache(llo *o, int layer, const double *q, const double *k, const double *v,
+                int n_frames, int gh, int gw, double theta,
+                const int64_t *rows, int64_t n_rows,
+                double *q_roped_out, double *out, double *lse)
+{
+    if (!o || layer < 0 || layer >= o->L) return LLO_ERR_ARG;
+    if (gh * gw != o->P) return LLO_ERR_ARG;
+    int64_t end = o->end[layer];
+    int64_t r0 = end - o->W; if (r0 < o->S) r0 = o->S;
+    int64_t resident = end - r0; if (resident < 0) resident = 0;
+    if (n_frames != resident) return LLO_ERR_POSITION;
+    if (n_frames == 0) return LLO_OK;
+    if (!q || !k || !v || !out) return LLO_ERR_ARG;
+
+    const int32_t *sf = o->slot_frame + (size_t)layer * slots(o);
+    double *K = o->K + (size_t)layer * layer_elems(o);
+    double *V = o->V + (size_t)layer * layer_elems(o);
+    size_t re = row_elems(o);
+    for (int i = 0; i < n_frames; ++i) {
+        int64_t f = r0 + i;
+        int slot = llo_slot_of(o, f);
+        if (sf[slot] != (int32_t)f) return LLO_ERR_NOT_RESIDENT;
+        for (int n = 0; n < o->P; ++n) {
+            int y = n / gw, x = n % gw;
+            size_t src = ((size_t)i * o->P + n) * re;
+            size_t dst = ((size_t)slot * o->P + n) * re;
+            for (int h = 0; h < o->H; ++h)
+                rope_row(k + src + (size_t)h * o->D, K + dst + (size_t)h * o->D,
+                         o->D, theta, f, y, x, o->faithful);
+            memcpy(V + dst, v + src, re * sizeof(double));
+        }
+    }
+    int64_t nq = (int64_t)n_frames * o->P;
+    double *qr = q_roped_out ? q_roped_out : (double *)malloc(sizeof(double) * (size_t)nq * re);
+    llo_rope(q, qr, nq, o->H, o->D, r0, gh, gw, theta, o->faithful);
+    int st = llo_attn(o, layer, qr, r0, n_frames, r0, rows, n_rows, out, lse);
+    if (!q_roped_out) free(qr);
+    return st;
+}
+
+/* Read back one cache row (slot*P + token) of K and V, [H, D] each. */
+int llo_read_row(const llo *o, int layer, int64_t cache_row, double *k_out, double *v_out)
+{
+    if (!o || layer < 0 || layer >= o->L) return LLO_ERR_ARG;
+    if (cache_row < 0 || cache_row >= (int64_t)slots(o) * o->P) return LLO_ERR_ARG;
+    size_t off = (size_t)layer * layer_elems(o) + (size_t)cache_row * row_elems(o);
+    memcpy(k_out, o->K + off, row_elems(o) * sizeof(double));
+    memcpy(v_out, o->V + off, row_elems(o) * sizeof(double));
+    return LLO_OK;
+}
+
+/* Bulk read of a layer's cache, [S+W, P, H, D] each. */
+int llo_read_layer(const llo *o, int layer, double *k_out, double *v_out)
+{
+    if (!o || layer < 0 || layer >= o->L) return LLO_ERR_ARG;
+    size_t off = (size_t)layer * layer_elems(o);
+    memcpy(k_out, o->K + off, layer_elems(o) * sizeof(double));
+    memcpy(v_out, o->V + off, layer_elems(o) * sizeof(double));
+    return LLO_OK;
+}

@@ -1,0 +1,448 @@
+"""Pins for the CPU oracle: facts fixed by the paper and by mathematics.
+
+None of these tests re-types the oracle's own formula.  Each one checks the
+oracle against something independent: a literal list-based cache (Sec. 3.3
+"Frame Sink"), a flat library-softmax attention over the full history, closed
+forms, a complex-number textbook RoPE, and constants the paper prints.
+"""
+import os
+
+import numpy as np
+import pytest
+from scipy.special import logsumexp, softmax
+
+from paper_2509_22622_b200 import synth
+
+GOLDEN = os.path.join(os.path.dirname(__file__), "golden", "paper_constants.txt")
+
+
+def golden():
+    out = {}
+    with open(GOLDEN) as fh:
+        for line in fh:
+            line = line.split("#")[0].split()
+            if line:
+                out[line[0]] = [int(t) for t in line[1:]]
+    return out
+
+
+def rand(shape, seed):
+    return synth.bf16_bits_to_f64(synth.normal_bf16(np.random.default_rng(seed), shape))
+
+
+# ---------------------------------------------------------------------------
+# independent references used by the pins
+# ---------------------------------------------------------------------------
+
+def literal_cache_frames(end, S, W):
+    """Sec. 3.3 read literally: the first chunk stays, the rest is the last W frames."""
+    frames = list(range(end))
+    sink = frames[:S]
+    rest = frames[S:]
+    window = [f for f in frames[-W:] if f in rest] if W > 0 else []
+    return sink + window
+
+
+def textbook_rope_1d(x, pos, theta):
+    """RoFormer's rotary embedding on pairs (2i, 2i+1), as complex multiplication."""
+    d = x.shape[-1]
+    z = x[..., 0::2] + 1j * x[..., 1::2]
+    freq = theta ** (-np.arange(0, d, 2) / d)
+    z = z * np.exp(1j * pos * freq)
+    out = np.empty_like(x)
+    out[..., 0::2] = z.real
+    out[..., 1::2] = z.imag
+    return out
+
+
+def flat_block_causal(q, keys, vals, q_chunk, key_chunk):
+    """Full-history attention with library softmax.  q [nq,H,D]; keys/vals [nk,H,D];
+    key j is visible iff its chunk id <= the query's chunk id."""
+    D = q.shape[-1]
+    s = np.einsum("qhd,khd->hqk", q, keys) / np.sqrt(D)
+    mask = key_chunk[None, :] <= q_chunk[:, None]
+    s = np.where(mask[None], s, -np.inf)
+    p = softmax(s, axis=-1)
+    return np.einsum("hqk,khd->qhd", p, vals), logsumexp(s, axis=-1).T
+
+
+# ---------------------------------------------------------------------------
+# slot rule, visible set, sink persistence
+# ---------------------------------------------------------------------------
+
+@pytest.mark.parametrize("C,S,W", [(1, 1, 2), (3, 3, 9), (2, 2, 4), (1, 0, 3), (2, 4, 6), (3, 3, 3)])
+def test_resident_frames_match_literal_cache(oracle_mod, C, S, W):
+    """After every append the slot table holds exactly sink + last W frames."""
+    o = oracle_mod.Oracle(1, 1, 2, 1, C, S, W)
+    for chunk in range(12):
+        x = np.zeros((C, 1, 2))
+        o.append(0, x, x, chunk * C, 1, 1)
+        st = o.state()
+        end = (chunk + 1) * C
+        assert st["end"] == end
+        resident = sorted(int(f) for f in st["slot_frame"] if f >= 0)
+        assert resident == sorted(set(literal_cache_frames(end, S, W)))
+        # every resident frame sits where the slot rule says
+        for f in resident:
+            assert st["slot_frame"][o.slot_of(f)] == f
+
+
+@pytest.mark.parametrize("C,S,W", [(1, 1, 2), (3, 3, 9), (2, 2, 4), (1, 0, 3), (3, 3, 3)])
+def test_visible_set_bruteforce(oracle_mod, C, S, W):
+    """visible(fq, fk) for the newest chunk == the literal cache content, for every fq, fk."""
+    o = oracle_mod.Oracle(1, 1, 2, 1, C, S, W)
+    for chunk in range(10):
+        end = (chunk + 1) * C
+        expect = set(literal_cache_frames(end, S, W))
+        for fq in range(chunk * C, end):
+            got = {fk for fk in range(-2, end + 4) if o.visible(fq, fk)}
+            assert got == expect, (chunk, fq)
+
+
+def test_visible_set_is_block_causal_for_old_queries(oracle_mod):
+    """A query of an older chunk sees nothing from later chunks, all of its own chunk."""
+    o = oracle_mod.Oracle(1, 1, 2, 1, 3, 3, 9)
+    for fq in range(0, 30):
+        hi = (fq // 3 + 1) * 3
+        vis = {fk for fk in range(40) if o.visible(fq, fk)}
+        assert max(vis) == hi - 1
+        assert set(range(fq // 3 * 3, hi)) <= vis
+        assert vis == set(literal_cache_frames(hi, 3, 9))
+
+
+def test_steady_state_key_count_matches_paper(oracle_mod):
+    g = golden()
+    C, S, W = g["chunk_frames"][0], g["sink_frames"][0], g["window_frames"][0]
+    o = oracle_mod.Oracle(1, 1, 2, 1, C, S, W)
+    n_vis = sum(o.visible(20 * C, fk) for fk in range(100))
+    assert n_vis == g["effective_frames"][0]
+    assert n_vis * g["tokens_per_frame"][0] == g["max_keys"][0]
+    # a 21-frame clip under sink 3 + window 18 is full block-causal attention
+    o2 = oracle_mod.Oracle(1, 1, 2, 1, C, S, 18)
+    for fq in range(g["clip_latent_frames"][0]):
+        hi = (fq // C + 1) * C
+        assert {fk for fk in range(30) if o2.visible(fq, fk)} == set(range(hi))
+
+
+def test_sink_never_evicted_and_bytes_stable(oracle_mod):
+    C, S, W, P, H, D = 2, 2, 4, 3, 2, 8
+    o = oracle_mod.Oracle(1, H, D, P, C, S, W)
+    sink_k = sink_v = None
+    for chunk in range(9):
+        k, v = rand((C * P, H, D), 10 + chunk), rand((C * P, H, D), 50 + chunk)
+        o.append(0, k, v, chunk * C, 1, 3)
+        K, V = o.read_layer()
+        if chunk == 0:
+            sink_k, sink_v = K[:S].copy(), V[:S].copy()
+            assert np.array_equal(V[:S].reshape(C * P, H, D), v)
+        if chunk == 4:   # a recache in the middle must not touch the sink
+            n = min(W, (chunk + 1) * C - S)
+            qn, kn, vn = (rand((n * P, H, D), 90 + i) for i in range(3))
+            o.recache(0, qn, kn, vn, n, 1, 3)
+            K, V = o.read_layer()
+        assert list(o.state()["slot_frame"][:S]) == list(range(S))
+        assert np.array_equal(K[:S], sink_k) and np.array_equal(V[:S], sink_v)
+    assert o.state()["evictions"] == 9 * C - S - W
+
+
+def test_append_position_rules(oracle_mod):
+    o = oracle_mod.Oracle(1, 1, 2, 1, 2, 2, 4)
+    x = np.zeros((2, 1, 2))
+    with pytest.raises(oracle_mod.OracleError):
+        o.append(0, x, x, 2, 1, 1)          # skips chunk 0
+    o.append(0, x, x, 0, 1, 1)
+    o.append(0, x, x, 0, 1, 1)              # overwrite newest: state unchanged
+    assert o.state()["end"] == 2
+    o.append(0, x, x, 2, 1, 1)
+    with pytest.raises(oracle_mod.OracleError):
+        o.append(0, x, x, 0, 1, 1)          # not the newest chunk any more
+    o.reset()
+    assert o.state()["end"] == 0 and all(o.state()["slot_frame"] == -1)
+
+
+# ---------------------------------------------------------------------------
+# RoPE
+# ---------------------------------------------------------------------------
+
+def test_rope_band_sizes_match_definition(oracle_mod):
+    g = golden()
+    assert list(oracle_mod.rope_split(128)) == g["rope_pairs_d128"]
+    assert [2 * n for n in oracle_mod.rope_split(64)] == g["rope_dims_d64"]
+
+
+@pytest.mark.parametrize("D", [64, 128])
+def test_rope_reduces_to_textbook_1d(oracle_mod, D):
+    """On a 1x1 grid only the t band turns, and it is RoFormer's rotation."""
+    n_t, n_h, n_w = oracle_mod.rope_split(D)
+    x = rand((5, 3, D), 3)
+    got = oracle_mod.rope(x, frame_start=7, gh=1, gw=1, theta=10000.0)
+    for i in range(5):
+        want = x[i].copy()
+        want[:, :2 * n_t] = textbook_rope_1d(x[i][:, :2 * n_t], 7 + i, 10000.0)
+        np.testing.assert_allclose(got[i], want, rtol=0, atol=1e-12)
+
+
+@pytest.mark.parametrize("D", [64, 128])
+def test_rope_each_axis_is_textbook_on_its_band(oracle_mod, D):
+    """Frame 0: t band idle; h and w bands turn by y and x (row-major tokens)."""
+    n_t, n_h, n_w = oracle_mod.rope_split(D)
+    gh, gw = 3, 4
+    x = rand((gh * gw, 2, D), 4)
+    got = oracle_mod.rope(x, 0, gh, gw, 100.0)
+    a, b = 2 * n_t, 2 * (n_t + n_h)
+    for n in range(gh * gw):
+        yy, xx = divmod(n, gw)
+        want = x[n].copy()
+        want[:, a:b] = textbook_rope_1d(x[n][:, a:b], yy, 100.0)
+        want[:, b:] = textbook_rope_1d(x[n][:, b:], xx, 100.0)
+        np.testing.assert_allclose(got[n], want, rtol=0, atol=1e-12)
+
+
+def test_rope_identity_norm_and_relative_property(oracle_mod):
+    D, gh, gw = 128, 2, 3
+    x = rand((gh * gw, 2, D), 5)
+    r = oracle_mod.rope(x, 0, gh, gw)
+    assert np.array_equal(r[0], x[0])                       # position (0,0,0)
+    pair_norm = lambda a: a[..., 0::2] ** 2 + a[..., 1::2] ** 2
+    np.testing.assert_allclose(pair_norm(r), pair_norm(x), rtol=1e-12)
+    # scores depend on position differences only: shift t of both q and k
+    q, k = rand((gh * gw, 2, D), 6), rand((gh * gw, 2, D), 7)
+    s0 = np.einsum("qhd,khd->hqk", oracle_mod.rope(q, 3, gh, gw), oracle_mod.rope(k, 1, gh, gw))
+    s1 = np.einsum("qhd,khd->hqk", oracle_mod.rope(q, 903, gh, gw), oracle_mod.rope(k, 901, gh, gw))
+    np.testing.assert_allclose(s0, s1, rtol=0, atol=1e-9)
+    # ...but do change when only one side moves
+    s2 = np.einsum("qhd,khd->hqk", oracle_mod.rope(q, 4, gh, gw), oracle_mod.rope(k, 1, gh, gw))
+    assert np.abs(s2 - s0).max() > 1e-3
+
+
+def test_round_bf16_matches_bit_rounding(oracle_mod):
+    x = np.random.default_rng(0).standard_normal(2000).astype(np.float32)
+    want = synth.bf16_bits_to_f64(synth.f32_to_bf16_bits(x))
+    np.testing.assert_array_equal(oracle_mod.round_bf16(x.astype(np.float64)), want)
+    ties = np.array([1 + 2.0 ** -8, 1 + 3 * 2.0 ** -8, -(2 + 2.0 ** -7)])
+    np.testing.assert_array_equal(oracle_mod.round_bf16(ties), [1.0, 1.015625, -2.0])
+
+
+# ---------------------------------------------------------------------------
+# attention
+# ---------------------------------------------------------------------------
+
+def stream(o, n_chunks, gh, gw, seed, theta=10000.0):
+    """Append n_chunks chunks, attend each as it arrives.  Returns per-chunk
+    (out, lse) plus the flat roped history for the flat reference."""
+    P = gh * gw
+    outs, hist_k, hist_v, hist_q = [], [], [], []
+    for c in range(n_chunks):
+        q, k, v = (rand((o.C * P, o.H, o.D), seed + 3 * c + i) for i in range(3))
+        o.append(0, k, v, c * o.C, gh, gw, theta)
+        qr = o.rope_q(q, c * o.C, gh, gw, theta)
+        outs.append(o.attn(0, qr, c * o.C))
+        hist_q.append(qr)
+        hist_k.append(oracle_mod_rope(k, c * o.C, gh, gw, theta))
+        hist_v.append(v)
+    return outs, hist_q, hist_k, hist_v
+
+
+def oracle_mod_rope(x, fs, gh, gw, theta):
+    import oracle
+    return oracle.rope(x, fs, gh, gw, theta)
+
+
+@pytest.mark.parametrize("C,S,W,n_chunks", [(1, 1, 7, 8), (2, 2, 8, 5), (2, 0, 10, 5), (3, 3, 9, 4)])
+def test_window_covering_history_is_full_causal(oracle_mod, C, S, W, n_chunks):
+    """W >= total - S: sink+window equals flat block-causal attention."""
+    gh, gw, H, D = 2, 3, 2, 16
+    P = gh * gw
+    o = oracle_mod.Oracle(1, H, D, P, C, S, W)
+    outs, hq, hk, hv = stream(o, n_chunks, gh, gw, 100)
+    keys, vals = np.concatenate(hk), np.concatenate(hv)
+    key_chunk = np.repeat(np.arange(n_chunks), C * P)
+    for c in range(n_chunks):
+        want, want_lse = flat_block_causal(hq[c], keys, vals, np.full(C * P, c), key_chunk)
+        np.testing.assert_allclose(outs[c][0], want, rtol=0, atol=1e-12)
+        np.testing.assert_allclose(outs[c][1], want_lse, rtol=0, atol=1e-12)
+
+
+def test_short_window_equals_flat_attention_over_literal_cache(oracle_mod):
+    """With eviction: equals library-softmax attention over sink + last W frames."""
+    C, S, W, gh, gw, H, D = 2, 2, 4, 2, 2, 2, 16
+    P = gh * gw
+    o = oracle_mod.Oracle(1, H, D, P, C, S, W)
+    outs, hq, hk, hv = stream(o, 7, gh, gw, 200)
+    keys, vals = np.concatenate(hk), np.concatenate(hv)
+    differs = False
+    for c in range(7):
+        frames = literal_cache_frames((c + 1) * C, S, W)
+        idx = np.concatenate([np.arange(f * P, (f + 1) * P) for f in frames])
+        s = np.einsum("qhd,khd->hqk", hq[c], keys[idx]) / np.sqrt(D)
+        want = np.einsum("hqk,khd->qhd", softmax(s, axis=-1), vals[idx])
+        np.testing.assert_allclose(outs[c][0], want, rtol=0, atol=1e-12)
+        full, _ = flat_block_causal(hq[c], keys, vals, np.full(C * P, c), np.repeat(np.arange(7), C * P))
+        differs |= np.abs(full - want).max() > 1e-6
+    assert differs      # once frames are evicted the result is not full attention
+
+
+def test_single_visible_key_returns_its_value(oracle_mod):
+    o = oracle_mod.Oracle(1, 2, 8, 1, 1, 1, 2)
+    q, k, v = rand((1, 2, 8), 1), rand((1, 2, 8), 2), rand((1, 2, 8), 3)
+    o.append(0, k, v, 0, 1, 1)
+    out, lse = o.attn(0, o.rope_q(q, 0, 1, 1), 0)
+    np.testing.assert_array_equal(out, v)
+    np.testing.assert_allclose(lse[0], np.einsum("hd,hd->h", q[0], k[0]) / np.sqrt(8), atol=1e-13)
+
+
+def test_softmax_rows_sum_to_one_and_keys_are_the_resident_rows(oracle_mod):
+    C, S, W, gh, gw, H, D = 1, 1, 2, 4, 4, 2, 64
+    P = gh * gw
+    o = oracle_mod.Oracle(1, H, D, P, C, S, W)
+    for c in range(6):
+        q, k, v = (rand((P, H, D), 300 + 3 * c + i) for i in range(3))
+        o.append(0, k, v, c, gh, gw)
+        qr = o.rope_q(q, c, gh, gw)
+        out, lse = o.attn(0, qr, c)
+        K, V = o.read_layer()
+        for row in (0, P - 1):
+            for h in range(H):
+                p, kr = o.attn_probs(0, qr, c, row, h)
+                assert abs(p.sum() - 1.0) < 1e-12
+                frames = literal_cache_frames(c + 1, S, W)
+                want_rows = sorted(o.slot_of(f) * P + n for f in frames for n in range(P))
+                assert sorted(kr) == want_rows
+                vv = V.reshape(-1, H, D)[kr, h]
+                np.testing.assert_allclose(p @ vv, out[row, h], atol=1e-12)
+                kk = K.reshape(-1, H, D)[kr, h]
+                s = kk @ qr[row, h] / np.sqrt(D)
+                np.testing.assert_allclose(logsumexp(s), lse[row, h], atol=1e-12)
+
+
+def test_zero_keys_give_visible_histogram(oracle_mod):
+    """K == 0: uniform weights, so with V = one-hot(frame id) the output is the
+    histogram of visible frames; with V constant the output is that constant."""
+    C, S, W, gh, gw, H = 3, 3, 9, 2, 2, 1
+    P = gh * gw
+    D = 32
+    o = oracle_mod.Oracle(1, H, D, P, C, S, W)
+    for c in range(8):
+        k = np.zeros((C * P, H, D))
+        v = np.zeros((C * P, H, D))
+        for i in range(C):
+            v[i * P:(i + 1) * P, :, c * C + i] = 1.0
+        o.append(0, k, v, c * C, gh, gw)
+        out, lse = o.attn(0, rand((C * P, H, D), c), c * C)
+        frames = literal_cache_frames((c + 1) * C, S, W)
+        want = np.zeros(D)
+        want[frames] = 1.0 / len(frames)
+        np.testing.assert_allclose(out, np.broadcast_to(want, out.shape), atol=1e-15)
+        np.testing.assert_allclose(lse, np.log(len(frames) * P), atol=1e-13)
+    o2 = oracle_mod.Oracle(1, H, D, P, C, S, W)
+    for c in range(5):
+        o2.append(0, rand((C * P, H, D), 40 + c), np.full((C * P, H, D), 0.75), c * C, gh, gw)
+        out, _ = o2.attn(0, rand((C * P, H, D), c), c * C)
+        np.testing.assert_allclose(out, 0.75, atol=1e-14)
+
+
+def test_recache_equals_streaming_when_nothing_was_evicted(oracle_mod):
+    """Bulk block-causal recache over chunks 1..k == attending them one by one."""
+    C, S, W, gh, gw, H, D = 2, 2, 6, 2, 2, 2, 16
+    P = gh * gw
+    o = oracle_mod.Oracle(1, H, D, P, C, S, W)
+    qs, ks, vs, outs = [], [], [], []
+    for c in range(4):                       # sink chunk + 3 ring chunks, no eviction
+        q, k, v = (rand((C * P, H, D), 500 + 3 * c + i) for i in range(3))
+        o.append(0, k, v, c * C, gh, gw)
+        outs.append(o.attn(0, o.rope_q(q, c * C, gh, gw), c * C))
+        qs.append(q); ks.append(k); vs.append(v)
+    before = o.state()
+    qr, out, lse = o.recache(0, np.concatenate(qs[1:]), np.concatenate(ks[1:]),
+                             np.concatenate(vs[1:]), 3 * C, gh, gw)
+    after = o.state()
+    assert before["end"] == after["end"] and np.array_equal(before["slot_frame"], after["slot_frame"])
+    np.testing.assert_allclose(out, np.concatenate([x[0] for x in outs[1:]]), atol=1e-13)
+    np.testing.assert_allclose(lse, np.concatenate([x[1] for x in outs[1:]]), atol=1e-13)
+
+
+def test_recache_after_wraparound_matches_flat_reference(oracle_mod):
+    """Ring wrapped: recache rows see sink + window frames up to their own chunk."""
+    C, S, W, gh, gw, H, D = 1, 1, 3, 2, 2, 2, 16
+    P = gh * gw
+    o = oracle_mod.Oracle(1, H, D, P, C, S, W)
+    sink_k = sink_v = None
+    for c in range(6):
+        k, v = rand((P, H, D), 700 + c), rand((P, H, D), 800 + c)
+        o.append(0, k, v, c, gh, gw)
+        if c == 0:
+            sink_k, sink_v = oracle_mod.rope(k, 0, gh, gw), v
+    q, k, v = (rand((W * P, H, D), 900 + i) for i in range(3))
+    qr, out, lse = o.recache(0, q, k, v, W, gh, gw)
+    r0 = 6 - W
+    kr = oracle_mod.rope(k, r0, gh, gw)
+    np.testing.assert_allclose(qr, oracle_mod.rope(q, r0, gh, gw), atol=0)
+    keys = np.concatenate([sink_k, kr]); vals = np.concatenate([sink_v, v])
+    key_chunk = np.concatenate([np.full(P, -1), np.repeat(np.arange(W), P)])
+    want, want_lse = flat_block_causal(qr, keys, vals, np.repeat(np.arange(W), P), key_chunk)
+    np.testing.assert_allclose(out, want, atol=1e-12)
+    np.testing.assert_allclose(lse, want_lse, atol=1e-12)
+    # the next chunk then attends over the rebuilt ring
+    q2, k2, v2 = (rand((P, H, D), 950 + i) for i in range(3))
+    o.append(0, k2, v2, 6, gh, gw)
+    out2, _ = o.attn(0, o.rope_q(q2, 6, gh, gw), 6)
+    keys2 = np.concatenate([sink_k, kr[P:], oracle_mod.rope(k2, 6, gh, gw)])
+    vals2 = np.concatenate([sink_v, v[P:], v2])
+    s = np.einsum("qhd,khd->hqk", oracle_mod.rope(q2, 6, gh, gw), keys2) / np.sqrt(D)
+    np.testing.assert_allclose(out2, np.einsum("hqk,khd->qhd", softmax(s, -1), vals2), atol=1e-12)
+
+
+def test_recache_with_only_sink_is_a_noop(oracle_mod):
+    o = oracle_mod.Oracle(1, 1, 4, 1, 2, 2, 4)
+    x = np.zeros((2, 1, 4))
+    o.append(0, x, x, 0, 1, 1)
+    e = np.zeros((0, 1, 4))
+    qr, out, lse = o.recache(0, e, e, e, 0, 1, 1)
+    assert out.shape[0] == 0
+    with pytest.raises(oracle_mod.OracleError):
+        o.recache(0, x, x, x, 2, 1, 1)
+
+
+def test_sampled_rows_equal_full_evaluation(oracle_mod):
+    C, S, W, gh, gw, H, D = 2, 2, 4, 2, 3, 2, 16
+    P = gh * gw
+    o = oracle_mod.Oracle(1, H, D, P, C, S, W)
+    for c in range(4):
+        q, k, v = (rand((C * P, H, D), 600 + 3 * c + i) for i in range(3))
+        o.append(0, k, v, c * C, gh, gw)
+    qr = o.rope_q(q, 3 * C, gh, gw)
+    full, lse = o.attn(0, qr, 3 * C)
+    rows = np.array([0, 5, C * P - 1])
+    part, lse_p = o.attn(0, qr, 3 * C, rows=rows)
+    np.testing.assert_array_equal(part, full[rows])
+    np.testing.assert_array_equal(lse_p, lse[rows])
+
+
+def test_faithful_mode_rounds_stored_keys_only(oracle_mod):
+    C, S, W, gh, gw, H, D = 1, 1, 2, 2, 2, 1, 64
+    P = gh * gw
+    a = oracle_mod.Oracle(1, H, D, P, C, S, W, faithful=False)
+    b = oracle_mod.Oracle(1, H, D, P, C, S, W, faithful=True)
+    k, v = rand((P, H, D), 1), rand((P, H, D), 2)
+    a.append(0, k, v, 0, gh, gw); b.append(0, k, v, 0, gh, gw)
+    Ka, Va = a.read_layer(); Kb, Vb = b.read_layer()
+    np.testing.assert_array_equal(Va, Vb)
+    np.testing.assert_array_equal(Kb[0], oracle_mod.round_bf16(Ka[0]))
+    assert np.abs(Ka[0] - Kb[0]).max() <= 2.0 ** -8 * np.abs(Ka[0]).max()
+
+
+def test_ring_fills_from_its_first_slot(oracle_mod):
+    """The slot contract: while the ring is filling, resident frames are a
+    contiguous prefix of the storage (frame f sits in slot f), and the first
+    evicted frame is the oldest window frame."""
+    C, S, W = 3, 3, 9
+    o = oracle_mod.Oracle(1, 1, 2, 1, C, S, W)
+    x = np.zeros((C, 1, 2))
+    for chunk in range(4):
+        o.append(0, x, x, chunk * C, 1, 1)
+        sf = list(o.state()["slot_frame"])
+        end = (chunk + 1) * C
+        assert sf == list(range(end)) + [-1] * (S + W - end)
+    o.append(0, x, x, 12, 1, 1)      # frames 12..14 replace frames 3..5 in place
+    assert list(o.state()["slot_frame"]) == [0, 1, 2, 12, 13, 14, 6, 7, 8, 9, 10, 11]
+    assert o.state()["evictions"] == 3

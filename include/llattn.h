@@ -1,0 +1,196 @@
+/*
+ * llattn - sink+window attention over a rolling per-layer KV cache (sm_100a).
+ *
+ * C ABI of the inference hot path of a causal, chunk-wise autoregressive video
+ * generator that keeps the first frame chunk as a permanent attention sink and
+ * a short rolling window of recent frames (Sec. 3.3 "Short-window Attention",
+ * "Frame Sink"), and rebuilds the window on a prompt switch (Sec. 3.1 "KV
+ * Recache"; Algorithm 2).
+ *
+ * Conventions for every call
+ *   - Return value: LL_OK (0) or a negative LL_ERR_* code.  On any error the
+ *     cache's integer state is unchanged and ll_last_error() (thread-local)
+ *     describes the failure.
+ *   - "device" pointers are CUDA global memory owned by the caller, contiguous
+ *     and 16-byte aligned; "host" pointers are ordinary process memory.
+ *   - bf16 tensors are bfloat16 bit patterns.  Activations are token-major
+ *     [tokens, heads, head_dim]; token n of a frame is grid cell
+ *     (y, x) = (n / grid_w, n % grid_w).
+ *   - Kernels are enqueued on the caller's stream and the call returns without
+ *     synchronising.  The integer state lives on the host inside the handle
+ *     and is updated by the call itself, so calls on one handle must be issued
+ *     in program order from one thread, on one stream (or on streams the caller
+ *     orders).  Handles are independent of each other.
+ *   - No CPU fallback exists: without a CUDA device the compute calls fail with
+ *     LL_ERR_CUDA.
+ */
+#ifndef LLATTN_H
+#define LLATTN_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct ll_cache ll_cache;   /* opaque; owned by the library */
+typedef void *ll_stream;            /* a cudaStream_t (NULL = default stream) */
+typedef uint16_t ll_bf16;           /* bfloat16 bit pattern */
+
+enum {
+    LL_OK = 0,
+    LL_ERR_INVALID_ARG = -1,        /* null/misaligned pointer, bad layer, bad size */
+    LL_ERR_BAD_POSITION = -2,       /* frame_start / n_frames do not fit the stream state */
+    LL_ERR_UNSUPPORTED_SHAPE = -3,  /* shape outside what the kernels were built for */
+    LL_ERR_NO_STORAGE = -4,         /* compute call before ll_cache_bind_storage */
+    LL_ERR_CUDA = -5,               /* a CUDA runtime/driver call failed */
+    LL_ERR_DEVICE_TIMEOUT = -6      /* a kernel gave up on a bounded wait (see ll_cache_device_status) */
+};
+
+#define LL_MAX_SLOTS 64             /* sink_frames + window_frames <= LL_MAX_SLOTS */
+#define LL_MAX_RANGES 4             /* contiguous cache-row runs a query group can see */
+
+/* Integer state of one layer's cache.  Bit-exact contract:
+ *   frame f lives in slot f if f < S, else in slot S + (f - S) mod W;
+ *   slot_frame[slot] is the absolute frame held there, -1 if empty.          */
+typedef struct ll_state {
+    int64_t end;                        /* frames appended so far */
+    int32_t n_slots;                    /* S + W */
+    int32_t ring_valid;                 /* ring slots that hold a frame */
+    int32_t slot_frame[LL_MAX_SLOTS];
+    int64_t n_appends;                  /* new-chunk appends */
+    int64_t n_overwrites;               /* overwrite-newest appends */
+    int64_t n_evictions;                /* frames replaced by a newer frame */
+    int64_t n_recaches;
+    int64_t n_attn_calls;
+} ll_state;
+
+/* ---- lifetime ----------------------------------------------------------- */
+
+/* Create the host-side handle of one stream's cache: `layers` independent
+ * per-layer caches of S = sink_frames pinned frames (Sec. 3.3 "Frame Sink")
+ * plus a ring of W = window_frames frames (Sec. 3.3 "Short-window Attention";
+ * W counts the chunk being generated), tokens_per_frame tokens each.
+ * Requires head_dim in {64, 128}; chunk_frames >= 1; sink_frames and
+ * window_frames multiples of chunk_frames; window_frames >= chunk_frames;
+ * sink_frames + window_frames <= LL_MAX_SLOTS; window_frames / chunk_frames <= 24;
+ * else LL_ERR_UNSUPPORTED_SHAPE.  Touches no device.  *out is owned by the
+ * library until ll_cache_destroy. */
+int ll_cache_create(int layers, int heads, int head_dim, int tokens_per_frame,
+                    int chunk_frames, int sink_frames, int window_frames, ll_cache **out);
+
+/* Frees the handle (host memory only; bound storage stays the caller's). */
+void ll_cache_destroy(ll_cache *cache);
+
+/* Bytes of device memory the caller must provide: a small aux block (status
+ * words, RoPE tables) followed by, per layer, K then V as
+ * [heads][(S+W)*tokens_per_frame rows][head_dim] bf16, sink rows first. */
+size_t ll_cache_storage_bytes(const ll_cache *cache);
+
+/* Attach caller-owned device memory (`dev`, >= ll_cache_storage_bytes, 1024-byte
+ * aligned).  Zero-fills it on `stream` (rows of empty slots may be fetched by
+ * partially valid tiles and must hold finite numbers) and encodes the TMA
+ * descriptors.  The memory must outlive every later call on the handle. */
+int ll_cache_bind_storage(ll_cache *cache, void *dev, size_t bytes, ll_stream stream);
+
+/* Byte offset, inside the bound storage, of head `head` of layer `layer`'s K
+ * (which = 0) or V (which = 1) matrix: (S+W)*tokens_per_frame rows of head_dim
+ * bf16, row = slot * tokens_per_frame + token.  For tests and checkpointing. */
+int ll_cache_kv_offset(const ll_cache *cache, int layer, int which, int head, size_t *offset);
+
+/* ---- the hot path --------------------------------------------------------- */
+
+/* Fused 3-D RoPE + K/V append (Algorithm 2: every pass of a chunk writes the
+ * chunk's K/V into the cache before attending; the final clean pass commits it.
+ * Slot rule: Sec. 3.3 "Frame Sink").
+ *   q, k, v   device, bf16 [n_frames*grid_h*grid_w, heads, head_dim]; q may be
+ *             NULL when q_out is NULL.
+ *   q_out     device, same shape as q, nullable: receives RoPE(q) (may alias q).
+ *   n_frames  must equal chunk_frames; grid_h*grid_w must equal tokens_per_frame.
+ *   frame_start == end      : a new chunk; evicts the frames W behind it, end += C.
+ *   frame_start == end - C  : overwrites the newest chunk in place (state unchanged).
+ *   anything else           : LL_ERR_BAD_POSITION.
+ * RoPE: the D/2 rotation pairs are split t|h|w with n_h = n_w = D/6 (floor) and
+ * n_t = D/2 - 2*n_h pairs; pair j is elements (2j, 2j+1); pair i of an axis with
+ * n_a pairs turns by pos * rope_theta^(-i/n_a); t is the absolute frame index.
+ * K rows are stored rotated, V rows verbatim.  The arithmetic is fp32 on
+ * fp64-accurate sine/cosine tables kept in the aux block. */
+int ll_rope_append_kv(ll_cache *cache, int layer, const ll_bf16 *q, const ll_bf16 *k,
+                      const ll_bf16 *v, int64_t frame_start, int n_frames,
+                      int grid_h, int grid_w, float rope_theta, ll_bf16 *q_out,
+                      ll_stream stream);
+
+/* Sink+window attention of the newest chunk's queries (Sec. 3.3): every query
+ * attends to all sink rows and all resident window rows (the chunk itself
+ * included; bidirectional inside the chunk), softmax scale 1/sqrt(head_dim).
+ *   q_roped   device, bf16 [n_q_frames*tokens_per_frame, heads, head_dim], after RoPE.
+ *   q_frame_start must equal end - C and n_q_frames must equal C.
+ *   out       device, bf16, same shape as q_roped.
+ *   lse_out   device, float [heads, n_q_frames*tokens_per_frame], nullable:
+ *             natural-log softmax denominators.
+ * QK^T and PV run on tcgen05 tensor cores with fp32 accumulation in TMEM; the
+ * softmax is fp32. */
+int ll_sink_window_attn(ll_cache *cache, int layer, const ll_bf16 *q_roped,
+                        int64_t q_frame_start, int n_q_frames, ll_bf16 *out,
+                        float *lse_out, ll_stream stream);
+
+/* KV-recache (Sec. 3.1; Sec. 3.3 last paragraph: only the most recent W frames
+ * are rebuilt; the sink is left alone).  q, k, v hold fresh activations for the
+ * resident window frames [r0, end), r0 = max(S, end - W), oldest first.
+ *   n_frames  must equal end - r0 (0 while only sink frames exist: no work).
+ * Re-ropes and overwrites those frames' ring rows (slot table and end
+ * unchanged), then attends all their queries block-causally: a query of chunk c
+ * sees the sink and window frames [r0, (c+1)*C).  out/lse_out as above with
+ * n_frames*tokens_per_frame rows; q_out nullable receives RoPE(q). */
+int ll_recache(ll_cache *cache, int layer, const ll_bf16 *q, const ll_bf16 *k,
+               const ll_bf16 *v, int n_frames, int grid_h, int grid_w, float rope_theta,
+               ll_bf16 *q_out, ll_bf16 *out, float *lse_out, ll_stream stream);
+
+/* Forget everything in every layer (Algorithm 2 "C <- []"): end = 0, all slots
+ * empty, counters kept.  Stored bytes are not cleared. */
+int ll_cache_reset(ll_cache *cache);
+
+/* ---- state, diagnostics ----------------------------------------------------- */
+
+int ll_cache_get_state(const ll_cache *cache, int layer, ll_state *out);
+
+/* Restore a state saved by ll_cache_get_state (checkpoint/resume); validates
+ * that every resident frame sits in the slot the slot rule gives it. */
+int ll_cache_set_state(ll_cache *cache, int layer, const ll_state *state);
+
+/* Cache-row runs [start, start+len) (row = slot*tokens_per_frame + token) that
+ * the queries of frames [q_frame_start, q_frame_start + chunk_frames) can see
+ * given the current state; lo_floor hides window frames older than it (pass 0
+ * for decode).  Writes up to LL_MAX_RANGES pairs, returns the count in
+ * *n_ranges.  Host-only; used by the attention calls and by tests. */
+int ll_cache_visible_ranges(const ll_cache *cache, int layer, int64_t q_frame_start,
+                            int64_t lo_floor, int64_t *starts, int64_t *lens, int *n_ranges);
+
+/* Bookkeeping-only mode (on != 0): compute calls validate arguments and update
+ * the integer state but launch nothing and need no device or storage.  For
+ * planning and host-side tests; outputs are NOT produced. */
+int ll_cache_set_dry_run(ll_cache *cache, int on);
+
+/* Synchronise `stream`, read the aux status words and clear them.  LL_OK, or
+ * LL_ERR_DEVICE_TIMEOUT if a kernel abandoned a bounded wait (its outputs are
+ * then invalid); ll_last_error() names the role and barrier. */
+int ll_cache_device_status(ll_cache *cache, ll_stream stream);
+
+/* Test-only triage kernel: the same computation as ll_sink_window_attn with one
+ * thread block per (query row, head) and plain fp32 FMAs.  Never used by the
+ * calls above. */
+int ll_debug_attn_simt(ll_cache *cache, int layer, const ll_bf16 *q_roped,
+                       int64_t q_frame_start, int n_q_frames, ll_bf16 *out,
+                       float *lse_out, ll_stream stream);
+
+/* Kernel launches made by this process through the library so far. */
+int64_t ll_launch_count(void);
+
+const char *ll_last_error(void);
+const char *ll_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* LLATTN_H */

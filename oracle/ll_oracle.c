@@ -99,11 +99,12 @@ void llo_destroy(llo *o)
 }
 
 /* Reset (Algorithm 2, "initialise KV cache C <- []"): every layer forgets
- * everything; stored bytes need not be cleared. */
+ * everything; stored bytes need not be cleared.  The eviction count is a
+ * lifetime diagnostic and keeps running. */
 int llo_reset(llo *o)
 {
     if (!o) return LLO_ERR_ARG;
-    for (int l = 0; l < o->L; ++l) { o->end[l] = 0; o->evictions[l] = 0; }
+    for (int l = 0; l < o->L; ++l) o->end[l] = 0;
     for (size_t i = 0; i < (size_t)o->L * slots(o); ++i) o->slot_frame[i] = -1;
     return LLO_OK;
 }

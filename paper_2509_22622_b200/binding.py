@@ -1,0 +1,262 @@
+"""ctypes binding of ``libllattn.so``: same names as the C ABI, argument marshalling only.
+
+Every step of the path runs in the library's CUDA kernels.  PyTorch is used
+for device memory and streams; nothing here computes.  If the shared library
+has not been built, importing the binding's functions raises: there is no
+fallback.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+
+HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(HERE, "libllattn.so")
+
+LL_OK = 0
+LL_ERR_INVALID_ARG = -1
+LL_ERR_BAD_POSITION = -2
+LL_ERR_UNSUPPORTED_SHAPE = -3
+LL_ERR_NO_STORAGE = -4
+LL_ERR_CUDA = -5
+LL_ERR_DEVICE_TIMEOUT = -6
+LL_MAX_SLOTS = 64
+LL_MAX_RANGES = 4
+
+
+class ll_state(C.Structure):
+    _fields_ = [
+        ("end", C.c_int64),
+        ("n_slots", C.c_int32),
+        ("ring_valid", C.c_int32),
+        ("slot_frame", C.c_int32 * LL_MAX_SLOTS),
+        ("n_appends", C.c_int64),
+        ("n_overwrites", C.c_int64),
+        ("n_evictions", C.c_int64),
+        ("n_recaches", C.c_int64),
+        ("n_attn_calls", C.c_int64),
+    ]
+
+
+class LLError(RuntimeError):
+    def __init__(self, code: int, message: str):
+        super().__init__("llattn error %d: %s" % (code, message))
+        self.code = code
+
+
+_lib = None
+
+# name -> (restype, argtypes); also the list of symbols include/llattn.h declares
+SIGNATURES = {
+    "ll_cache_create": (C.c_int, [C.c_int] * 7 + [C.POINTER(C.c_void_p)]),
+    "ll_cache_destroy": (None, [C.c_void_p]),
+    "ll_cache_storage_bytes": (C.c_size_t, [C.c_void_p]),
+    "ll_cache_bind_storage": (C.c_int, [C.c_void_p, C.c_void_p, C.c_size_t, C.c_void_p]),
+    "ll_cache_kv_offset": (C.c_int, [C.c_void_p, C.c_int, C.c_int, C.c_int, C.POINTER(C.c_size_t)]),
+    "ll_rope_append_kv": (C.c_int, [C.c_void_p, C.c_int, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int64,
+                                    C.c_int, C.c_int, C.c_int, C.c_float, C.c_void_p, C.c_void_p]),
+    "ll_sink_window_attn": (C.c_int, [C.c_void_p, C.c_int, C.c_void_p, C.c_int64, C.c_int, C.c_void_p,
+                                      C.c_void_p, C.c_void_p]),
+    "ll_recache": (C.c_int, [C.c_void_p, C.c_int, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int, C.c_int,
+                             C.c_int, C.c_float, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]),
+    "ll_cache_reset": (C.c_int, [C.c_void_p]),
+    "ll_cache_get_state": (C.c_int, [C.c_void_p, C.c_int, C.POINTER(ll_state)]),
+    "ll_cache_set_state": (C.c_int, [C.c_void_p, C.c_int, C.POINTER(ll_state)]),
+    "ll_cache_visible_ranges": (C.c_int, [C.c_void_p, C.c_int, C.c_int64, C.c_int64, C.POINTER(C.c_int64),
+                                          C.POINTER(C.c_int64), C.POINTER(C.c_int)]),
+    "ll_cache_set_dry_run": (C.c_int, [C.c_void_p, C.c_int]),
+    "ll_cache_device_status": (C.c_int, [C.c_void_p, C.c_void_p]),
+    "ll_debug_attn_simt": (C.c_int, [C.c_void_p, C.c_int, C.c_void_p, C.c_int64, C.c_int, C.c_void_p,
+                                     C.c_void_p, C.c_void_p]),
+    "ll_launch_count": (C.c_int64, []),
+    "ll_last_error": (C.c_char_p, []),
+    "ll_version": (C.c_char_p, []),
+}
+
+
+def lib():
+    """Load the shared library (fails loudly when it is missing)."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise RuntimeError(
+                "%s is missing: build it with `python -m paper_2509_22622_b200.build` "
+                "(there is no CPU or PyTorch fallback)" % LIB_PATH)
+        L = C.CDLL(LIB_PATH)
+        for name, (res, args) in SIGNATURES.items():
+            fn = getattr(L, name)
+            fn.restype = res
+            fn.argtypes = args
+        _lib = L
+    return _lib
+
+
+def _check(code: int):
+    if code != LL_OK:
+        raise LLError(code, lib().ll_last_error().decode())
+
+
+def _ptr(t):
+    """Device (or host) address of a torch tensor, None -> NULL."""
+    return None if t is None else C.c_void_p(t.data_ptr())
+
+
+def _stream(stream):
+    if stream is None:
+        import torch
+        if not torch.cuda.is_available():      # bookkeeping-only handles never launch
+            return C.c_void_p(0)
+        return C.c_void_p(torch.cuda.current_stream().cuda_stream)
+    return C.c_void_p(stream if isinstance(stream, int) else stream.cuda_stream)
+
+
+# ---- the C ABI, one Python function per entry point -----------------------------
+
+def ll_cache_create(layers, heads, head_dim, tokens_per_frame, chunk_frames, sink_frames, window_frames):
+    h = C.c_void_p()
+    _check(lib().ll_cache_create(layers, heads, head_dim, tokens_per_frame, chunk_frames, sink_frames,
+                                 window_frames, C.byref(h)))
+    return h
+
+
+def ll_cache_destroy(h):
+    lib().ll_cache_destroy(h)
+
+
+def ll_cache_storage_bytes(h) -> int:
+    return lib().ll_cache_storage_bytes(h)
+
+
+def ll_cache_bind_storage(h, storage, stream=None):
+    _check(lib().ll_cache_bind_storage(h, _ptr(storage), storage.numel() * storage.element_size(), _stream(stream)))
+
+
+def ll_cache_kv_offset(h, layer, which, head) -> int:
+    off = C.c_size_t()
+    _check(lib().ll_cache_kv_offset(h, layer, which, head, C.byref(off)))
+    return off.value
+
+
+def ll_rope_append_kv(h, layer, q, k, v, frame_start, n_frames, grid_h, grid_w, rope_theta=10000.0,
+                      q_out=None, stream=None):
+    _check(lib().ll_rope_append_kv(h, layer, _ptr(q), _ptr(k), _ptr(v), frame_start, n_frames, grid_h, grid_w,
+                                   rope_theta, _ptr(q_out), _stream(stream)))
+
+
+def ll_sink_window_attn(h, layer, q_roped, q_frame_start, n_q_frames, out, lse_out=None, stream=None):
+    _check(lib().ll_sink_window_attn(h, layer, _ptr(q_roped), q_frame_start, n_q_frames, _ptr(out),
+                                     _ptr(lse_out), _stream(stream)))
+
+
+def ll_debug_attn_simt(h, layer, q_roped, q_frame_start, n_q_frames, out, lse_out=None, stream=None):
+    _check(lib().ll_debug_attn_simt(h, layer, _ptr(q_roped), q_frame_start, n_q_frames, _ptr(out),
+                                    _ptr(lse_out), _stream(stream)))
+
+
+def ll_recache(h, layer, q, k, v, n_frames, grid_h, grid_w, rope_theta, q_out, out, lse_out=None, stream=None):
+    _check(lib().ll_recache(h, layer, _ptr(q), _ptr(k), _ptr(v), n_frames, grid_h, grid_w, rope_theta,
+                            _ptr(q_out), _ptr(out), _ptr(lse_out), _stream(stream)))
+
+
+def ll_cache_reset(h):
+    _check(lib().ll_cache_reset(h))
+
+
+def ll_cache_get_state(h, layer=0) -> ll_state:
+    st = ll_state()
+    _check(lib().ll_cache_get_state(h, layer, C.byref(st)))
+    return st
+
+
+def ll_cache_set_state(h, layer, st: ll_state):
+    _check(lib().ll_cache_set_state(h, layer, C.byref(st)))
+
+
+def ll_cache_visible_ranges(h, layer, q_frame_start, lo_floor=0):
+    starts = (C.c_int64 * LL_MAX_RANGES)()
+    lens = (C.c_int64 * LL_MAX_RANGES)()
+    n = C.c_int()
+    _check(lib().ll_cache_visible_ranges(h, layer, q_frame_start, lo_floor, starts, lens, C.byref(n)))
+    return [(starts[i], lens[i]) for i in range(n.value)]
+
+
+def ll_cache_set_dry_run(h, on: bool):
+    _check(lib().ll_cache_set_dry_run(h, int(on)))
+
+
+def ll_cache_device_status(h, stream=None):
+    _check(lib().ll_cache_device_status(h, _stream(stream)))
+
+
+def ll_launch_count() -> int:
+    return lib().ll_launch_count()
+
+
+def ll_version() -> str:
+    return lib().ll_version().decode()
+
+
+# ---- a small convenience owner ---------------------------------------------------
+
+class Cache:
+    """Owns a handle plus the torch tensor that backs it.  Marshalling only."""
+
+    def __init__(self, layers, heads, head_dim, tokens_per_frame, chunk_frames, sink_frames, window_frames,
+                 device="cuda:0", dry_run=False):
+        self.L, self.H, self.D, self.P = layers, heads, head_dim, tokens_per_frame
+        self.C, self.S, self.W = chunk_frames, sink_frames, window_frames
+        self.h = ll_cache_create(layers, heads, head_dim, tokens_per_frame, chunk_frames, sink_frames,
+                                 window_frames)
+        self.storage = None
+        if dry_run:
+            ll_cache_set_dry_run(self.h, True)
+        else:
+            import torch
+            if not torch.cuda.is_available():
+                raise RuntimeError("llattn needs a CUDA device; there is no CPU fallback")
+            nbytes = ll_cache_storage_bytes(self.h)
+            # over-allocate so the bound address can be rounded up to 1024 bytes
+            self._raw = torch.empty(nbytes + 1024, dtype=torch.uint8, device=device)
+            shift = (-self._raw.data_ptr()) % 1024
+            self.storage = self._raw[shift:shift + nbytes]
+            ll_cache_bind_storage(self.h, self.storage)
+
+    def close(self):
+        if self.h is not None:
+            ll_cache_destroy(self.h)
+            self.h = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    def state(self, layer=0):
+        st = ll_cache_get_state(self.h, layer)
+        return {"end": st.end, "slot_frame": list(st.slot_frame[:st.n_slots]), "ring_valid": st.ring_valid,
+                "evictions": st.n_evictions, "appends": st.n_appends, "overwrites": st.n_overwrites,
+                "recaches": st.n_recaches, "attn_calls": st.n_attn_calls}
+
+    def kv_view(self, layer, which):
+        """bf16 view [H, rows, D] of a layer's K (which=0) or V (which=1) matrix."""
+        import torch
+        rows = (self.S + self.W) * self.P
+        off = ll_cache_kv_offset(self.h, layer, which, 0)
+        n = self.H * rows * self.D * 2
+        return self.storage[off:off + n].view(torch.bfloat16).view(self.H, rows, self.D)
+
+    def rope_append_kv(self, layer, q, k, v, frame_start, grid_h, grid_w, theta=10000.0, q_out=None, stream=None):
+        ll_rope_append_kv(self.h, layer, q, k, v, frame_start, self.C, grid_h, grid_w, theta, q_out, stream)
+
+    def sink_window_attn(self, layer, q_roped, q_frame_start, out, lse_out=None, stream=None):
+        ll_sink_window_attn(self.h, layer, q_roped, q_frame_start, self.C, out, lse_out, stream)
+
+    def recache(self, layer, q, k, v, n_frames, grid_h, grid_w, theta, q_out, out, lse_out=None, stream=None):
+        ll_recache(self.h, layer, q, k, v, n_frames, grid_h, grid_w, theta, q_out, out, lse_out, stream)
+
+    def reset(self):
+        ll_cache_reset(self.h)
+
+    def check_device(self, stream=None):
+        ll_cache_device_status(self.h, stream)

@@ -1,0 +1,525 @@
+// Host side of the library: handle, integer cache state, argument checks,
+// TMA descriptor encoding and kernel dispatch.  No tensor arithmetic here.
+#include <algorithm>
+#include <atomic>
+#include <cmath>
+#include <cstdarg>
+#include <cstdio>
+#include <cstring>
+
+#include "ll_internal.h"
+
+namespace {
+
+thread_local std::string g_err;
+std::atomic<int64_t> g_launches{0};
+
+int fail(int code, const char *fmt, ...)
+{
+    char buf[512];
+    va_list ap;
+    va_start(ap, fmt);
+    vsnprintf(buf, sizeof buf, fmt, ap);
+    va_end(ap);
+    g_err = buf;
+    return code;
+}
+
+int cuda_fail(cudaError_t e, const char *what)
+{
+    return fail(LL_ERR_CUDA, "%s: %s", what, cudaGetErrorString(e));
+}
+
+size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+void rope_split(int D, int *n_t, int *n_h)
+{
+    *n_h = D / 6;
+    *n_t = D / 2 - 2 * (D / 6);
+}
+
+// Slot rule: sink frames are pinned, later frames roll through the ring.
+int slot_of(const ll_cache *c, int64_t f)
+{
+    return f < c->S ? (int)f : c->S + (int)((f - c->S) % c->W);
+}
+
+bool layer_ok(const ll_cache *c, int layer) { return c && layer >= 0 && layer < c->L; }
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *,
+                                  const cuuint64_t *, const cuuint64_t *, const cuuint32_t *,
+                                  const cuuint32_t *, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_fn()
+{
+    static EncodeTiledFn fn = nullptr;
+    static bool tried = false;
+    if (!tried) {
+        tried = true;
+        void *p = nullptr;
+        cudaDriverEntryPointQueryResult qr;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qr) == cudaSuccess &&
+            qr == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<EncodeTiledFn>(p);
+    }
+    return fn;
+}
+
+// 3-D bf16 tensor map with 128-byte swizzle; box = {64 elements, box1, box2}.
+int encode_map(CUtensorMap *m, const void *base, uint64_t d0, uint64_t d1, uint64_t d2,
+               uint64_t stride1_bytes, uint64_t stride2_bytes, uint32_t box1, uint32_t box2)
+{
+    EncodeTiledFn fn = encode_fn();
+    if (!fn) return fail(LL_ERR_CUDA, "cuTensorMapEncodeTiled is not available from the driver");
+    cuuint64_t dims[3] = {d0, d1, d2};
+    cuuint64_t strides[2] = {stride1_bytes, stride2_bytes};
+    cuuint32_t box[3] = {64, box1, box2};
+    cuuint32_t estr[3] = {1, 1, 1};
+    CUresult r = fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void *>(base), dims, strides,
+                    box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                    CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) return fail(LL_ERR_CUDA, "cuTensorMapEncodeTiled failed with CUresult %d", (int)r);
+    return LL_OK;
+}
+
+char *layer_k(const ll_cache *c, int layer) { return c->storage + c->aux_bytes + (size_t)layer * 2 * c->kv_bytes; }
+char *layer_v(const ll_cache *c, int layer) { return layer_k(c, layer) + c->kv_bytes; }
+
+// Visible cache-row runs for queries of the chunk holding q_frame_start.
+int visible_ranges(const ll_cache *c, int layer, int64_t q_frame_start, int64_t lo_floor,
+                   int64_t *starts, int64_t *lens, int *n_ranges)
+{
+    const ll::LayerState &st = c->layers[layer];
+    if (q_frame_start < 0 || q_frame_start >= st.end)
+        return fail(LL_ERR_BAD_POSITION, "query frame %lld is outside the stream [0, %lld)",
+                    (long long)q_frame_start, (long long)st.end);
+    const int64_t hi = (q_frame_start / c->C + 1) * c->C;
+    int64_t lo = std::max<int64_t>(std::max<int64_t>(c->S, hi - c->W), lo_floor);
+    bool seen[LL_MAX_SLOTS] = {false};
+    auto mark = [&](int64_t f) -> bool {
+        int s = slot_of(c, f);
+        if (st.slot_frame[s] != (int32_t)f) return false;
+        seen[s] = true;
+        return true;
+    };
+    for (int64_t f = 0; f < std::min<int64_t>(c->S, hi); ++f)
+        if (!mark(f)) return fail(LL_ERR_BAD_POSITION, "sink frame %lld is not resident", (long long)f);
+    for (int64_t f = lo; f < hi; ++f)
+        if (!mark(f)) return fail(LL_ERR_BAD_POSITION, "window frame %lld is not resident", (long long)f);
+    int n = 0;
+    for (int s = 0; s < c->n_slots;) {
+        if (!seen[s]) { ++s; continue; }
+        int e = s;
+        while (e < c->n_slots && seen[e]) ++e;
+        if (n >= LL_MAX_RANGES) return fail(LL_ERR_UNSUPPORTED_SHAPE, "visible set needs more than %d runs", LL_MAX_RANGES);
+        starts[n] = (int64_t)s * c->P;
+        lens[n] = (int64_t)(e - s) * c->P;
+        ++n;
+        s = e;
+    }
+    *n_ranges = n;
+    return LL_OK;
+}
+
+// Make sure the RoPE tables cover frames [f0, f1) and this grid/theta.
+int ensure_tables(ll_cache *c, int64_t f0, int64_t f1, int gh, int gw, float theta, cudaStream_t stream)
+{
+    int n_t, n_h;
+    rope_split(c->D, &n_t, &n_h);
+    bool do_hw = !(c->hw_valid && c->tab_gh == gh && c->tab_gw == gw && c->tab_theta == theta);
+    bool do_t = do_hw || c->t_base < 0 || f0 < c->t_base || f1 > c->t_base + ll::kTTabFrames;
+    if (!do_t && !do_hw) return LL_OK;
+    int64_t base = do_t ? f0 / ll::kTTabAlign * ll::kTTabAlign : c->t_base;
+    float2 *t_tab = reinterpret_cast<float2 *>(c->storage + c->off_ttab);
+    float2 *h_tab = reinterpret_cast<float2 *>(c->storage + c->off_hwtab);
+    float2 *w_tab = h_tab + (size_t)gh * n_h;
+    cudaError_t e = ll::launch_rope_tables(t_tab, base, ll::kTTabFrames, n_t, h_tab, gh, w_tab, gw, n_h,
+                                           theta, do_t, do_hw, stream);
+    if (e != cudaSuccess) return cuda_fail(e, "rope table kernel");
+    c->t_base = base;
+    c->hw_valid = true; c->tab_gh = gh; c->tab_gw = gw; c->tab_theta = theta;
+    return LL_OK;
+}
+
+int need_storage(const ll_cache *c)
+{
+    if (!c->storage) return fail(LL_ERR_NO_STORAGE, "no device storage bound (call ll_cache_bind_storage)");
+    return LL_OK;
+}
+
+int fill_rope_params(ll_cache *c, int layer, const ll_bf16 *q, const ll_bf16 *k, const ll_bf16 *v,
+                     ll_bf16 *q_out, int64_t frame_start, int n_frames, int gw, ll::RopeAppendParams *p)
+{
+    int n_t, n_h;
+    rope_split(c->D, &n_t, &n_h);
+    p->q = q; p->k = k; p->v = v; p->q_out = q_out;
+    p->kcache = reinterpret_cast<ll_bf16 *>(layer_k(c, layer));
+    p->vcache = reinterpret_cast<ll_bf16 *>(layer_v(c, layer));
+    const float2 *t_tab = reinterpret_cast<const float2 *>(c->storage + c->off_ttab);
+    p->t_tab = t_tab + (size_t)(frame_start - c->t_base) * n_t;
+    p->h_tab = reinterpret_cast<const float2 *>(c->storage + c->off_hwtab);
+    p->w_tab = p->h_tab + (size_t)c->tab_gh * n_h;
+    p->rows_per_head = c->rows;
+    p->n_tokens = n_frames * c->P;
+    p->heads = c->H; p->P = c->P; p->grid_w = gw;
+    p->n_t = n_t; p->n_h = n_h;
+    for (int i = 0; i < n_frames; ++i) p->slot[i] = slot_of(c, frame_start + i);
+    return LL_OK;
+}
+
+// Split a group's rows into query tiles and fill the launch parameters.
+int build_attn_params(ll_cache *c, int layer, const ll_bf16 *q, ll_bf16 *out, float *lse,
+                      int n_groups, const int64_t *group_frame_start, int64_t lo_floor,
+                      ll::AttnParams *p)
+{
+    if (n_groups > ll::kMaxGroups) return fail(LL_ERR_UNSUPPORTED_SHAPE, "more than %d query groups", ll::kMaxGroups);
+    memset(p, 0, sizeof *p);
+    p->n_groups = n_groups;
+    p->heads = c->H;
+    p->rows_per_head = c->rows;
+    p->scale_log2 = (float)(1.4426950408889634 / std::sqrt((double)c->D));
+    p->q = q; p->out = out; p->lse = lse;
+    p->kbase = reinterpret_cast<const ll_bf16 *>(c->storage ? layer_k(c, layer) : nullptr);
+    p->vbase = reinterpret_cast<const ll_bf16 *>(c->storage ? layer_v(c, layer) : nullptr);
+    p->status = reinterpret_cast<uint32_t *>(c->storage ? c->storage + c->off_status : nullptr);
+    const int rows_per_group = c->C * c->P;
+    int tile = 0;
+    for (int g = 0; g < n_groups; ++g) {
+        ll::AttnGroup &G = p->g[g];
+        G.q_begin = g * rows_per_group;
+        G.q_rows = rows_per_group;
+        G.tile_begin = tile;
+        tile += (rows_per_group + ll::kQTileRows - 1) / ll::kQTileRows;
+        int64_t starts[LL_MAX_RANGES], lens[LL_MAX_RANGES];
+        int n = 0;
+        int st = visible_ranges(c, layer, group_frame_start[g], lo_floor, starts, lens, &n);
+        if (st != LL_OK) return st;
+        G.n_ranges = n;
+        for (int r = 0; r < n; ++r) { G.k_start[r] = (int)starts[r]; G.k_len[r] = (int)lens[r]; }
+    }
+    p->nq_total = n_groups * rows_per_group;
+    p->total_qtiles = tile;
+    return LL_OK;
+}
+
+int launch_attention(ll_cache *c, int layer, const ll::AttnParams &p, cudaStream_t stream, bool simt)
+{
+    if (simt) {
+        cudaError_t e = ll::launch_attn_simt(p, c->D, stream);
+        return e == cudaSuccess ? LL_OK : cuda_fail(e, "simt attention kernel");
+    }
+    CUtensorMap qmap;
+    int st = encode_map(&qmap, p.q, (uint64_t)c->D, (uint64_t)c->H, (uint64_t)p.nq_total,
+                        (uint64_t)c->D * 2, (uint64_t)c->H * c->D * 2, 1, 128);
+    if (st != LL_OK) return st;
+    cudaError_t e = ll::launch_attn_sm100(p, c->D, qmap, c->kmap[layer], c->vmap[layer], stream);
+    return e == cudaSuccess ? LL_OK : cuda_fail(e, "sink+window attention kernel");
+}
+
+int attn_entry(ll_cache *c, int layer, const ll_bf16 *q_roped, int64_t q_frame_start, int n_q_frames,
+               ll_bf16 *out, float *lse_out, ll_stream stream, bool simt)
+{
+    if (!layer_ok(c, layer)) return fail(LL_ERR_INVALID_ARG, "bad cache handle or layer %d", layer);
+    ll::LayerState &st = c->layers[layer];
+    if (n_q_frames != c->C) return fail(LL_ERR_BAD_POSITION, "n_q_frames %d != chunk_frames %d", n_q_frames, c->C);
+    if (st.end < c->C || q_frame_start != st.end - c->C)
+        return fail(LL_ERR_BAD_POSITION, "queries must be the newest chunk: q_frame_start %lld, end %lld",
+                    (long long)q_frame_start, (long long)st.end);
+    if (!c->dry_run) {
+        if (!q_roped || !out) return fail(LL_ERR_INVALID_ARG, "null q_roped or out");
+        if (!aligned16(q_roped) || !aligned16(out) || (lse_out && !aligned16(lse_out)))
+            return fail(LL_ERR_INVALID_ARG, "q_roped/out/lse_out must be 16-byte aligned");
+        int s = need_storage(c);
+        if (s != LL_OK) return s;
+    }
+    ll::AttnParams p;
+    int s = build_attn_params(c, layer, q_roped, out, lse_out, 1, &q_frame_start, 0, &p);
+    if (s != LL_OK) return s;
+    if (!c->dry_run) {
+        s = launch_attention(c, layer, p, (cudaStream_t)stream, simt);
+        if (s != LL_OK) return s;
+    }
+    st.n_attn += 1;
+    return LL_OK;
+}
+
+}  // namespace
+
+namespace ll {
+void count_launch(int n) { g_launches.fetch_add(n, std::memory_order_relaxed); }
+}  // namespace ll
+
+extern "C" {
+
+const char *ll_last_error(void) { return g_err.c_str(); }
+const char *ll_version(void) { return "llattn 0.1 (sm_100a)"; }
+int64_t ll_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
+
+int ll_cache_create(int layers, int heads, int head_dim, int tokens_per_frame, int chunk_frames,
+                    int sink_frames, int window_frames, ll_cache **out)
+{
+    if (!out) return fail(LL_ERR_INVALID_ARG, "out is null");
+    *out = nullptr;
+    if (layers <= 0 || heads <= 0 || tokens_per_frame <= 0 || chunk_frames <= 0 || sink_frames < 0 ||
+        window_frames <= 0)
+        return fail(LL_ERR_INVALID_ARG, "non-positive size");
+    if (head_dim != 64 && head_dim != 128)
+        return fail(LL_ERR_UNSUPPORTED_SHAPE, "head_dim %d: only 64 and 128 are built", head_dim);
+    if (sink_frames % chunk_frames || window_frames % chunk_frames || window_frames < chunk_frames)
+        return fail(LL_ERR_UNSUPPORTED_SHAPE, "sink_frames and window_frames must be multiples of chunk_frames");
+    if (sink_frames + window_frames > LL_MAX_SLOTS)
+        return fail(LL_ERR_UNSUPPORTED_SHAPE, "sink_frames + window_frames > %d", LL_MAX_SLOTS);
+    if (window_frames / chunk_frames > ll::kMaxGroups)
+        return fail(LL_ERR_UNSUPPORTED_SHAPE, "window_frames / chunk_frames > %d", ll::kMaxGroups);
+    int64_t rows = (int64_t)(sink_frames + window_frames) * tokens_per_frame;
+    if (rows > (1ll << 30) || (int64_t)window_frames * tokens_per_frame > (1ll << 30))
+        return fail(LL_ERR_UNSUPPORTED_SHAPE, "cache rows per head exceed 2^30");
+
+    ll_cache *c = new ll_cache();
+    c->L = layers; c->H = heads; c->D = head_dim; c->P = tokens_per_frame;
+    c->C = chunk_frames; c->S = sink_frames; c->W = window_frames;
+    c->n_slots = sink_frames + window_frames;
+    c->rows = rows;
+    c->layers.resize(layers);
+    for (auto &l : c->layers)
+        for (int s = 0; s < LL_MAX_SLOTS; ++s) l.slot_frame[s] = -1;
+    int n_t, n_h;
+    rope_split(head_dim, &n_t, &n_h);
+    c->off_status = 0;
+    c->off_ttab = align_up(ll::kStatusWords * sizeof(uint32_t), 256);
+    c->off_hwtab = align_up(c->off_ttab + (size_t)ll::kTTabFrames * n_t * sizeof(float2), 256);
+    // grid_h + grid_w <= tokens_per_frame + 1 for any grid with grid_h*grid_w == tokens_per_frame
+    c->aux_bytes = align_up(c->off_hwtab + (size_t)(tokens_per_frame + 1) * n_h * sizeof(float2), 1024);
+    c->kv_bytes = (size_t)heads * rows * head_dim * sizeof(ll_bf16);
+    *out = c;
+    return LL_OK;
+}
+
+void ll_cache_destroy(ll_cache *cache) { delete cache; }
+
+size_t ll_cache_storage_bytes(const ll_cache *c)
+{
+    if (!c) return 0;
+    return c->aux_bytes + (size_t)c->L * 2 * c->kv_bytes;
+}
+
+int ll_cache_bind_storage(ll_cache *c, void *dev, size_t bytes, ll_stream stream)
+{
+    if (!c || !dev) return fail(LL_ERR_INVALID_ARG, "null handle or storage");
+    if (reinterpret_cast<uintptr_t>(dev) & 1023u) return fail(LL_ERR_INVALID_ARG, "storage must be 1024-byte aligned");
+    if (bytes < ll_cache_storage_bytes(c))
+        return fail(LL_ERR_INVALID_ARG, "storage too small: %zu < %zu bytes", bytes, ll_cache_storage_bytes(c));
+    if (c->dry_run) return fail(LL_ERR_INVALID_ARG, "handle is in bookkeeping-only mode");
+    cudaError_t e = cudaMemsetAsync(dev, 0, ll_cache_storage_bytes(c), (cudaStream_t)stream);
+    if (e != cudaSuccess) return cuda_fail(e, "cudaMemsetAsync(storage)");
+    std::vector<CUtensorMap> km(c->L), vm(c->L);
+    char *base = static_cast<char *>(dev) + c->aux_bytes;
+    for (int l = 0; l < c->L; ++l) {
+        char *k = base + (size_t)l * 2 * c->kv_bytes;
+        int s = encode_map(&km[l], k, c->D, (uint64_t)c->rows, c->H, (uint64_t)c->D * 2,
+                           (uint64_t)c->rows * c->D * 2, 128, 1);
+        if (s != LL_OK) return s;
+        s = encode_map(&vm[l], k + c->kv_bytes, c->D, (uint64_t)c->rows, c->H, (uint64_t)c->D * 2,
+                       (uint64_t)c->rows * c->D * 2, 128, 1);
+        if (s != LL_OK) return s;
+    }
+    c->kmap.swap(km); c->vmap.swap(vm);
+    c->storage = static_cast<char *>(dev);
+    c->storage_bytes = bytes;
+    c->hw_valid = false; c->t_base = -1;
+    return LL_OK;
+}
+
+int ll_cache_kv_offset(const ll_cache *c, int layer, int which, int head, size_t *offset)
+{
+    if (!layer_ok(c, layer) || !offset || which < 0 || which > 1 || head < 0 || head >= c->H)
+        return fail(LL_ERR_INVALID_ARG, "bad argument to ll_cache_kv_offset");
+    *offset = c->aux_bytes + (size_t)layer * 2 * c->kv_bytes + (size_t)which * c->kv_bytes +
+              (size_t)head * c->rows * c->D * sizeof(ll_bf16);
+    return LL_OK;
+}
+
+int ll_rope_append_kv(ll_cache *c, int layer, const ll_bf16 *q, const ll_bf16 *k, const ll_bf16 *v,
+                      int64_t frame_start, int n_frames, int grid_h, int grid_w, float rope_theta,
+                      ll_bf16 *q_out, ll_stream stream)
+{
+    if (!layer_ok(c, layer)) return fail(LL_ERR_INVALID_ARG, "bad cache handle or layer %d", layer);
+    if (grid_h <= 0 || grid_w <= 0 || (int64_t)grid_h * grid_w != c->P)
+        return fail(LL_ERR_INVALID_ARG, "grid %dx%d does not give %d tokens per frame", grid_h, grid_w, c->P);
+    if (!(rope_theta > 0.f)) return fail(LL_ERR_INVALID_ARG, "rope_theta must be positive");
+    if (n_frames != c->C) return fail(LL_ERR_BAD_POSITION, "n_frames %d != chunk_frames %d", n_frames, c->C);
+    ll::LayerState &st = c->layers[layer];
+    const bool is_new = frame_start == st.end;
+    const bool is_over = st.end >= c->C && frame_start == st.end - c->C;
+    if (!is_new && !is_over)
+        return fail(LL_ERR_BAD_POSITION, "frame_start %lld is neither end (%lld) nor end - chunk_frames",
+                    (long long)frame_start, (long long)st.end);
+    if (frame_start + n_frames > INT32_MAX) return fail(LL_ERR_BAD_POSITION, "frame index exceeds int32");
+    if (!c->dry_run) {
+        if (!k || !v) return fail(LL_ERR_INVALID_ARG, "null k or v");
+        if (q_out && !q) return fail(LL_ERR_INVALID_ARG, "q_out given without q");
+        if (!aligned16(k) || !aligned16(v) || !aligned16(q) || !aligned16(q_out))
+            return fail(LL_ERR_INVALID_ARG, "q/k/v/q_out must be 16-byte aligned");
+        int s = need_storage(c);
+        if (s != LL_OK) return s;
+        s = ensure_tables(c, frame_start, frame_start + n_frames, grid_h, grid_w, rope_theta, (cudaStream_t)stream);
+        if (s != LL_OK) return s;
+        ll::RopeAppendParams p;
+        fill_rope_params(c, layer, q_out ? q : nullptr, k, v, q_out, frame_start, n_frames, grid_w, &p);
+        cudaError_t e = ll::launch_rope_append(p, c->D, (cudaStream_t)stream);
+        if (e != cudaSuccess) return cuda_fail(e, "rope+append kernel");
+    }
+    if (is_new) {
+        for (int i = 0; i < n_frames; ++i) {
+            int64_t f = frame_start + i;
+            int s = slot_of(c, f);
+            if (st.slot_frame[s] >= 0 && st.slot_frame[s] != (int32_t)f) st.n_evictions += 1;
+            st.slot_frame[s] = (int32_t)f;
+        }
+        st.end += n_frames;
+        st.n_appends += 1;
+    } else {
+        st.n_overwrites += 1;
+    }
+    return LL_OK;
+}
+
+int ll_sink_window_attn(ll_cache *c, int layer, const ll_bf16 *q_roped, int64_t q_frame_start,
+                        int n_q_frames, ll_bf16 *out, float *lse_out, ll_stream stream)
+{
+    return attn_entry(c, layer, q_roped, q_frame_start, n_q_frames, out, lse_out, stream, false);
+}
+
+int ll_debug_attn_simt(ll_cache *c, int layer, const ll_bf16 *q_roped, int64_t q_frame_start,
+                       int n_q_frames, ll_bf16 *out, float *lse_out, ll_stream stream)
+{
+    return attn_entry(c, layer, q_roped, q_frame_start, n_q_frames, out, lse_out, stream, true);
+}
+
+int ll_recache(ll_cache *c, int layer, const ll_bf16 *q, const ll_bf16 *k, const ll_bf16 *v, int n_frames,
+               int grid_h, int grid_w, float rope_theta, ll_bf16 *q_out, ll_bf16 *out, float *lse_out,
+               ll_stream stream)
+{
+    if (!layer_ok(c, layer)) return fail(LL_ERR_INVALID_ARG, "bad cache handle or layer %d", layer);
+    if (grid_h <= 0 || grid_w <= 0 || (int64_t)grid_h * grid_w != c->P)
+        return fail(LL_ERR_INVALID_ARG, "grid %dx%d does not give %d tokens per frame", grid_h, grid_w, c->P);
+    if (!(rope_theta > 0.f)) return fail(LL_ERR_INVALID_ARG, "rope_theta must be positive");
+    ll::LayerState &st = c->layers[layer];
+    const int64_t r0 = std::max<int64_t>(c->S, st.end - c->W);
+    const int64_t resident = std::max<int64_t>(0, st.end - r0);
+    if (n_frames != resident)
+        return fail(LL_ERR_BAD_POSITION, "n_frames %d != resident window frames %lld", n_frames, (long long)resident);
+    if (n_frames == 0) return LL_OK;
+    const int n_groups = n_frames / c->C;
+    int64_t gstart[ll::kMaxGroups];
+    for (int g = 0; g < n_groups; ++g) gstart[g] = r0 + (int64_t)g * c->C;
+    if (!c->dry_run) {
+        if (!q || !k || !v || !q_out || !out) return fail(LL_ERR_INVALID_ARG, "null q/k/v/q_out/out");
+        if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(q_out) || !aligned16(out) ||
+            (lse_out && !aligned16(lse_out)))
+            return fail(LL_ERR_INVALID_ARG, "pointers must be 16-byte aligned");
+        int s = need_storage(c);
+        if (s != LL_OK) return s;
+    }
+    ll::AttnParams ap;
+    int s = build_attn_params(c, layer, q_out, out, lse_out, n_groups, gstart, r0, &ap);
+    if (s != LL_OK) return s;
+    if (!c->dry_run) {
+        s = ensure_tables(c, r0, st.end, grid_h, grid_w, rope_theta, (cudaStream_t)stream);
+        if (s != LL_OK) return s;
+        ll::RopeAppendParams rp;
+        fill_rope_params(c, layer, q, k, v, q_out, r0, n_frames, grid_w, &rp);
+        cudaError_t e = ll::launch_rope_append(rp, c->D, (cudaStream_t)stream);
+        if (e != cudaSuccess) return cuda_fail(e, "rope+append kernel (recache)");
+        s = launch_attention(c, layer, ap, (cudaStream_t)stream, false);
+        if (s != LL_OK) return s;
+    }
+    st.n_recaches += 1;
+    return LL_OK;
+}
+
+int ll_cache_reset(ll_cache *c)
+{
+    if (!c) return fail(LL_ERR_INVALID_ARG, "null handle");
+    for (auto &l : c->layers) {
+        l.end = 0;
+        for (int s = 0; s < LL_MAX_SLOTS; ++s) l.slot_frame[s] = -1;
+    }
+    return LL_OK;
+}
+
+int ll_cache_get_state(const ll_cache *c, int layer, ll_state *out)
+{
+    if (!layer_ok(c, layer) || !out) return fail(LL_ERR_INVALID_ARG, "bad argument to ll_cache_get_state");
+    const ll::LayerState &st = c->layers[layer];
+    memset(out, 0, sizeof *out);
+    out->end = st.end;
+    out->n_slots = c->n_slots;
+    int ring = 0;
+    for (int s = 0; s < LL_MAX_SLOTS; ++s) {
+        out->slot_frame[s] = s < c->n_slots ? st.slot_frame[s] : -1;
+        if (s >= c->S && s < c->n_slots && st.slot_frame[s] >= 0) ++ring;
+    }
+    out->ring_valid = ring;
+    out->n_appends = st.n_appends; out->n_overwrites = st.n_overwrites;
+    out->n_evictions = st.n_evictions; out->n_recaches = st.n_recaches;
+    out->n_attn_calls = st.n_attn;
+    return LL_OK;
+}
+
+int ll_cache_set_state(ll_cache *c, int layer, const ll_state *in)
+{
+    if (!layer_ok(c, layer) || !in) return fail(LL_ERR_INVALID_ARG, "bad argument to ll_cache_set_state");
+    if (in->n_slots != c->n_slots || in->end < 0 || in->end % c->C)
+        return fail(LL_ERR_INVALID_ARG, "state does not belong to a cache of this shape");
+    for (int s = 0; s < c->n_slots; ++s) {
+        int32_t f = in->slot_frame[s];
+        if (f < 0) continue;
+        if (f >= in->end || slot_of(c, f) != s)
+            return fail(LL_ERR_INVALID_ARG, "slot %d holds frame %d, which the slot rule does not allow", s, f);
+    }
+    ll::LayerState &st = c->layers[layer];
+    st.end = in->end;
+    for (int s = 0; s < LL_MAX_SLOTS; ++s) st.slot_frame[s] = s < c->n_slots ? in->slot_frame[s] : -1;
+    st.n_appends = in->n_appends; st.n_overwrites = in->n_overwrites;
+    st.n_evictions = in->n_evictions; st.n_recaches = in->n_recaches; st.n_attn = in->n_attn_calls;
+    return LL_OK;
+}
+
+int ll_cache_visible_ranges(const ll_cache *c, int layer, int64_t q_frame_start, int64_t lo_floor,
+                            int64_t *starts, int64_t *lens, int *n_ranges)
+{
+    if (!layer_ok(c, layer) || !starts || !lens || !n_ranges)
+        return fail(LL_ERR_INVALID_ARG, "bad argument to ll_cache_visible_ranges");
+    return visible_ranges(c, layer, q_frame_start, lo_floor, starts, lens, n_ranges);
+}
+
+int ll_cache_set_dry_run(ll_cache *c, int on)
+{
+    if (!c) return fail(LL_ERR_INVALID_ARG, "null handle");
+    c->dry_run = on != 0;
+    return LL_OK;
+}
+
+int ll_cache_device_status(ll_cache *c, ll_stream stream)
+{
+    if (!c) return fail(LL_ERR_INVALID_ARG, "null handle");
+    int s = need_storage(c);
+    if (s != LL_OK) return s;
+    cudaError_t e = cudaStreamSynchronize((cudaStream_t)stream);
+    if (e != cudaSuccess) return cuda_fail(e, "cudaStreamSynchronize");
+    uint32_t w[ll::kStatusWords];
+    e = cudaMemcpy(w, c->storage + c->off_status, sizeof w, cudaMemcpyDeviceToHost);
+    if (e != cudaSuccess) return cuda_fail(e, "cudaMemcpy(status)");
+    if (w[0] == ll::kStatusOk) return LL_OK;
+    e = cudaMemset(c->storage + c->off_status, 0, sizeof w);
+    if (e != cudaSuccess) return cuda_fail(e, "cudaMemset(status)");
+    return fail(LL_ERR_DEVICE_TIMEOUT,
+                "a kernel gave up on a bounded wait: code %u role %u barrier %u iteration %u block (%u,%u,%u)",
+                w[0], w[1], w[2], w[3], w[4], w[5], w[6]);
+}
+
+}  // extern "C"

@@ -1,0 +1,106 @@
+// Internal declarations shared by the host code and the kernel translation units.
+#pragma once
+
+#include <cuda.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include <string>
+#include <vector>
+
+#include "llattn.h"
+
+namespace ll {
+
+constexpr int kMaxGroups = 24;        // query groups (chunks) one attention launch can hold
+constexpr int kTTabFrames = 256;      // frames covered by the resident t-axis RoPE table
+constexpr int kTTabAlign = 128;       // table base is a multiple of this many frames
+constexpr int kStatusWords = 64;      // uint32 words at the head of the aux block
+constexpr int kQTileRows = 256;       // query rows one CTA owns (two 128-row MMA tiles)
+constexpr int kKeyTile = 128;         // keys per MMA tile
+
+// status word 0 is non-zero when a kernel abandoned a wait; words 1.. hold details
+enum StatusCode : uint32_t {
+    kStatusOk = 0,
+    kStatusTimeout = 1,
+};
+
+struct LayerState {
+    int64_t end = 0;
+    int32_t slot_frame[LL_MAX_SLOTS];
+    int64_t n_appends = 0, n_overwrites = 0, n_evictions = 0, n_recaches = 0, n_attn = 0;
+};
+
+// One group of query rows that share a visible key set.
+struct AttnGroup {
+    int q_begin;                      // first query row of the group in the q tensor
+    int q_rows;                       // rows in the group
+    int tile_begin;                   // index of the group's first query tile in the grid
+    int n_ranges;
+    int k_start[LL_MAX_RANGES];       // visible cache-row runs
+    int k_len[LL_MAX_RANGES];
+};
+
+struct AttnParams {
+    int n_groups;
+    int heads;
+    int nq_total;                     // rows of q / out
+    int total_qtiles;                 // grid.x
+    int64_t rows_per_head;            // (S+W)*P
+    float scale_log2;                 // log2(e) / sqrt(D)
+    const ll_bf16 *q;                 // [nq_total, H, D]
+    ll_bf16 *out;                     // [nq_total, H, D]
+    float *lse;                       // [H, nq_total] or null
+    const ll_bf16 *kbase;             // layer K: [H][rows][D]
+    const ll_bf16 *vbase;             // layer V
+    uint32_t *status;                 // aux status words
+    AttnGroup g[kMaxGroups];
+};
+
+struct RopeAppendParams {
+    const ll_bf16 *q, *k, *v;         // [n_tokens, H, D]; q may be null
+    ll_bf16 *q_out;                   // nullable
+    ll_bf16 *kcache, *vcache;         // layer base, [H][rows][D]
+    const float2 *t_tab;              // entry of the call's first frame: [frame][n_t] (cos, sin)
+    const float2 *h_tab;              // [grid_h][n_h]
+    const float2 *w_tab;              // [grid_w][n_w]
+    int64_t rows_per_head;
+    int n_tokens, heads, P, grid_w;
+    int n_t, n_h;                     // pairs of the t and h bands (w band takes the rest)
+    int slot[LL_MAX_SLOTS];           // storage slot of the call's i-th frame
+};
+
+// kernel launchers (each returns the cudaError of the launch)
+cudaError_t launch_rope_tables(float2 *t_tab, int64_t t_base, int n_t_frames, int n_t,
+                               float2 *h_tab, int grid_h, float2 *w_tab, int grid_w, int n_hw,
+                               float theta, bool do_t, bool do_hw, cudaStream_t stream);
+cudaError_t launch_rope_append(const RopeAppendParams &p, int head_dim, cudaStream_t stream);
+cudaError_t launch_attn_sm100(const AttnParams &p, int head_dim, const CUtensorMap &qmap,
+                              const CUtensorMap &kmap, const CUtensorMap &vmap,
+                              cudaStream_t stream);
+cudaError_t launch_attn_simt(const AttnParams &p, int head_dim, cudaStream_t stream);
+
+void count_launch(int n = 1);
+
+}  // namespace ll
+
+struct ll_cache {
+    int L, H, D, P, C, S, W;
+    int n_slots;
+    int64_t rows;                     // (S+W)*P cache rows per head
+    std::vector<ll::LayerState> layers;
+    bool dry_run = false;
+
+    char *storage = nullptr;
+    size_t storage_bytes = 0;
+    // aux block layout (byte offsets from storage)
+    size_t off_status = 0, off_ttab = 0, off_hwtab = 0, aux_bytes = 0;
+    size_t kv_bytes = 0;              // one K (or V) matrix set of one layer: H*rows*D*2
+    std::vector<CUtensorMap> kmap, vmap;
+
+    // which RoPE tables are resident
+    bool hw_valid = false;
+    int tab_gh = 0, tab_gw = 0;
+    float tab_theta = 0.f;
+    int64_t t_base = -1;
+};

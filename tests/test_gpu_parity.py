@@ -1,0 +1,303 @@
+"""GPU parity: the CUDA path, called through the C ABI, against the CPU oracle
+on the same seeded inputs.  Integer state and V rows bit-exact; roped K/Q within
+one bf16 ulp of the fp64 rotation; attention within 1e-2 max-abs / 1e-3 mean-abs
+of the fp64 oracle."""
+import dataclasses
+
+import numpy as np
+import pytest
+import torch
+
+from paper_2509_22622_b200 import binding as B
+from paper_2509_22622_b200 import synth
+
+from gpu_util import bits, check_attn, dev, f64, new_cache, ulp_distance
+
+pytestmark = pytest.mark.gpu
+
+MEDIUM = synth.Workload("medium_d128", 1, 2, 128, 10, 20, 3, 3, 9, n_chunks=7, seed=11)
+MEDIUM64 = synth.Workload("medium_d64", 1, 3, 64, 9, 14, 2, 2, 4, n_chunks=6, seed=12)
+ODD = synth.Workload("odd_rows", 1, 1, 128, 7, 19, 1, 1, 3, n_chunks=6, seed=13)     # 133 tokens per frame
+
+
+def oracle_for(oracle_mod, wl, faithful=False):
+    return oracle_mod.Oracle(1, wl.heads, wl.head_dim, wl.tokens_per_frame, wl.chunk_frames,
+                             wl.sink_frames, wl.window_frames, faithful=faithful)
+
+
+def cache_rows_of_slot(t, slot, P):
+    """[H, rows, D] device view -> [P, H, D] numpy bits of one slot."""
+    return bits(t[:, slot * P:(slot + 1) * P, :]).transpose(1, 0, 2)
+
+
+def check_rope_bits(got_bits, want_f64):
+    """Within one bf16 ulp of the correctly rounded fp64 rotation, >= 99% exact."""
+    want_bits = synth.f32_to_bf16_bits(want_f64.astype(np.float32))
+    d = ulp_distance(got_bits, want_bits)
+    assert d.max() <= 1, "max ulp distance %d" % d.max()
+    assert (d == 0).mean() >= 0.99, "only %.4f exact" % (d == 0).mean()
+
+
+# ---------------------------------------------------------------------------
+# rope + append
+# ---------------------------------------------------------------------------
+
+@pytest.mark.parametrize("wl", [synth.CONFIGS[0], MEDIUM, MEDIUM64, ODD], ids=lambda w: w.name)
+def test_rope_append_matches_oracle(oracle_mod, wl):
+    cache = new_cache(wl)
+    orc = oracle_for(oracle_mod, wl, faithful=True)
+    P, C = wl.tokens_per_frame, wl.chunk_frames
+    for chunk in range(wl.n_chunks):
+        q, k, v = synth.chunk_qkv(wl, chunk)
+        dq, dk, dv = dev(q), dev(k), dev(v)
+        q_out = torch.empty_like(dq)
+        for rep in range(2):          # second call overwrites the newest chunk in place
+            fs = chunk * C
+            cache.rope_append_kv(0, dq, dk, dv, fs, wl.grid_h, wl.grid_w, wl.rope_theta, q_out)
+            orc.append(0, synth.bf16_bits_to_f64(k), synth.bf16_bits_to_f64(v), fs, wl.grid_h, wl.grid_w,
+                       wl.rope_theta)
+        cache.check_device()
+        st, ost = cache.state(), orc.state()
+        assert st["end"] == ost["end"] and st["slot_frame"] == list(ost["slot_frame"])
+        assert st["evictions"] == ost["evictions"] and st["overwrites"] == chunk + 1
+        K, V = orc.read_layer()
+        kc, vc = cache.kv_view(0, 0), cache.kv_view(0, 1)
+        for slot, frame in enumerate(st["slot_frame"]):
+            if frame < 0:
+                continue
+            check_rope_bits(cache_rows_of_slot(kc, slot, P), K[slot])
+            want_v = synth.f32_to_bf16_bits(V[slot].astype(np.float32))
+            assert np.array_equal(cache_rows_of_slot(vc, slot, P), want_v)
+        want_q = oracle_mod.rope(synth.bf16_bits_to_f64(q), chunk * C, wl.grid_h, wl.grid_w, wl.rope_theta)
+        check_rope_bits(bits(q_out), want_q)
+    cache.close()
+
+
+def test_rope_append_in_place_and_without_q(oracle_mod):
+    wl = MEDIUM
+    cache = new_cache(wl)
+    q, k, v = synth.chunk_qkv(wl, 0)
+    dq, dk, dv = dev(q), dev(k), dev(v)
+    cache.rope_append_kv(0, None, dk, dv, 0, wl.grid_h, wl.grid_w)          # K/V only
+    k_first = bits(cache.kv_view(0, 0)).copy()
+    cache.rope_append_kv(0, dq, dk, dv, 0, wl.grid_h, wl.grid_w, q_out=dq)  # q rotated in place
+    cache.check_device()
+    assert np.array_equal(bits(cache.kv_view(0, 0)), k_first)
+    check_rope_bits(bits(dq), oracle_mod.rope(synth.bf16_bits_to_f64(q), 0, wl.grid_h, wl.grid_w))
+    cache.close()
+
+
+def test_rope_append_late_in_a_long_stream(oracle_mod):
+    """Frame 957 (the 240 s horizon): table accuracy at large t, ring wrapped many times."""
+    wl = dataclasses.replace(MEDIUM, heads=1)
+    cache = new_cache(wl)
+    orc = oracle_for(oracle_mod, wl, faithful=True)
+    # jump both sides to end = 957 through their state setters / replay
+    st = B.ll_cache_get_state(cache.h, 0)
+    st.end = 957
+    S, W = wl.sink_frames, wl.window_frames
+    for f in list(range(S)) + list(range(957 - W, 957)):
+        st.slot_frame[f if f < S else S + (f - S) % W] = f
+    B.ll_cache_set_state(cache.h, 0, st)
+    q, k, v = synth.chunk_qkv(wl, 319)
+    dq, dk, dv = dev(q), dev(k), dev(v)
+    q_out = torch.empty_like(dq)
+    cache.rope_append_kv(0, dq, dk, dv, 957, wl.grid_h, wl.grid_w, wl.rope_theta, q_out)
+    cache.check_device()
+    assert cache.state()["end"] == 960
+    want_k = oracle_mod.rope(synth.bf16_bits_to_f64(k), 957, wl.grid_h, wl.grid_w, wl.rope_theta)
+    want_q = oracle_mod.rope(synth.bf16_bits_to_f64(q), 957, wl.grid_h, wl.grid_w, wl.rope_theta)
+    P = wl.tokens_per_frame
+    kc = cache.kv_view(0, 0)
+    for i, f in enumerate(range(957, 960)):
+        slot = orc.slot_of(f)
+        check_rope_bits(cache_rows_of_slot(kc, slot, P), want_k[i * P:(i + 1) * P])
+    check_rope_bits(bits(q_out), want_q)
+    cache.close()
+
+
+# ---------------------------------------------------------------------------
+# attention (decode) streamed chunk by chunk
+# ---------------------------------------------------------------------------
+
+def stream_and_check(oracle_mod, wl, attn, n_chunks=None, rows_per_chunk=None, relative=False, passes=1):
+    cache = new_cache(wl)
+    orc = oracle_for(oracle_mod, wl)
+    C, P = wl.chunk_frames, wl.tokens_per_frame
+    nq = C * P
+    worst = (0.0, 0.0)
+    for chunk in range(n_chunks or wl.n_chunks):
+        for pass_id in range(passes):
+            q, k, v = synth.chunk_qkv(wl, chunk, pass_id=pass_id)
+            dq, dk, dv = dev(q), dev(k), dev(v)
+            q_out = torch.empty_like(dq)
+            out = torch.full_like(dq, float("nan"))
+            lse = torch.full((wl.heads, nq), float("nan"), device="cuda", dtype=torch.float32)
+            cache.rope_append_kv(0, dq, dk, dv, chunk * C, wl.grid_h, wl.grid_w, wl.rope_theta, q_out)
+            attn(cache.h, 0, q_out, chunk * C, C, out, lse)
+            cache.check_device()
+            orc.append(0, synth.bf16_bits_to_f64(k), synth.bf16_bits_to_f64(v), chunk * C, wl.grid_h, wl.grid_w,
+                       wl.rope_theta)
+        qr = orc.rope_q(synth.bf16_bits_to_f64(q), chunk * C, wl.grid_h, wl.grid_w, wl.rope_theta)
+        rows = None if rows_per_chunk is None else synth.sample_rows(nq, rows_per_chunk, seed=chunk)
+        want, want_lse = orc.attn(0, qr, chunk * C, rows=rows)
+        got = f64(out) if rows is None else f64(out)[rows]
+        got_lse = lse.cpu().numpy().T.astype(np.float64)
+        got_lse = got_lse if rows is None else got_lse[rows]
+        e = check_attn(got, want, relative=relative)
+        worst = (max(worst[0], e[0]), max(worst[1], e[1]))
+        assert np.abs(got_lse - want_lse).max() <= 2e-2, np.abs(got_lse - want_lse).max()
+        st, ost = cache.state(), orc.state()
+        assert st["end"] == ost["end"] and st["slot_frame"] == list(ost["slot_frame"])
+    cache.close()
+    return worst
+
+
+@pytest.mark.parametrize("wl", [synth.CONFIGS[0], MEDIUM64, ODD], ids=lambda w: w.name)
+def test_simt_triage_kernel_matches_oracle(oracle_mod, wl):
+    stream_and_check(oracle_mod, wl, B.ll_debug_attn_simt)
+
+
+@pytest.mark.parametrize("wl", [synth.CONFIGS[0], MEDIUM, MEDIUM64, ODD], ids=lambda w: w.name)
+def test_sink_window_attn_matches_oracle(oracle_mod, wl):
+    stream_and_check(oracle_mod, wl, B.ll_sink_window_attn)
+
+
+def test_sink_window_attn_with_denoising_passes(oracle_mod):
+    """Every pass overwrites the newest chunk's K/V before attending (Algorithm 2)."""
+    stream_and_check(oracle_mod, MEDIUM, B.ll_sink_window_attn, n_chunks=5, passes=3)
+
+
+def test_sink_window_attn_outliers(oracle_mod):
+    wl = dataclasses.replace(MEDIUM, outlier_frac=0.01, seed=14)
+    stream_and_check(oracle_mod, wl, B.ll_sink_window_attn, relative=True)
+
+
+def test_sink_window_attn_is_deterministic():
+    wl = MEDIUM
+    cache = new_cache(wl)
+    C = wl.chunk_frames
+    outs = []
+    for chunk in range(5):
+        q, k, v = synth.chunk_qkv(wl, chunk)
+        dq, dk, dv = dev(q), dev(k), dev(v)
+        q_out = torch.empty_like(dq)
+        cache.rope_append_kv(0, dq, dk, dv, chunk * C, wl.grid_h, wl.grid_w, q_out=q_out)
+    for rep in range(3):
+        out = torch.empty_like(q_out)
+        B.ll_sink_window_attn(cache.h, 0, q_out, 4 * C, C, out)
+        outs.append(bits(out))
+    cache.check_device()
+    assert np.array_equal(outs[0], outs[1]) and np.array_equal(outs[0], outs[2])
+    cache.close()
+
+
+def test_closed_form_visible_histogram():
+    """K = 0 and V = one-hot(frame id): the output is the histogram of visible
+    frames, a check that needs no oracle and holds at any size."""
+    wl = synth.Workload("hist", 1, 2, 128, 8, 25, 3, 3, 9, n_chunks=8, seed=0)
+    cache = new_cache(wl)
+    C, P, D = wl.chunk_frames, wl.tokens_per_frame, wl.head_dim
+    for chunk in range(wl.n_chunks):
+        q, _, _ = synth.chunk_qkv(wl, chunk)
+        k = torch.zeros(C * P, wl.heads, D, device="cuda", dtype=torch.bfloat16)
+        v = torch.zeros_like(k)
+        for i in range(C):
+            v[i * P:(i + 1) * P, :, (chunk * C + i) % D] = 1.0
+        dq = dev(q)
+        out = torch.empty_like(dq)
+        cache.rope_append_kv(0, dq, k, v, chunk * C, wl.grid_h, wl.grid_w, q_out=dq)
+        B.ll_sink_window_attn(cache.h, 0, dq, chunk * C, C, out)
+        cache.check_device()
+        end = (chunk + 1) * C
+        frames = [f for f in range(end) if f < wl.sink_frames or f >= end - wl.window_frames]
+        want = np.zeros(D)
+        want[[f % D for f in frames]] = 1.0 / len(frames)
+        got = f64(out)
+        assert np.abs(got - want).max() <= 2.0 ** -9 * want.max() + 1e-6
+    cache.close()
+
+
+# ---------------------------------------------------------------------------
+# recache
+# ---------------------------------------------------------------------------
+
+@pytest.mark.parametrize("wl,at_chunks", [(synth.CONFIGS[0], (0, 1, 2, 5, 7)), (MEDIUM, (1, 3, 4, 6)),
+                                          (MEDIUM64, (2, 5)), (ODD, (4,))], ids=lambda x: getattr(x, "name", None))
+def test_recache_matches_oracle(oracle_mod, wl, at_chunks):
+    cache = new_cache(wl)
+    orc = oracle_for(oracle_mod, wl)
+    C, P, S, W = wl.chunk_frames, wl.tokens_per_frame, wl.sink_frames, wl.window_frames
+    for chunk in range(wl.n_chunks):
+        q, k, v = synth.chunk_qkv(wl, chunk)
+        dq, dk, dv = dev(q), dev(k), dev(v)
+        q_out = torch.empty_like(dq)
+        cache.rope_append_kv(0, dq, dk, dv, chunk * C, wl.grid_h, wl.grid_w, wl.rope_theta, q_out)
+        orc.append(0, synth.bf16_bits_to_f64(k), synth.bf16_bits_to_f64(v), chunk * C, wl.grid_h, wl.grid_w,
+                   wl.rope_theta)
+        if chunk not in at_chunks:
+            continue
+        end = (chunk + 1) * C
+        n = max(0, end - max(S, end - W))
+        rq, rk, rv = synth.chunk_qkv(wl, chunk, pass_id=synth.RECACHE_PASS, n_frames=n)
+        before = cache.state()
+        if n == 0:
+            B.ll_recache(cache.h, 0, None, None, None, 0, wl.grid_h, wl.grid_w, wl.rope_theta, None, None)
+            assert cache.state() == before
+            continue
+        drq, drk, drv = dev(rq), dev(rk), dev(rv)
+        rq_out = torch.empty_like(drq)
+        out = torch.full_like(drq, float("nan"))
+        lse = torch.full((wl.heads, n * P), float("nan"), device="cuda", dtype=torch.float32)
+        cache.recache(0, drq, drk, drv, n, wl.grid_h, wl.grid_w, wl.rope_theta, rq_out, out, lse)
+        cache.check_device()
+        _, want, want_lse = orc.recache(0, synth.bf16_bits_to_f64(rq), synth.bf16_bits_to_f64(rk),
+                                        synth.bf16_bits_to_f64(rv), n, wl.grid_h, wl.grid_w, wl.rope_theta)
+        check_attn(f64(out), want)
+        assert np.abs(lse.cpu().numpy().T - want_lse).max() <= 2e-2
+        after = cache.state()
+        assert after["end"] == before["end"] and after["slot_frame"] == before["slot_frame"]
+        assert after["recaches"] == before["recaches"] + 1
+        # the sink rows were not touched, the ring rows hold the new K/V
+        K, V = orc.read_layer()
+        vc = cache.kv_view(0, 1)
+        for slot, frame in enumerate(after["slot_frame"]):
+            if frame >= 0:
+                assert np.array_equal(cache_rows_of_slot(vc, slot, P),
+                                      synth.f32_to_bf16_bits(V[slot].astype(np.float32)))
+    # the stream goes on over the rebuilt window
+    chunk = wl.n_chunks
+    q, k, v = synth.chunk_qkv(wl, chunk)
+    dq, dk, dv = dev(q), dev(k), dev(v)
+    q_out, out = torch.empty_like(dq), torch.empty_like(dq)
+    cache.rope_append_kv(0, dq, dk, dv, chunk * C, wl.grid_h, wl.grid_w, wl.rope_theta, q_out)
+    B.ll_sink_window_attn(cache.h, 0, q_out, chunk * C, C, out)
+    cache.check_device()
+    orc.append(0, synth.bf16_bits_to_f64(k), synth.bf16_bits_to_f64(v), chunk * C, wl.grid_h, wl.grid_w, wl.rope_theta)
+    want, _ = orc.attn(0, orc.rope_q(synth.bf16_bits_to_f64(q), chunk * C, wl.grid_h, wl.grid_w, wl.rope_theta), chunk * C)
+    check_attn(f64(out), want)
+    cache.close()
+
+
+# ---------------------------------------------------------------------------
+# error paths on a live device
+# ---------------------------------------------------------------------------
+
+def test_errors_leave_state_unchanged():
+    wl = MEDIUM
+    cache = new_cache(wl)
+    q, k, v = synth.chunk_qkv(wl, 0)
+    dq, dk, dv = dev(q), dev(k), dev(v)
+    with pytest.raises(B.LLError) as e:
+        cache.rope_append_kv(0, dq, dk, dv, 3, wl.grid_h, wl.grid_w)
+    assert e.value.code == B.LL_ERR_BAD_POSITION
+    with pytest.raises(B.LLError) as e:
+        B.ll_rope_append_kv(cache.h, 0, dq, dk[1:].reshape(-1)[1:], dv, 0, 3, wl.grid_h, wl.grid_w)   # misaligned
+    assert e.value.code == B.LL_ERR_INVALID_ARG
+    assert cache.state()["end"] == 0
+    cache.rope_append_kv(0, dq, dk, dv, 0, wl.grid_h, wl.grid_w)
+    with pytest.raises(B.LLError) as e:
+        B.ll_recache(cache.h, 0, dq, dk, dv, 3, wl.grid_h, wl.grid_w, 10000.0, dq, dq)   # only sink frames exist
+    assert e.value.code == B.LL_ERR_BAD_POSITION
+    cache.check_device()
+    cache.close()

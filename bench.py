@@ -1,0 +1,397 @@
+#!/usr/bin/env python
+"""Benchmark of the sink+window attention hot path (one JSON line on stdout).
+
+A *step* is one pass of the whole hot path over one chunk of synthetic input at
+the Wan-1.3B-shaped single-layer workload: fused 3-D RoPE + K/V append of a new
+3-frame chunk (4680 tokens x 12 heads x 128), then sink+window attention of its
+queries over the full cache (18720 keys).  The caches of several layers are
+rotated from step to step so that every step finds its K/V cold in L2.
+
+    python bench.py --gpus N --steps K --warmup W [--impl reference]
+
+value      : attention TFLOP/s over the whole step time (append included), inputs
+             resident in HBM.
+e2e        : the same with pinned host Q/K/V copied in and the output copied out
+             inside the timed region.
+roofline   : the attention kernel alone against the measured dense bf16 peak.
+cpu_baseline / --impl reference: the fp64 CPU oracle on a bounded sample of the
+             same workload's query rows.
+With N > 1 every rank runs an independent replica (the path has no exchange
+step); value is the sum over ranks divided by the slowest rank's time.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+from paper_2509_22622_b200 import synth  # noqa: E402
+
+WL = synth.CONFIGS[1]
+N_LAYERS = 4               # caches rotated across steps (4 x 115 MB > L2)
+N_INPUT_SETS = 4
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+CLOCK_QUERY = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+               "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+               "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+
+def steady_keys(wl):
+    return (wl.sink_frames + wl.window_frames) * wl.tokens_per_frame
+
+
+def attn_flops(wl, n_rows=None):
+    nq = wl.chunk_tokens if n_rows is None else n_rows
+    return 4.0 * nq * steady_keys(wl) * wl.head_dim * wl.heads
+
+
+def append_bytes(wl):
+    # Q in + Q out + K in + K cache + V in + V cache
+    return 6.0 * wl.chunk_tokens * wl.heads * wl.head_dim * 2
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as fh:
+            d = json.load(fh)
+        return {k: float(d[k]) for k in FALLBACK_PEAKS if k in d}, "measured"
+    return dict(FALLBACK_PEAKS), "fallback"
+
+
+def load_traffic():
+    """Per-launch DRAM bytes of the kernels from the committed ncu summary, if any."""
+    path = os.path.join(ROOT, "profiles", "dram_traffic.txt")
+    out = {}
+    if os.path.exists(path):
+        with open(path) as fh:
+            for line in fh:
+                parts = line.split("#")[0].split()
+                if len(parts) == 2:
+                    out[parts[0]] = float(parts[1])
+    return out
+
+
+class ClockSampler:
+    """nvidia-smi clock/throttle samples taken while the timed region runs."""
+
+    def __init__(self, index: int):
+        self.path = "/tmp/llattn_clocks_%d_%d.csv" % (os.getpid(), index)
+        self.proc = None
+        try:
+            self.fh = open(self.path, "w")
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(index), "--query-gpu=" + CLOCK_QUERY,
+                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                         stdout=self.fh, stderr=subprocess.DEVNULL)
+        except Exception:
+            self.proc = None
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        self.fh.close()
+        sm, smax, power, reasons = [], [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        with open(self.path) as fh:
+            for line in fh:
+                f = [t.strip() for t in line.split(",")]
+                if len(f) < 9:
+                    continue
+                try:
+                    sm.append(float(f[1])); smax.append(float(f[2])); power.append(float(f[3]))
+                except ValueError:
+                    continue
+                for name, val in zip(names, f[5:9]):
+                    if val.lower().startswith("active"):
+                        reasons.add(name)
+        try:
+            os.remove(self.path)
+        except OSError:
+            pass
+        if not sm:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["no samples"]}
+        busy = [c for c, p in zip(sm, power) if p > 0.5 * max(power)] or sm
+        return {"sm_mhz": statistics.median(busy), "sm_max_mhz": max(smax), "reasons": sorted(reasons),
+                "samples": len(sm), "power_w_max": max(power)}
+
+
+# ---------------------------------------------------------------------------
+# the oracle leg (CPU baseline / reference arm)
+# ---------------------------------------------------------------------------
+
+def oracle_sample(target_seconds: float, steps: int = 1, warmup: int = 0):
+    """Time the fp64 oracle on a bounded sample of query rows of one steady-state
+    attention call of the workload.  Returns (tflops, cores, description, ms_per_step)."""
+    import oracle
+    oracle.build()
+    wl = WL
+    C, P = wl.chunk_frames, wl.tokens_per_frame
+    cores = len(os.sched_getaffinity(0))
+    orc = oracle.Oracle(1, wl.heads, wl.head_dim, P, C, wl.sink_frames, wl.window_frames)
+    n_fill = (wl.sink_frames + wl.window_frames) // C
+    t_append = 0.0
+    for chunk in range(n_fill):
+        _, k, v = synth.chunk_qkv(wl, chunk)
+        t0 = time.perf_counter()
+        orc.append(0, synth.bf16_bits_to_f64(k), synth.bf16_bits_to_f64(v), chunk * C, wl.grid_h, wl.grid_w)
+        t_append = time.perf_counter() - t0
+    q, _, _ = synth.chunk_qkv(wl, n_fill - 1)
+    qr = orc.rope_q(synth.bf16_bits_to_f64(q), (n_fill - 1) * C, wl.grid_h, wl.grid_w)
+    # calibrate: rows the oracle gets through in about target_seconds
+    probe = synth.sample_rows(C * P, 2 * cores, seed=1)
+    t0 = time.perf_counter()
+    orc.attn(0, qr, (n_fill - 1) * C, rows=probe)
+    per_row = (time.perf_counter() - t0) / len(probe)
+    n_rows = int(max(cores, min(C * P, target_seconds / per_row)))
+    n_rows = max(cores, n_rows // cores * cores)
+    rows = synth.sample_rows(C * P, n_rows, seed=2)
+    times = []
+    for i in range(warmup + steps):
+        t0 = time.perf_counter()
+        orc.attn(0, qr, (n_fill - 1) * C, rows=rows)
+        dt = time.perf_counter() - t0
+        if i >= warmup:
+            times.append(dt)
+    dt = sum(times) / len(times)
+    tflops = attn_flops(wl, len(rows)) / dt / 1e12
+    what = ("%d of %d query rows x all %d heads x %d keys of one steady-state attention call, fp64, "
+            "%d OpenMP threads; one oracle append of a chunk took %.2f s"
+            % (len(rows), C * P, wl.heads, steady_keys(wl), cores, t_append))
+    orc.close()
+    return tflops, cores, what, dt * 1e3
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    per_step = max(2.0, min(20.0, 120.0 / max(1, args.steps + args.warmup)))
+    tflops, cores, what, ms = oracle_sample(per_step, steps=args.steps, warmup=args.warmup)
+    line = {
+        "impl": "reference", "metric": "sink_window_attn_tflops", "value": tflops, "unit": "TFLOP/s",
+        "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": WL.name, "sample": what},
+        "cpu_baseline": {"value": tflops, "unit": "TFLOP/s", "cores": cores, "kind": "oracle", "sample": what},
+        "e2e": {"value": tflops, "unit": "TFLOP/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line))
+
+
+# ---------------------------------------------------------------------------
+# the CUDA leg
+# ---------------------------------------------------------------------------
+
+def run_ours(args):
+    import torch
+    from paper_2509_22622_b200 import binding as B
+    from paper_2509_22622_b200 import build as _build
+
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench.py needs a CUDA device: the library has no CPU fallback")
+    torch.cuda.set_device(local_rank)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+    if rank == 0:
+        _build.build()
+    if dist is not None:
+        dist.barrier()
+    B.lib()
+
+    wl = WL
+    C, P, H, D = wl.chunk_frames, wl.tokens_per_frame, wl.heads, wl.head_dim
+    nq = C * P
+    n_fill = (wl.sink_frames + wl.window_frames) // C
+    warmup = max(args.warmup, 3)
+    stream = torch.cuda.current_stream()
+
+    def dev(bits):
+        return torch.from_numpy(np.ascontiguousarray(bits).view(np.int16)).cuda().view(torch.bfloat16)
+
+    cache = B.Cache(N_LAYERS, H, D, P, C, wl.sink_frames, wl.window_frames, device="cuda:%d" % local_rank)
+    host_sets = [synth.chunk_qkv(wl, 100 + i, stream=rank) for i in range(N_INPUT_SETS)]
+    dev_sets = [tuple(dev(t) for t in s) for s in host_sets]
+    pinned = [tuple(torch.from_numpy(t.view(np.int16)).view(torch.bfloat16).pin_memory() for t in s)
+              for s in host_sets]
+    q_roped = torch.empty(nq, H, D, device="cuda", dtype=torch.bfloat16)
+    out = torch.empty_like(q_roped)
+    out_host = torch.empty(nq, H, D, dtype=torch.bfloat16).pin_memory()
+    stage = tuple(torch.empty_like(q_roped) for _ in range(3))
+
+    # untimed prefill: every layer reaches the steady state (ring full)
+    for layer in range(N_LAYERS):
+        for chunk in range(n_fill):
+            q, k, v = dev_sets[(layer + chunk) % N_INPUT_SETS]
+            cache.rope_append_kv(layer, q, k, v, chunk * C, wl.grid_h, wl.grid_w, wl.rope_theta, q_roped)
+    cache.check_device()
+    step_no = [0]
+
+    def step(e2e=False, ev=None):
+        s = step_no[0]
+        step_no[0] += 1
+        layer = s % N_LAYERS
+        fs = cache.state(layer)["end"]
+        if e2e:
+            for dst, src in zip(stage, pinned[s % N_INPUT_SETS]):
+                dst.copy_(src, non_blocking=True)
+            q, k, v = stage
+        else:
+            q, k, v = dev_sets[s % N_INPUT_SETS]
+        if ev:
+            ev[0].record(stream)
+        cache.rope_append_kv(layer, q, k, v, fs, wl.grid_h, wl.grid_w, wl.rope_theta, q_roped)
+        if ev:
+            ev[1].record(stream)
+        cache.sink_window_attn(layer, q_roped, fs, out)
+        if ev:
+            ev[2].record(stream)
+        if e2e:
+            out_host.copy_(out, non_blocking=True)
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(warmup):
+        step()
+    cache.check_device()
+
+    sampler = ClockSampler(local_rank) if rank == 0 else None
+    time.sleep(0.3)
+    launches0 = B.ll_launch_count()
+    events = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(args.steps)]
+    t_begin, t_end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    t_begin.record(stream)
+    for i in range(args.steps):
+        step(ev=events[i])
+    t_end.record(stream)
+    barrier()
+    launches = B.ll_launch_count() - launches0
+    total_ms = t_begin.elapsed_time(t_end)
+    append_ms = sum(e[0].elapsed_time(e[1]) for e in events) / args.steps
+    attn_ms = sum(e[1].elapsed_time(e[2]) for e in events) / args.steps
+    cache.check_device()
+
+    # end to end: pinned host inputs in, output back, every step
+    for _ in range(2):
+        step(e2e=True)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    e0.record(stream)
+    for _ in range(args.steps):
+        step(e2e=True)
+    e1.record(stream)
+    barrier()
+    e2e_ms = e0.elapsed_time(e1)
+    clocks = sampler.stop() if sampler else None
+    cache.check_device()
+
+    # recache of the full window (one launch pair), reported beside the headline
+    n_w = wl.window_frames
+    rq, rk, rv = (dev(t) for t in synth.chunk_qkv(wl, 200, pass_id=synth.RECACHE_PASS, n_frames=n_w, stream=rank))
+    rq_out, r_out = torch.empty_like(rq), torch.empty_like(rq)
+    rc = [torch.cuda.Event(enable_timing=True) for _ in range(2)]
+    cache.recache(0, rq, rk, rv, n_w, wl.grid_h, wl.grid_w, wl.rope_theta, rq_out, r_out)
+    torch.cuda.synchronize()
+    rc[0].record(stream)
+    for _ in range(3):
+        cache.recache(0, rq, rk, rv, n_w, wl.grid_h, wl.grid_w, wl.rope_theta, rq_out, r_out)
+    rc[1].record(stream)
+    torch.cuda.synchronize()
+    recache_ms = rc[0].elapsed_time(rc[1]) / 3
+    cache.check_device()
+
+    if dist is not None:
+        t = torch.tensor([total_ms, e2e_ms, attn_ms, append_ms], device="cuda", dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        total_ms, e2e_ms, attn_ms, append_ms = t.tolist()
+    if rank != 0:
+        if dist is not None:
+            dist.destroy_process_group()
+        return
+
+    flops_step = attn_flops(wl)
+    peaks, peak_kind = load_peaks()
+    traffic = load_traffic()
+    value = world * args.steps * flops_step / (total_ms * 1e-3) / 1e12
+    e2e_value = world * args.steps * flops_step / (e2e_ms * 1e-3) / 1e12
+    attn_tflops = flops_step / (attn_ms * 1e-3) / 1e12
+    append_gbs = append_bytes(wl) / (append_ms * 1e-3) / 1e9
+    ms_per_step = total_ms / args.steps
+    in_bytes = 3 * nq * H * D * 2
+    cpu = None
+    if world == 1 and not args.no_cpu_baseline:
+        tf, cores, what, _ = oracle_sample(15.0)
+        cpu = {"value": tf, "unit": "TFLOP/s", "cores": cores, "kind": "oracle", "sample": what}
+    line = {
+        "metric": "sink_window_attn_tflops", "value": value, "unit": "TFLOP/s", "n_gpus": world,
+        "steps": args.steps, "warmup": warmup, "ms_per_step": ms_per_step, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": wl.name, "heads": H, "head_dim": D, "tokens_per_frame": P, "chunk_frames": C,
+                   "sink_frames": wl.sink_frames, "window_frames": wl.window_frames, "query_rows": nq,
+                   "keys": steady_keys(wl), "parallelism": "replicas x%d" % world,
+                   "l2": "inputs larger than L2: %d layer caches (115 MB each) and %d q/k/v sets rotate"
+                         % (N_LAYERS, N_INPUT_SETS)},
+        "e2e": {"value": e2e_value, "unit": "TFLOP/s", "h2d_bytes_per_step": in_bytes,
+                "d2h_bytes_per_step": nq * H * D * 2, "ms_per_step": e2e_ms / args.steps},
+        "gpu_launches": int(launches),
+        "clocks": clocks,
+        "roofline": {"bound": "tensor", "kernel": "attn_sm100_kernel<128>", "achieved": attn_tflops,
+                     "peak": peaks["bf16_tflops"], "unit": "TFLOP/s", "frac": attn_tflops / peaks["bf16_tflops"],
+                     "peak_kind": "of %s (burst bf16 GEMM)" % peak_kind, "ms_per_launch": attn_ms,
+                     "frac_of_nominal_2250": attn_tflops / 2250.0,
+                     "traffic": traffic.get("attn_sm100_kernel")},
+        "roofline_append": {"bound": "hbm", "kernel": "rope_append_kernel<128>", "achieved": append_gbs,
+                            "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": append_gbs / peaks["hbm_gbs"],
+                            "peak_kind": "of %s (copy)" % peak_kind, "ms_per_launch": append_ms,
+                            "traffic": traffic.get("rope_append_kernel")},
+        "cpu_baseline": cpu,
+        "extra": {"latent_frames_per_s_30_layers_5_passes": C / (150 * ms_per_step * 1e-3),
+                  "latent_frames_per_s_30_layers_4_passes": C / (120 * ms_per_step * 1e-3),
+                  "recache_ms_per_layer": recache_ms,
+                  "recache_tflops": 9 * attn_flops(wl) / 4 / (recache_ms * 1e-3) / 1e12,
+                  "paper_context": "20.7 video FPS (about 5.2 latent frames/s) for the whole 1.3B model on one H100"},
+    }
+    print(json.dumps(line))
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=4)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

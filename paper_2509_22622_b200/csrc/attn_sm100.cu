@@ -154,7 +154,8 @@ attn_sm100_kernel(const __grid_constant__ AttnParams p, const __grid_constant__ 
             if (i == kPFull || i == kPFull + 1) count = 128;
             mbar_init(bar(i), count);
         }
-        *abort_flag = 0;
+        // an earlier CTA already gave up on a wait: this one does not start (flag value 2)
+        *abort_flag = (*reinterpret_cast<volatile uint32_t *>(p.status) != kStatusOk) ? 2 : 0;
         fence_mbar_init();
     }
     if (warp == kTmaWarp) {
@@ -167,8 +168,11 @@ attn_sm100_kernel(const __grid_constant__ AttnParams p, const __grid_constant__ 
     const uint32_t tmem = *tmem_slot;
 
     WaitCtx ctx{abort_flag, p.status, warp};
+    const bool skip = *abort_flag != 0;
 
-    if (warp == kTmaWarp) {
+    if (skip) {
+        // nothing to do
+    } else if (warp == kTmaWarp) {
         // =========================== TMA producer ===========================
         if (lane == 0) {
             prefetch_tensormap(&qmap);
@@ -362,7 +366,7 @@ attn_sm100_kernel(const __grid_constant__ AttnParams p, const __grid_constant__ 
     // ---- common exit -------------------------------------------------------------
     tc_fence_before_sync();
     __syncthreads();
-    if (*abort_flag) {
+    if (*abort_flag == 1) {
         // give copies and MMAs that may still be in flight time to land before the
         // shared and tensor memory go back to the SM
         const uint64_t t0 = globaltimer_ns();

@@ -194,6 +194,25 @@ def run_reference(args):
 
 
 # ---------------------------------------------------------------------------
+# multi-rank aggregation (replicas only: no data-path collective)
+# ---------------------------------------------------------------------------
+
+def reduce_max(values, dist, device="cpu"):
+    """Element-wise max over ranks of a short list of per-rank timings (ms)."""
+    if dist is None:
+        return list(values)
+    import torch
+    t = torch.tensor(list(values), device=device, dtype=torch.float64)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return t.tolist()
+
+
+def whole_job_tflops(world: int, steps: int, flops_per_step: float, slowest_ms: float) -> float:
+    """Every rank ran `steps` independent steps; the job took as long as its slowest rank."""
+    return world * steps * flops_per_step / (slowest_ms * 1e-3) / 1e12
+
+
+# ---------------------------------------------------------------------------
 # the CUDA leg
 # ---------------------------------------------------------------------------
 
@@ -323,10 +342,7 @@ def run_ours(args):
     recache_ms = rc[0].elapsed_time(rc[1]) / 3
     cache.check_device()
 
-    if dist is not None:
-        t = torch.tensor([total_ms, e2e_ms, attn_ms, append_ms], device="cuda", dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        total_ms, e2e_ms, attn_ms, append_ms = t.tolist()
+    total_ms, e2e_ms, attn_ms, append_ms = reduce_max([total_ms, e2e_ms, attn_ms, append_ms], dist, "cuda")
     if rank != 0:
         if dist is not None:
             dist.destroy_process_group()
@@ -335,8 +351,8 @@ def run_ours(args):
     flops_step = attn_flops(wl)
     peaks, peak_kind = load_peaks()
     traffic = load_traffic()
-    value = world * args.steps * flops_step / (total_ms * 1e-3) / 1e12
-    e2e_value = world * args.steps * flops_step / (e2e_ms * 1e-3) / 1e12
+    value = whole_job_tflops(world, args.steps, flops_step, total_ms)
+    e2e_value = whole_job_tflops(world, args.steps, flops_step, e2e_ms)
     attn_tflops = flops_step / (attn_ms * 1e-3) / 1e12
     append_gbs = append_bytes(wl) / (append_ms * 1e-3) / 1e9
     ms_per_step = total_ms / args.steps

@@ -56,6 +56,7 @@ def lib():
             L.llo_create.argtypes = [C.c_int] * 8
             L.llo_destroy.argtypes = [C.c_void_p]
             L.llo_reset.argtypes = [C.c_void_p]
+            L.llo_seek.argtypes = [C.c_void_p, C.c_int, C.c_int64]
             L.llo_get_state.argtypes = [C.c_void_p, C.c_int, C.POINTER(C.c_int64),
                                         C.POINTER(C.c_int32), C.POINTER(C.c_int64)]
             L.llo_slot_of.argtypes = [C.c_void_p, C.c_int64]
@@ -162,6 +163,12 @@ class Oracle:
         st = lib().llo_reset(self._h)
         if st != OK:
             raise OracleError(st, "reset")
+
+    def seek(self, layer: int, end: int):
+        """Continue the stream at frame ``end`` with an empty window (sink kept)."""
+        st = lib().llo_seek(self._h, layer, end)
+        if st != OK:
+            raise OracleError(st, "seek")
 
     # -- the path ---------------------------------------------------------
     def append(self, layer, k, v, frame_start, gh, gw, theta=10000.0, n_frames=None):

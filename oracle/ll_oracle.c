@@ -109,6 +109,21 @@ int llo_reset(llo *o)
     return LLO_OK;
 }
 
+/* Skip ahead: continue the stream at frame `end` (a multiple of C, not before
+ * the current end) as if the frames in between had been generated and had
+ * rolled out of the window again.  The sink stays; the ring is left empty.
+ * Lets a test reach a late point of a long stream by replaying only the chunks
+ * that are still resident there. */
+int llo_seek(llo *o, int layer, int64_t end)
+{
+    if (!o || layer < 0 || layer >= o->L) return LLO_ERR_ARG;
+    if (end % o->C || end < o->end[layer] || end < o->S) return LLO_ERR_POSITION;
+    int32_t *sf = o->slot_frame + (size_t)layer * slots(o);
+    for (int s = o->S; s < o->S + o->W; ++s) sf[s] = -1;
+    o->end[layer] = end;
+    return LLO_OK;
+}
+
 int llo_get_state(const llo *o, int layer, int64_t *end, int32_t *slot_frame,
                   int64_t *evictions)
 {

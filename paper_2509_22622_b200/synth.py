@@ -143,3 +143,25 @@ def sample_rows(n_rows: int, n_samples: int, tile: int = 128, seed: int = 0) -> 
     if rest > 0:
         must.update(int(r) for r in rng.integers(0, n_rows, size=rest))
     return np.asarray(sorted(must), dtype=np.int64)
+
+
+class InputPool:
+    """A few pre-drawn (q, k, v) chunk sets that long schedules index into.
+
+    The full-stack and long-stream workloads make tens of thousands of calls;
+    drawing fresh tensors for each would take hours on the host.  Call
+    (chunk, layer, pass, stream) uses set ``index(...)`` of the pool, so any call's
+    inputs can be regenerated on their own (the oracle replays only sampled calls).
+    """
+
+    def __init__(self, wl: Workload, n_sets: int = 6, n_frames: int | None = None,
+                 pass_id: int = 0):
+        self.wl = wl
+        self.n_sets = n_sets
+        self.sets = [chunk_qkv(wl, 1000 + i, pass_id=pass_id, n_frames=n_frames) for i in range(n_sets)]
+
+    def index(self, chunk: int, layer: int = 0, pass_id: int = 0, stream: int = 0) -> int:
+        return (chunk * 7 + layer * 3 + pass_id * 5 + stream * 11) % self.n_sets
+
+    def get(self, chunk: int, layer: int = 0, pass_id: int = 0, stream: int = 0):
+        return self.sets[self.index(chunk, layer, pass_id, stream)]

@@ -446,3 +446,27 @@ def test_ring_fills_from_its_first_slot(oracle_mod):
     o.append(0, x, x, 12, 1, 1)      # frames 12..14 replace frames 3..5 in place
     assert list(o.state()["slot_frame"]) == [0, 1, 2, 12, 13, 14, 6, 7, 8, 9, 10, 11]
     assert o.state()["evictions"] == 3
+
+
+def test_seek_equals_full_replay(oracle_mod):
+    """Skipping evicted history gives the same attention as replaying all of it."""
+    C, S, W, gh, gw, H, D = 2, 2, 4, 2, 2, 2, 16
+    P = gh * gw
+    full = oracle_mod.Oracle(1, H, D, P, C, S, W)
+    data = [tuple(rand((C * P, H, D), 1000 + 3 * c + i) for i in range(3)) for c in range(9)]
+    for c, (q, k, v) in enumerate(data):
+        full.append(0, k, v, c * C, gh, gw)
+    want = full.attn(0, full.rope_q(data[8][0], 16, gh, gw), 16)
+    short = oracle_mod.Oracle(1, H, D, P, C, S, W)
+    short.append(0, data[0][1], data[0][2], 0, gh, gw)          # the sink chunk
+    short.seek(0, 14)                                           # window = chunks 7, 8
+    with pytest.raises(oracle_mod.OracleError):
+        short.attn(0, short.rope_q(data[8][0], 16, gh, gw), 12)  # nothing resident yet
+    for c in (7, 8):
+        short.append(0, data[c][1], data[c][2], c * C, gh, gw)
+    got = short.attn(0, short.rope_q(data[8][0], 16, gh, gw), 16)
+    np.testing.assert_array_equal(got[0], want[0])
+    np.testing.assert_array_equal(got[1], want[1])
+    assert list(short.state()["slot_frame"]) == list(full.state()["slot_frame"])
+    with pytest.raises(oracle_mod.OracleError):
+        short.seek(0, 4)                                        # cannot go back

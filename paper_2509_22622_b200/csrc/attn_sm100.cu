@@ -37,6 +37,9 @@ constexpr int kTmaWarp = 8;
 constexpr int kMmaWarp = 9;
 constexpr uint64_t kWaitLimitNs = 2000000000ull;    // 2 s
 constexpr float kRescaleThreshold = 8.f;            // log2 units
+// 384 threads start with 168 registers each; (2 * 224 + 56) * 128 is the same total
+constexpr int kSoftmaxRegs = 224;
+constexpr int kProducerRegs = 56;
 
 template <int D>
 struct Cfg {
@@ -82,7 +85,7 @@ struct WaitCtx {
 };
 
 // Bounded wait on an mbarrier phase.  Returns false when the CTA is aborting.
-__device__ __noinline__ bool wait_slow(uint32_t bar, uint32_t parity, const WaitCtx &ctx, int bar_id, int iter)
+__device__ __forceinline__ bool wait_slow(uint32_t bar, uint32_t parity, const WaitCtx &ctx, int bar_id, int iter)
 {
     const uint64_t t0 = globaltimer_ns();
     uint32_t spins = 0;
@@ -170,8 +173,12 @@ attn_sm100_kernel(const __grid_constant__ AttnParams p, const __grid_constant__ 
     WaitCtx ctx{abort_flag, p.status, warp};
     const bool skip = *abort_flag != 0;
 
+    // Register reallocation: the softmax warpgroups hold a whole S row per thread, the
+    // producer warpgroup (TMA, MMA and two idle warps) needs little.
+    if (warp >= 8) {
+        setmaxnreg_dec<kProducerRegs>();
     if (skip) {
-        // nothing to do
+        // an earlier CTA gave up: nothing to do
     } else if (warp == kTmaWarp) {
         // =========================== TMA producer ===========================
         if (lane == 0) {
@@ -264,10 +271,12 @@ attn_sm100_kernel(const __grid_constant__ AttnParams p, const __grid_constant__ 
                 }
             }
         }
-    } else if (warp < 8) {
+    }
+    } else {
         // ========================= softmax warpgroups =========================
+        setmaxnreg_inc<kSoftmaxRegs>();
         const int w = warp >> 2;                       // query tile of this warpgroup
-        if (w < n_sub) {
+        if (!skip && w < n_sub) {
             const int r = threadIdx.x & 127;           // row inside the tile = TMEM lane
             const uint32_t lane_base = (uint32_t)((warp & 3) * 32) << 16;
             const uint32_t t_s = tmem + lane_base + C::kColS + 128 * w;
@@ -280,20 +289,31 @@ attn_sm100_kernel(const __grid_constant__ AttnParams p, const __grid_constant__ 
                 ok = __all_sync(0xffffffffu, wait_bar(bar(kSFull + w), (uint32_t)j & 1u, ctx, kSFull + w, j));
                 if (!ok) break;
                 tc_fence_after_sync();
-                uint32_t v[128];
-#pragma unroll
-                for (int i = 0; i < 4; ++i) tmem_ld32(t_s + 32 * i, v + 32 * i);
-                tmem_wait_ld();
                 const int nvalid = it.valid();
-                if (nvalid < kKeyTile) {
+                // ---- pass 1: row max of the tile (the values are fetched again below) ----
+                float m_tile;
+                uint32_t ca[32], cb[32];
+                {
+                    uint32_t v[128];
 #pragma unroll
-                    for (int i = 0; i < 128; ++i)
-                        if (i >= nvalid) v[i] = 0xff800000u;   // -inf
+                    for (int i = 0; i < 4; ++i) tmem_ld32(t_s + 32 * i, v + 32 * i);
+                    tmem_wait_ld();
+                    tmem_ld32(t_s, ca);                    // chunk 0 of pass 2, in flight during the max
+                    if (nvalid < kKeyTile) {
+#pragma unroll
+                        for (int i = 0; i < 128; ++i)
+                            if (i >= nvalid) v[i] = 0xff800000u;   // -inf
+                    }
+                    float mc[4];
+#pragma unroll
+                    for (int ch = 0; ch < 4; ++ch) {
+                        mc[ch] = fmaxf(__uint_as_float(v[32 * ch]), __uint_as_float(v[32 * ch + 1]));
+#pragma unroll
+                        for (int i = 2; i < 32; i += 2)
+                            mc[ch] = max3(mc[ch], __uint_as_float(v[32 * ch + i]), __uint_as_float(v[32 * ch + i + 1]));
+                    }
+                    m_tile = max3(mc[0], mc[1], fmaxf(mc[2], mc[3])) * c;
                 }
-                float mx = __uint_as_float(v[0]);
-#pragma unroll
-                for (int i = 1; i < 128; ++i) mx = fmaxf(mx, __uint_as_float(v[i]));
-                const float m_tile = mx * c;
                 if (j == 0) {
                     m = m_tile;
                 } else {
@@ -315,19 +335,37 @@ attn_sm100_kernel(const __grid_constant__ AttnParams p, const __grid_constant__ 
                         }
                     }
                 }
-                const float neg_m = -m;
-                float sum0 = 0.f, sum1 = 0.f;
+                // ---- pass 2: p = 2^(s*c - m) in 32-key chunks; P chunk k (16 packed columns)
+                //      lands on S columns that chunks <= k no longer need ----
+                const uint64_t c2 = pack2(c, c);
+                const uint64_t nm2 = pack2(-m, -m);
+                uint64_t acc[2] = {0ull, 0ull};
 #pragma unroll
-                for (int i = 0; i < 64; ++i) {
-                    const float p0 = ex2(fmaf(__uint_as_float(v[2 * i]), c, neg_m));
-                    const float p1 = ex2(fmaf(__uint_as_float(v[2 * i + 1]), c, neg_m));
-                    sum0 += p0;
-                    sum1 += p1;
-                    v[i] = pack_bf16(p0, p1);          // key 2i in the low half
+                for (int k = 0; k < 4; ++k) {
+                    uint32_t *cur = (k & 1) ? cb : ca;
+                    uint32_t *nxt = (k & 1) ? ca : cb;
+                    tmem_wait_ld();
+                    if (k < 3) tmem_ld32(t_s + 32 * (k + 1), nxt);
+                    if (nvalid < kKeyTile) {
+#pragma unroll
+                        for (int i = 0; i < 32; ++i)
+                            if (32 * k + i >= nvalid) cur[i] = 0xff800000u;
+                    }
+                    uint32_t pk[16];
+#pragma unroll
+                    for (int i = 0; i < 16; ++i) {
+                        const uint64_t t2 = fma2(pack2(__uint_as_float(cur[2 * i]), __uint_as_float(cur[2 * i + 1])), c2, nm2);
+                        float t0, t1;
+                        unpack2(t2, t0, t1);
+                        const float p0 = ex2(t0), p1 = ex2(t1);
+                        acc[i & 1] = add2(acc[i & 1], pack2(p0, p1));
+                        pk[i] = pack_bf16(p0, p1);         // key 2i in the low half
+                    }
+                    tmem_st16(t_s + 16 * k, pk);
                 }
+                float sum0, sum1;
+                unpack2(add2(acc[0], acc[1]), sum0, sum1);
                 l += sum0 + sum1;
-                tmem_st32(t_s, v);
-                tmem_st32(t_s + 32, v + 32);
                 tmem_wait_st();
                 tc_fence_before_sync();
                 mbar_arrive(bar(kPFull + w));

@@ -32,13 +32,18 @@ def ulp_distance(a_bits: np.ndarray, b_bits: np.ndarray) -> np.ndarray:
     return np.abs(key(a_bits) - key(b_bits))
 
 
-def check_attn(got_f64, want_f64, relative=False):
-    """The parity bar.  relative=True is the outlier workload's bar: the error is
-    measured against max(1, |reference|) because bf16 output rounding alone
-    exceeds 1e-2 absolute once |o| grows past ~5."""
+def check_attn(got_f64, want_f64, scale=None):
+    """The parity bar: max-abs <= 1e-2 and mean-abs <= 1e-3 against the oracle.
+
+    ``scale`` is used by the outlier workload only.  It is sum_j p_j |v_j| (the
+    oracle's attention over |V|), the magnitude of what each output element
+    sums: rounding P to bf16 for the PV product and rounding the output to bf16
+    each cost at most 2^-9 of it, so the error is measured in units of
+    max(1, scale).  For unit-variance inputs scale < 1 and this is the absolute
+    bar itself."""
     err = np.abs(got_f64 - want_f64)
-    if relative:
-        err = err / np.maximum(1.0, np.abs(want_f64))
+    if scale is not None:
+        err = err / np.maximum(1.0, scale)
     assert np.isfinite(got_f64).all()
     assert err.max() <= MAX_ABS, "max-abs error %.3e" % err.max()
     assert err.mean() <= MEAN_ABS, "mean-abs error %.3e" % err.mean()

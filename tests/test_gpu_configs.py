@@ -42,12 +42,13 @@ class DevicePool:
         return self.sets[self.pool.index(*key)]
 
 
-def check_rows(orc, cache_out, q_bits, frame_start, wl, n_rows, seed, relative=False):
+def check_rows(orc, cache_out, q_bits, frame_start, wl, n_rows, seed, orc_abs=None):
     nq = wl.chunk_tokens
     rows = synth.sample_rows(nq, n_rows, seed=seed)
     qr = orc.rope_q(F64(q_bits), frame_start, wl.grid_h, wl.grid_w, wl.rope_theta)
     want, _ = orc.attn(0, qr, frame_start, rows=rows)
-    return check_attn(f64(cache_out)[rows], want, relative=relative)
+    scale = orc_abs.attn(0, qr, frame_start, rows=rows)[0] if orc_abs else None
+    return check_attn(f64(cache_out)[rows], want, scale=scale)
 
 
 # ---------------------------------------------------------------------------
@@ -246,19 +247,22 @@ def test_config4_ragged_streams_window_sweep(oracle_mod, W):
         out = torch.full_like(q_out, float("nan"))
         cache.sink_window_attn(0, q_out, pos * C, out)
         cache.check_device()
+        # reference: storage-faithful oracle; a twin with |V| gives the error scale sum_j p_j |v_j|
         orc = make_oracle(oracle_mod, wl, faithful=True)
+        orc_abs = make_oracle(oracle_mod, wl, faithful=True)
         first = max(1, pos + 1 - W // C)
-        _, k, v = pool.get(0, 0, 0, stream)
-        orc.append(0, F64(k), F64(v), 0, wl.grid_h, wl.grid_w, wl.rope_theta)
-        if pos > 0:
-            orc.seek(0, first * C)
-        for chunk in range(first, pos + 1):
+        for chunk in [0] + list(range(first, pos + 1)):
+            if chunk == first and pos > 0:
+                orc.seek(0, first * C)
+                orc_abs.seek(0, first * C)
             _, k, v = pool.get(chunk, 0, 0, stream)
             orc.append(0, F64(k), F64(v), chunk * C, wl.grid_h, wl.grid_w, wl.rope_theta)
+            orc_abs.append(0, F64(k), np.abs(F64(v)), chunk * C, wl.grid_h, wl.grid_w, wl.rope_theta)
         assert cache.state()["slot_frame"] == list(orc.state()["slot_frame"]), (W, pos)
         q, _, _ = pool.get(pos, 0, 0, stream)
-        e = check_rows(orc, out, q, pos * C, wl, 32, pos, relative=True)
+        e = check_rows(orc, out, q, pos * C, wl, 32, pos, orc_abs=orc_abs)
         worst = (max(worst[0], e[0]), max(worst[1], e[1]))
         orc.close()
+        orc_abs.close()
         cache.close()
-    print("parity config4 W=%d: worst relative max %.3e mean %.3e" % (W, worst[0], worst[1]))
+    print("parity config4 W=%d: worst scaled max %.3e mean %.3e" % (W, worst[0], worst[1]))

@@ -124,6 +124,7 @@ def stream_and_check(oracle_mod, wl, attn, n_chunks=None, rows_per_chunk=None, r
                      faithful=False):
     cache = new_cache(wl)
     orc = oracle_for(oracle_mod, wl, faithful=faithful)
+    orc_abs = oracle_for(oracle_mod, wl, faithful=faithful) if relative else None   # same K, |V|
     C, P = wl.chunk_frames, wl.tokens_per_frame
     nq = C * P
     worst = (0.0, 0.0)
@@ -139,13 +140,17 @@ def stream_and_check(oracle_mod, wl, attn, n_chunks=None, rows_per_chunk=None, r
             cache.check_device()
             orc.append(0, synth.bf16_bits_to_f64(k), synth.bf16_bits_to_f64(v), chunk * C, wl.grid_h, wl.grid_w,
                        wl.rope_theta)
+            if orc_abs:
+                orc_abs.append(0, synth.bf16_bits_to_f64(k), np.abs(synth.bf16_bits_to_f64(v)), chunk * C,
+                               wl.grid_h, wl.grid_w, wl.rope_theta)
         qr = orc.rope_q(synth.bf16_bits_to_f64(q), chunk * C, wl.grid_h, wl.grid_w, wl.rope_theta)
         rows = None if rows_per_chunk is None else synth.sample_rows(nq, rows_per_chunk, seed=chunk)
         want, want_lse = orc.attn(0, qr, chunk * C, rows=rows)
         got = f64(out) if rows is None else f64(out)[rows]
         got_lse = lse.cpu().numpy().T.astype(np.float64)
         got_lse = got_lse if rows is None else got_lse[rows]
-        e = check_attn(got, want, relative=relative)
+        scale = orc_abs.attn(0, qr, chunk * C, rows=rows)[0] if orc_abs else None
+        e = check_attn(got, want, scale=scale)
         worst = (max(worst[0], e[0]), max(worst[1], e[1]))
         assert np.abs(got_lse - want_lse).max() <= 2e-2, np.abs(got_lse - want_lse).max()
         st, ost = cache.state(), orc.state()
@@ -175,7 +180,7 @@ def test_sink_window_attn_outliers(oracle_mod):
     single bf16 rounding of a rotated outlier (|x| ~ 60, half-ulp 0.12) moves a
     score by ~0.5, so the reference is the oracle in storage-faithful mode (rotated
     Q/K rounded to bf16, which is what the cache format holds) and the error is
-    measured relative to max(1, |reference|)."""
+    measured in units of max(1, sum_j p_j |v_j|)."""
     wl = dataclasses.replace(MEDIUM, name="medium_outliers", outlier_frac=0.01, seed=14)
     stream_and_check(oracle_mod, wl, B.ll_sink_window_attn, relative=True, faithful=True)
 

@@ -151,6 +151,42 @@ int ll_recache(ll_cache *cache, int layer, const ll_bf16 *q, const ll_bf16 *k,
  * empty, counters kept.  Stored bytes are not cleared. */
 int ll_cache_reset(ll_cache *cache);
 
+/* 3-D RoPE of a query tensor without any device allocation.  (The paper has no
+ * counterpart: this entry point exists for integration, not for the method.)
+ *
+ * Who it is for: code that must not, or cannot, obtain device memory at the
+ * time of the call - a serving process whose memory manager has already taken
+ * the whole GPU, a component that is forbidden to allocate after start-up so
+ * its latency stays predictable, a plug-in that is handed tensors but no
+ * allocator.  Such a caller cannot provide the storage block that
+ * ll_cache_bind_storage wants, and that block is where ll_rope_append_kv keeps
+ * its sine/cosine tables.  Here the tables live in a fixed array inside the
+ * library image instead (180 KB, present on every GPU that loads the library
+ * for as long as the process runs), and the call itself never calls cudaMalloc,
+ * cudaFree or anything else that allocates.
+ *
+ *   q, q_out  device, bf16 [n_frames*grid_h*grid_w, heads, head_dim], 16-byte
+ *             aligned; q_out may alias q.  Caller-owned, as everywhere else.
+ *   result    q_out = RoPE(q), the same values ll_rope_append_kv writes to its
+ *             q_out for the same frame_start, grid and rope_theta.
+ *   limits    head_dim 64 or 128; n_frames <= LL_STATIC_MAX_FRAMES;
+ *             grid_h + grid_w <= LL_STATIC_MAX_GRID_SUM.  Larger requests are
+ *             refused with LL_ERR_UNSUPPORTED_SHAPE (the fixed array cannot hold
+ *             their tables) and ll_last_error() says which limit was hit.
+ *   sharing   all calls on a GPU use the one array.  A call first writes the
+ *             table entries it needs and then reads them, on `stream`, so it does
+ *             not depend on what an earlier call left there; but two calls that
+ *             are in flight on the same GPU at the same time (two streams, two
+ *             threads) overwrite each other's tables.  Order them.
+ *   set-up    the first call on each device looks up where that device's copy
+ *             of the array lives (once, with that device current).  Make that
+ *             first call outside of any stream capture. */
+#define LL_STATIC_MAX_FRAMES 64
+#define LL_STATIC_MAX_GRID_SUM 1024
+int ll_rope_q_static(const ll_bf16 *q, ll_bf16 *q_out, int heads, int head_dim,
+                     int64_t frame_start, int n_frames, int grid_h, int grid_w,
+                     float rope_theta, ll_stream stream);
+
 /* ---- state, diagnostics ----------------------------------------------------- */
 
 int ll_cache_get_state(const ll_cache *cache, int layer, ll_state *out);

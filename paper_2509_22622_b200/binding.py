@@ -22,6 +22,8 @@ LL_ERR_CUDA = -5
 LL_ERR_DEVICE_TIMEOUT = -6
 LL_MAX_SLOTS = 64
 LL_MAX_RANGES = 4
+LL_STATIC_MAX_FRAMES = 64
+LL_STATIC_MAX_GRID_SUM = 1024
 
 
 class ll_state(C.Structure):
@@ -59,6 +61,8 @@ SIGNATURES = {
                                       C.c_void_p, C.c_void_p]),
     "ll_recache": (C.c_int, [C.c_void_p, C.c_int, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int, C.c_int,
                              C.c_int, C.c_float, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]),
+    "ll_rope_q_static": (C.c_int, [C.c_void_p, C.c_void_p, C.c_int, C.c_int, C.c_int64, C.c_int, C.c_int, C.c_int,
+                                   C.c_float, C.c_void_p]),
     "ll_cache_reset": (C.c_int, [C.c_void_p]),
     "ll_cache_get_state": (C.c_int, [C.c_void_p, C.c_int, C.POINTER(ll_state)]),
     "ll_cache_set_state": (C.c_int, [C.c_void_p, C.c_int, C.POINTER(ll_state)]),
@@ -156,6 +160,13 @@ def ll_debug_attn_simt(h, layer, q_roped, q_frame_start, n_q_frames, out, lse_ou
 def ll_recache(h, layer, q, k, v, n_frames, grid_h, grid_w, rope_theta, q_out, out, lse_out=None, stream=None):
     _check(lib().ll_recache(h, layer, _ptr(q), _ptr(k), _ptr(v), n_frames, grid_h, grid_w, rope_theta,
                             _ptr(q_out), _ptr(out), _ptr(lse_out), _stream(stream)))
+
+
+def ll_rope_q_static(q, q_out, heads, head_dim, frame_start, n_frames, grid_h, grid_w, rope_theta=10000.0,
+                     stream=None):
+    """RoPE(q) -> q_out through the entry point that allocates nothing (tables in a fixed array)."""
+    _check(lib().ll_rope_q_static(_ptr(q), _ptr(q_out), heads, head_dim, frame_start, n_frames, grid_h, grid_w,
+                                  rope_theta, _stream(stream)))
 
 
 def ll_cache_reset(h):

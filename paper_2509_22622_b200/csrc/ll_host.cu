@@ -250,6 +250,7 @@ int attn_entry(ll_cache *c, int layer, const ll_bf16 *q_roped, int64_t q_frame_s
 
 namespace ll {
 void count_launch(int n) { g_launches.fetch_add(n, std::memory_order_relaxed); }
+void set_last_error(const char *msg) { g_err = msg; }
 }  // namespace ll
 
 extern "C" {

@@ -81,6 +81,7 @@ cudaError_t launch_attn_sm100(const AttnParams &p, int head_dim, const CUtensorM
 cudaError_t launch_attn_simt(const AttnParams &p, int head_dim, cudaStream_t stream);
 
 void count_launch(int n = 1);
+void set_last_error(const char *msg);     // what ll_last_error() returns on this thread
 
 }  // namespace ll
 

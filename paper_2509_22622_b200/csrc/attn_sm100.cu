@@ -1,26 +1,39 @@
 // Sink+window attention on tcgen05 tensor cores (sm_100a).
 //
-// One CTA owns up to 256 query rows of one head (two 128-row MMA tiles) and
-// streams that head's visible cache rows past them in 128-key tiles:
+// Work decomposition.  A *column* is up to 256 query rows of one head (two
+// 128-row MMA tiles, "lanes" 0 and 1) and a *step* is one 128-key tile of that
+// column's visible cache rows.  All steps of all columns are laid end to end and
+// cut into equal shares, one per persistent CTA (one CTA per SM), so every SM
+// gets the same number of steps whatever the number of columns.  A column whose
+// steps fall into several CTAs is finished by whichever of them arrives last:
+// every part leaves its unnormalised O rows, reference maxima and sums in a
+// scratch slot, bumps the column's arrival counter, and the last one merges the
+// parts and writes the output.  Nothing waits on another CTA.
 //
-//   warp 8  (one lane)  TMA producer: Q tiles once, then K_0 V_0 K_1 V_1 ... into a
-//                       ring of 128-byte-swizzled shared-memory stages
-//   warp 9  (one lane)  MMA issuer: S_w = Q_w K_j^T (operands in shared memory,
+// Inside a CTA (640 threads):
+//   warp 16 (one lane)  TMA producer: the column's Q tiles, then K_j V_j K_j+1 ...
+//                       into a ring of 128-byte-swizzled shared-memory stages
+//   warp 17 (one lane)  MMA issuer: S_w = Q_w K_j^T (operands in shared memory,
 //                       accumulator in TMEM), O_w += P_w V_j (P read from TMEM)
-//   warps 0-3 / 4-7     softmax warpgroup of query tile 0 / 1: one thread per
-//                       query row reads its S row from TMEM, keeps the running
-//                       max and sum in fp32, writes P (bf16) back over S, and
-//                       rescales O in TMEM only when the max moved by > 2^8
+//   warps 0-15          softmax: warp (w, q, h) owns the 16 rows 32q + 16h .. of
+//                       lane w; its threads read S with the 16x256b TMEM shape, so
+//                       a row lives in the four threads of a quad and the row
+//                       maximum and sum are two shuffles away.  P (bf16) is
+//                       written back over S; O is rescaled in TMEM only when a
+//                       row's maximum moved by more than 2^8.
+//   While the softmax warps of one lane work, the tensor pipe runs the other
+//   lane's MMAs.  A share of the exponentials is evaluated with a cubic on the
+//   FMA pipe instead of the special-function unit, which both lanes would
+//   otherwise keep saturated.
 //
-// While one warpgroup runs its softmax the tensor pipe works on the other
-// tile's MMAs.  TMEM columns: S_0 | S_1 | O_0 | O_1 (fp32), P_w aliases the
-// first half of S_w.  The visible keys are a short list of contiguous cache-row
-// runs (sink, ring, wrapped ring); softmax does not care about key order, so
-// the only masking is the ragged last tile of each run.
+// TMEM columns: S_0 | S_1 | O_0 | O_1 (fp32); P_w aliases the first half of S_w.
+// The visible keys are a short list of contiguous cache-row runs (sink, ring,
+// wrapped ring); softmax does not care about key order, so the only masking is
+// the ragged last tile of each run.
 //
-// Every wait is bounded: a role that waits longer than kWaitLimitNs records a
-// status word, raises the CTA's abort flag, and all roles drain to the common
-// exit where TMEM is released.
+// Every mbarrier wait is bounded: a role that waits longer than kWaitLimitNs
+// records a status word, raises the CTA's abort flag, and all roles drain to the
+// common exit where TMEM is released.
 #include <cuda_bf16.h>
 
 #include "ll_internal.h"
@@ -32,14 +45,25 @@ namespace {
 
 using namespace ptx;
 
-constexpr int kThreads = 384;
-constexpr int kTmaWarp = 8;
-constexpr int kMmaWarp = 9;
+constexpr int kThreads = 640;
+constexpr int kSoftmaxWarps = 16;
+constexpr int kTmaWarp = 16;
+constexpr int kMmaWarp = 17;
 constexpr uint64_t kWaitLimitNs = 2000000000ull;    // 2 s
 constexpr float kRescaleThreshold = 8.f;            // log2 units
-// 384 threads start with 168 registers each; (2 * 224 + 56) * 128 is the same total
-constexpr int kSoftmaxRegs = 224;
-constexpr int kProducerRegs = 56;
+// Register reallocation draws on what the CTA was launched with: 640 threads x 96
+// registers = (16 softmax warps x 104 + 4 producer-group warps x 64) x 32.  A
+// request beyond that total would block forever.
+constexpr int kLaunchRegs = 96;
+constexpr int kSoftmaxRegs = 104;
+constexpr int kProducerRegs = 64;
+static_assert(kSoftmaxWarps * kSoftmaxRegs + (kThreads / 32 - kSoftmaxWarps) * kProducerRegs <= (kThreads / 32) * kLaunchRegs,
+              "setmaxnreg targets exceed the CTA's register allocation");
+// 8-key groups (bit k of 16 per 128-key tile) whose exponentials use the cubic
+#ifndef LL_POLY_MASK
+#define LL_POLY_MASK 0x8888u
+#endif
+constexpr uint32_t kPolyMask = LL_POLY_MASK;
 
 template <int D>
 struct Cfg {
@@ -52,16 +76,27 @@ struct Cfg {
     static constexpr int kTmemCols = 512;
     static constexpr int kColS = 0;                         // S_w at kColS + 128 w
     static constexpr int kColO = 256;                       // O_w at kColO + D w
+    static constexpr int kOChunks = D / 64;                 // 64-column pieces of an O row
 };
 
-// barrier indices inside the shared barrier array
-enum Bar { kQFull = 0, kSFull = 2, kPFull = 4, kOFull = 6, kKvFull = 8 /* + stage */, kKvEmpty = 24 /* + stage */, kNumBars = 40 };
+// barrier indices inside the shared barrier array (+ lane or + stage)
+enum Bar {
+    kQFull = 0, kQEmpty = 2, kSFull = 4, kPFull = 6, kOFull = 8, kOEmpty = 10,
+    kKvFull = 12, kKvEmpty = 20, kNumBars = 28
+};
 
 // Walks the visible key tiles of a group: runs in order, 128 rows at a time.
 struct KeyIter {
     const AttnGroup *g;
     int r, off;
-    __device__ KeyIter(const AttnGroup *grp) : g(grp), r(0), off(0) {}
+    __device__ KeyIter(const AttnGroup *grp, int first_tile) : g(grp), r(0), off(0)
+    {
+        while (first_tile > 0) {
+            const int nt = (g->k_len[r] + kKeyTile - 1) / kKeyTile;
+            if (first_tile >= nt) { first_tile -= nt; ++r; }
+            else { off = first_tile * kKeyTile; first_tile = 0; }
+        }
+    }
     __device__ int row() const { return g->k_start[r] + off; }
     __device__ int valid() const { return min(kKeyTile, g->k_len[r] - off); }
     __device__ void next()
@@ -71,12 +106,54 @@ struct KeyIter {
     }
 };
 
-__device__ int count_key_tiles(const AttnGroup &g)
+// One CTA's piece of one column.
+struct Segment {
+    int g, head, tile;      // the column
+    int kt0, kt1;           // its steps [kt0, kt1) run here
+    int q0;                 // first query row of the column
+    int rows_valid;         // live rows of the 256
+    int n_sub;              // live 128-row tiles
+    long long col_begin;    // global index of the column's first step
+};
+
+// First global step of CTA `cta`'s share (the next CTA's is one past its last).
+__device__ __forceinline__ long long share_begin(const AttnParams &p, int cta)
 {
-    int n = 0;
-    for (int r = 0; r < g.n_ranges; ++r) n += (g.k_len[r] + kKeyTile - 1) / kKeyTile;
-    return n;
+    return p.total_steps * cta / p.n_ctas;
 }
+
+// The CTA whose share holds global step u.
+__device__ __forceinline__ int cta_of_step(const AttnParams &p, long long u)
+{
+    return (int)(((u + 1) * p.n_ctas - 1) / p.total_steps);
+}
+
+struct WorkIter {
+    const AttnParams &p;
+    long long u, end;
+    __device__ WorkIter(const AttnParams &prm, int cta)
+        : p(prm), u(share_begin(prm, cta)), end(share_begin(prm, cta + 1)) {}
+    __device__ bool next(Segment &s)
+    {
+        if (u >= end) return false;
+        int g = 0;
+        while (g + 1 < p.n_groups && u >= p.g[g + 1].step_begin) ++g;
+        const AttnGroup &G = p.g[g];
+        const long long off = u - G.step_begin;
+        const int col = (int)(off / G.n_kt);
+        s.g = g;
+        s.head = col / G.tiles;
+        s.tile = col - s.head * G.tiles;
+        s.kt0 = (int)(off - (long long)col * G.n_kt);
+        s.kt1 = (int)min((long long)G.n_kt, s.kt0 + (end - u));
+        s.q0 = G.q_begin + s.tile * kQTileRows;
+        s.rows_valid = min(kQTileRows, G.q_rows - s.tile * kQTileRows);
+        s.n_sub = s.rows_valid > 128 ? 2 : 1;
+        s.col_begin = u - s.kt0;
+        u += s.kt1 - s.kt0;
+        return true;
+    }
+};
 
 struct WaitCtx {
     volatile int *abort_flag;
@@ -114,10 +191,51 @@ __device__ __forceinline__ bool wait_bar(uint32_t bar, uint32_t parity, const Wa
     return wait_slow(bar, parity, ctx, bar_id, iter);
 }
 
-__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi)
+__device__ __forceinline__ float as_f(uint32_t u) { return __uint_as_float(u); }
+__device__ __forceinline__ uint32_t as_u(float f) { return __float_as_uint(f); }
+
+// 2^x for two values on the special-function unit.
+__device__ __forceinline__ uint64_t exp2_sfu2(uint64_t x2)
 {
-    __nv_bfloat162 t = __floats2bfloat162_rn(lo, hi);
-    return *reinterpret_cast<uint32_t *>(&t);
+    float x0, x1;
+    unpack2(x2, x0, x1);
+    return pack2(ex2(x0), ex2(x1));
+}
+
+// 2^x for two values on the FMA pipe: x = n + f with n = floor(x) taken from the
+// low mantissa bits of x + 1.5 * 2^23 (rounded down), 2^f by a cubic with maximum
+// relative error 7.5e-5 on [0, 1), and n added to the result's exponent field.
+// Inputs below -126 are treated as -126 (a weight of 2^-126 instead of less).
+__device__ __forceinline__ uint64_t exp2_poly2(uint64_t x2)
+{
+    constexpr float kMagic = 12582912.f;
+    float x0, x1;
+    unpack2(x2, x0, x1);
+    x0 = fmaxf(x0, -126.f);
+    x1 = fmaxf(x1, -126.f);
+    x2 = pack2(x0, x1);
+    const uint64_t r2 = add2_rm(x2, pack2(kMagic, kMagic));
+    const uint64_t n2 = add2(r2, pack2(-kMagic, -kMagic));                  // floor(x), exact
+    const uint64_t f2 = fma2(n2, pack2(-1.f, -1.f), x2);                    // x - floor(x), exact
+    uint64_t y2 = fma2(f2, pack2(0.07802491635f, 0.07802491635f), pack2(0.22606660426f, 0.22606660426f));
+    y2 = fma2(y2, f2, pack2(0.69583368301f, 0.69583368301f));
+    y2 = fma2(y2, f2, pack2(0.99992519617f, 0.99992519617f));
+    float y0, y1, r0, r1;
+    unpack2(y2, y0, y1);
+    unpack2(r2, r0, r1);
+    y0 = as_f(as_u(y0) + (as_u(r0) << 23));
+    y1 = as_f(as_u(y1) + (as_u(r1) << 23));
+    return pack2(y0, y1);
+}
+
+// -inf into the registers of one 64-column piece (first column col0) whose key is not valid.
+__device__ __forceinline__ void mask_piece(uint32_t *v, int col0, int cq, int nvalid)
+{
+#pragma unroll
+    for (int k = 0; k < 8; ++k) {
+        if (col0 + 8 * k + cq >= nvalid) v[4 * k] = v[4 * k + 2] = 0xff800000u;
+        if (col0 + 8 * k + cq + 1 >= nvalid) v[4 * k + 1] = v[4 * k + 3] = 0xff800000u;
+    }
 }
 
 template <int D>
@@ -138,23 +256,13 @@ attn_sm100_kernel(const __grid_constant__ AttnParams p, const __grid_constant__ 
 
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
-    const int head = blockIdx.y;
-
-    // ---- which query rows and which keys ----------------------------------
-    int g = 0;
-    while (g + 1 < p.n_groups && (int)blockIdx.x >= p.g[g + 1].tile_begin) ++g;
-    const AttnGroup &G = p.g[g];
-    const int local_tile = blockIdx.x - G.tile_begin;
-    const int q0 = G.q_begin + local_tile * kQTileRows;                  // first query row of the CTA
-    const int rows_valid = min(kQTileRows, G.q_rows - local_tile * kQTileRows);
-    const int n_sub = rows_valid > 128 ? 2 : 1;                          // live 128-row tiles
-    const int n_kt = count_key_tiles(G);
+    const int cta = blockIdx.x;
 
     // ---- setup ------------------------------------------------------------------
     if (threadIdx.x == 0) {
         for (int i = 0; i < kNumBars; ++i) {
             uint32_t count = 1;
-            if (i == kPFull || i == kPFull + 1) count = 128;
+            if (i == kPFull || i == kPFull + 1 || i == kOEmpty || i == kOEmpty + 1) count = kSoftmaxWarps / 2;
             mbar_init(bar(i), count);
         }
         // an earlier CTA already gave up on a wait: this one does not start (flag value 2)
@@ -172,233 +280,381 @@ attn_sm100_kernel(const __grid_constant__ AttnParams p, const __grid_constant__ 
 
     WaitCtx ctx{abort_flag, p.status, warp};
     const bool skip = *abort_flag != 0;
+    auto wait = [&](int bar_id, uint32_t parity, int iter) -> bool {
+        return wait_bar(bar(bar_id), parity & 1u, ctx, bar_id, iter);
+    };
 
-    // Register reallocation: the softmax warpgroups hold a whole S row per thread, the
-    // producer warpgroup (TMA, MMA and two idle warps) needs little.
-    if (warp >= 8) {
+    if (warp >= kSoftmaxWarps) {
+        // Register reallocation: the softmax warps hold half an S row pair per thread,
+        // the producer warpgroup (TMA, MMA and two idle warps) needs little.
         setmaxnreg_dec<kProducerRegs>();
-    if (skip) {
-        // an earlier CTA gave up: nothing to do
-    } else if (warp == kTmaWarp) {
-        // =========================== TMA producer ===========================
-        if (lane == 0) {
-            prefetch_tensormap(&qmap);
-            prefetch_tensormap(&kmap);
-            prefetch_tensormap(&vmap);
-            for (int w = 0; w < n_sub; ++w) {
-                mbar_arrive_expect_tx(bar(kQFull + w), C::kTileBytes);
-                for (int a = 0; a < C::kAtoms; ++a)
-                    tma_load_3d(q_smem + w * C::kTileBytes + a * C::kAtomBytes, &qmap, bar(kQFull + w),
-                                a * 64, head, q0 + 128 * w);
-            }
-            KeyIter it(&G);
-            bool ok = true;
-            for (int j = 0; j < n_kt && ok; ++j, it.next()) {
-                const int row = it.row();
-                for (int kv = 0; kv < 2 && ok; ++kv) {
-                    const int n = 2 * j + kv;
-                    const int stage = n % C::kStages;
-                    const uint32_t phase = (uint32_t)(n / C::kStages) & 1u;
-                    ok = wait_bar(bar(kKvEmpty + stage), phase ^ 1u, ctx, kKvEmpty + stage, n);
-                    if (!ok) break;
-                    mbar_arrive_expect_tx(bar(kKvFull + stage), C::kTileBytes);
-                    const CUtensorMap *m = kv ? &vmap : &kmap;
-                    for (int a = 0; a < C::kAtoms; ++a)
-                        tma_load_3d(kv_smem + stage * C::kTileBytes + a * C::kAtomBytes, m,
-                                    bar(kKvFull + stage), a * 64, row, head);
+        if (skip) {
+            // an earlier CTA gave up: nothing to do
+        } else if (warp == kTmaWarp && lane == 0) {
+            // =========================== TMA producer ===========================
+            [&]() {
+                prefetch_tensormap(&qmap);
+                prefetch_tensormap(&kmap);
+                prefetch_tensormap(&vmap);
+                uint32_t n = 0;                 // K/V tiles issued so far
+                uint32_t seg = 0;
+                Segment s;
+                for (WorkIter it(p, cta); it.next(s); ++seg) {
+                    KeyIter kit(&p.g[s.g], s.kt0);
+                    auto load_kv = [&](const CUtensorMap *m) -> bool {
+                        const int stage = n % C::kStages;
+                        if (!wait(kKvEmpty + stage, (n / C::kStages) ^ 1u, (int)n)) return false;
+                        mbar_arrive_expect_tx(bar(kKvFull + stage), C::kTileBytes);
+                        for (int a = 0; a < C::kAtoms; ++a)
+                            tma_load_3d(kv_smem + stage * C::kTileBytes + a * C::kAtomBytes, m,
+                                        bar(kKvFull + stage), a * 64, kit.row(), s.head);
+                        ++n;
+                        return true;
+                    };
+                    // the first key tile goes out before Q: it needs no Q buffer and is in
+                    // flight while the previous column's last products drain
+                    if (!load_kv(&kmap) || !load_kv(&vmap)) return;
+                    if (seg > 0 && !wait(kQEmpty, seg - 1, (int)seg)) return;
+                    for (int w = 0; w < s.n_sub; ++w) {
+                        mbar_arrive_expect_tx(bar(kQFull + w), C::kTileBytes);
+                        for (int a = 0; a < C::kAtoms; ++a)
+                            tma_load_3d(q_smem + w * C::kTileBytes + a * C::kAtomBytes, &qmap, bar(kQFull + w),
+                                        a * 64, s.head, s.q0 + 128 * w);
+                    }
+                    for (int j = s.kt0 + 1; j < s.kt1; ++j) {
+                        kit.next();
+                        if (!load_kv(&kmap) || !load_kv(&vmap)) return;
+                    }
                 }
-            }
-        }
-    } else if (warp == kMmaWarp) {
-        // ============================ MMA issuer ============================
-        if (lane == 0) {
-            constexpr uint32_t idesc_qk = idesc_bf16_f32(128, 128, 0, 0);
-            constexpr uint32_t idesc_pv = idesc_bf16_f32(128, D, 0, 1);
-            // S_w = Q_w K^T: both operands K-major, 64-element atoms, 16 elements (32 bytes) per MMA
-            auto issue_qk = [&](int w, int stage) {
-                const uint32_t qa = q_smem + w * C::kTileBytes;
-                const uint32_t kb = kv_smem + stage * C::kTileBytes;
+            }();
+        } else if (warp == kMmaWarp && lane == 0) {
+            // ============================ MMA issuer ============================
+            [&]() {
+                constexpr uint32_t idesc_qk = idesc_bf16_f32(128, 128, 0, 0);
+                constexpr uint32_t idesc_pv = idesc_bf16_f32(128, D, 0, 1);
+                // S_w = Q_w K^T: both operands K-major, 64-element atoms, 16 elements (32 bytes) per MMA
+                auto issue_qk = [&](int w, int stage) {
+                    const uint32_t qa = q_smem + w * C::kTileBytes;
+                    const uint32_t kb = kv_smem + stage * C::kTileBytes;
 #pragma unroll
-                for (int kk = 0; kk < D / 16; ++kk) {
-                    const uint32_t off = (kk / 4) * C::kAtomBytes + (kk % 4) * 32;
-                    mma_ss(tmem + C::kColS + 128 * w, smem_desc_sw128(qa + off, 16, 1024),
-                           smem_desc_sw128(kb + off, 16, 1024), idesc_qk, kk > 0);
-                }
-            };
-            // O_w += P_w V: P from TMEM (16 keys = 8 packed columns per MMA); V is MN-major:
-            // 8-key groups 1024 bytes apart, 64-wide d atoms kAtomBytes apart
-            auto issue_pv = [&](int w, int stage, bool first) {
-                const uint32_t vb = kv_smem + stage * C::kTileBytes;
+                    for (int kk = 0; kk < D / 16; ++kk) {
+                        const uint32_t off = (kk / 4) * C::kAtomBytes + (kk % 4) * 32;
+                        mma_ss(tmem + C::kColS + 128 * w, smem_desc_sw128(qa + off, 16, 1024),
+                               smem_desc_sw128(kb + off, 16, 1024), idesc_qk, kk > 0);
+                    }
+                };
+                // O_w += P_w V: P from TMEM (16 keys = 8 packed columns per MMA); V is MN-major:
+                // 8-key groups 1024 bytes apart, 64-wide d atoms kAtomBytes apart
+                auto issue_pv = [&](int w, int stage, bool first) {
+                    const uint32_t vb = kv_smem + stage * C::kTileBytes;
 #pragma unroll
-                for (int kk = 0; kk < kKeyTile / 16; ++kk) {
-                    mma_ts(tmem + C::kColO + D * w, tmem + C::kColS + 128 * w + 8 * kk,
-                           smem_desc_sw128(vb + kk * 2048, C::kAtomBytes, 1024), idesc_pv,
-                           (!first || kk > 0) ? 1u : 0u);
-                }
-            };
-            bool ok = true;
-            for (int w = 0; w < n_sub && ok; ++w) ok = wait_bar(bar(kQFull + w), 0, ctx, kQFull + w, 0);
-            if (ok) ok = wait_bar(bar(kKvFull + 0), 0, ctx, kKvFull, 0);
-            if (ok) {
-                tc_fence_after_sync();
-                for (int w = 0; w < n_sub; ++w) {
-                    issue_qk(w, 0);
-                    tc_commit(bar(kSFull + w));
-                }
-                tc_commit(bar(kKvEmpty + 0));
-            }
-            for (int j = 0; j < n_kt && ok; ++j) {
-                const int nv = 2 * j + 1, nk = 2 * j + 2;
-                const int sv = nv % C::kStages, sk = nk % C::kStages;
-                const bool more = j + 1 < n_kt;
-                ok = wait_bar(bar(kKvFull + sv), (uint32_t)(nv / C::kStages) & 1u, ctx, kKvFull + sv, nv);
-                if (ok && more) ok = wait_bar(bar(kKvFull + sk), (uint32_t)(nk / C::kStages) & 1u, ctx, kKvFull + sk, nk);
-                for (int w = 0; w < n_sub && ok; ++w) {
-                    ok = wait_bar(bar(kPFull + w), (uint32_t)j & 1u, ctx, kPFull + w, j);
-                    if (!ok) break;
+                    for (int kk = 0; kk < kKeyTile / 16; ++kk) {
+                        mma_ts(tmem + C::kColO + D * w, tmem + C::kColS + 128 * w + 8 * kk,
+                               smem_desc_sw128(vb + kk * 2048, C::kAtomBytes, 1024), idesc_pv,
+                               (!first || kk > 0) ? 1u : 0u);
+                    }
+                };
+                uint32_t n = 0;                 // K/V tiles consumed so far
+                uint32_t sc[2] = {0, 0};        // steps lane w has been through
+                uint32_t oc[2] = {0, 0};        // columns lane w took part in so far
+                Segment s;
+                for (WorkIter it(p, cta); it.next(s);) {
+                    const int n_steps = s.kt1 - s.kt0;
+                    for (int w = 0; w < s.n_sub; ++w)
+                        if (!wait(kQFull + w, oc[w], 0)) return;
+                    if (!wait(kKvFull + n % C::kStages, n / C::kStages, (int)n)) return;
                     tc_fence_after_sync();
-                    issue_pv(w, sv, j == 0);
-                    if (more) {
-                        issue_qk(w, sk);
+                    for (int w = 0; w < s.n_sub; ++w) {
+                        issue_qk(w, n % C::kStages);
                         tc_commit(bar(kSFull + w));
-                    } else {
-                        tc_commit(bar(kOFull + w));
                     }
+                    tc_commit(bar(kKvEmpty + n % C::kStages));
+                    ++n;
+                    if (n_steps == 1) tc_commit(bar(kQEmpty));
+                    for (int j = 0; j < n_steps; ++j) {
+                        const bool more = j + 1 < n_steps;
+                        const int sv = n % C::kStages, sk = (n + 1) % C::kStages;
+                        if (!wait(kKvFull + sv, n / C::kStages, (int)n)) return;
+                        if (more && !wait(kKvFull + sk, (n + 1) / C::kStages, (int)n + 1)) return;
+                        for (int w = 0; w < s.n_sub; ++w) {
+                            if (!wait(kPFull + w, sc[w], (int)sc[w])) return;
+                            ++sc[w];
+                            // the previous column's O rows must have been read out
+                            if (j == 0 && oc[w] > 0 && !wait(kOEmpty + w, oc[w] - 1, (int)oc[w])) return;
+                            tc_fence_after_sync();
+                            issue_pv(w, sv, j == 0);
+                            if (more) {
+                                issue_qk(w, sk);
+                                tc_commit(bar(kSFull + w));
+                            } else {
+                                tc_commit(bar(kOFull + w));
+                            }
+                        }
+                        tc_commit(bar(kKvEmpty + sv));
+                        ++n;
+                        if (more) {
+                            tc_commit(bar(kKvEmpty + sk));
+                            ++n;
+                        }
+                        if (j + 2 == n_steps) tc_commit(bar(kQEmpty));   // the column's last QK is in the pipe
+                    }
+                    for (int w = 0; w < s.n_sub; ++w) ++oc[w];
                 }
-                if (ok) {
-                    tc_commit(bar(kKvEmpty + sv));
-                    if (more) tc_commit(bar(kKvEmpty + sk));
-                }
-            }
+            }();
         }
-    }
     } else {
-        // ========================= softmax warpgroups =========================
+        // ============================= softmax warps =============================
         setmaxnreg_inc<kSoftmaxRegs>();
-        const int w = warp >> 2;                       // query tile of this warpgroup
-        if (!skip && w < n_sub) {
-            const int r = threadIdx.x & 127;           // row inside the tile = TMEM lane
-            const uint32_t lane_base = (uint32_t)((warp & 3) * 32) << 16;
-            const uint32_t t_s = tmem + lane_base + C::kColS + 128 * w;
-            const uint32_t t_o = tmem + lane_base + C::kColO + D * w;
+        if (!skip) [&]() {
+            const int q = warp & 3;                        // TMEM lane quarter this warp may touch
+            const int w = warp >> 3;                       // lane (query tile) of the column
+            const int h = (warp >> 2) & 1;                 // which 16 rows of the quarter
+            const uint32_t lane_off = (uint32_t)(32 * q + 16 * h) << 16;
+            const uint32_t t_s = tmem + lane_off + C::kColS + 128 * w;
+            const uint32_t t_o = tmem + lane_off + C::kColO + D * w;
+            const int row_a = 32 * q + 16 * h + (lane >> 2);   // row of registers 4k+{0,1}; 4k+{2,3} are row_a + 8
+            const int cq = 2 * (lane & 3);                     // first of this thread's two columns in each group of 8
+            const int slab = w * 8 + q * 2 + h;
             const float c = p.scale_log2;
-            float m = -INFINITY, l = 0.f;
-            KeyIter it(&G);
-            bool ok = true;
-            for (int j = 0; j < n_kt; ++j, it.next()) {
-                ok = __all_sync(0xffffffffu, wait_bar(bar(kSFull + w), (uint32_t)j & 1u, ctx, kSFull + w, j));
-                if (!ok) break;
-                tc_fence_after_sync();
-                const int nvalid = it.valid();
-                // ---- pass 1: row max of the tile (the values are fetched again below) ----
-                float m_tile;
-                uint32_t ca[32], cb[32];
-                {
-                    uint32_t v[128];
+            const uint64_t c2 = pack2(c, c);
+            uint32_t sc = 0, oc = 0;
+            Segment s;
+            for (WorkIter it(p, cta); it.next(s);) {
+                if (w >= s.n_sub) continue;
+                const AttnGroup &G = p.g[s.g];
+                KeyIter kit(&G, s.kt0);
+                float m_a = -INFINITY, m_b = -INFINITY;
+                uint64_t acc_a = 0ull, acc_b = 0ull;       // two partial sums per row
+                for (int j = s.kt0; j < s.kt1; ++j, kit.next(), ++sc) {
+                    if (!__all_sync(0xffffffffu, wait(kSFull + w, sc, j))) return;
+                    tc_fence_after_sync();
+                    const int nvalid = kit.valid();
+                    // ---- pass 1: row maxima of the tile: 32 columns per thread, then across the
+                    //      quad (the values are fetched again below) ----
+                    float ta = -INFINITY, tb = -INFINITY;
+                    uint32_t va[32];
 #pragma unroll
-                    for (int i = 0; i < 4; ++i) tmem_ld32(t_s + 32 * i, v + 32 * i);
-                    tmem_wait_ld();
-                    tmem_ld32(t_s, ca);                    // chunk 0 of pass 2, in flight during the max
-                    if (nvalid < kKeyTile) {
+                    for (int piece = 0; piece < 2; ++piece) {
+                        tmem_ld_16x256b_x8(t_s + 64 * piece, va);
+                        tmem_wait_ld();
+                        if (nvalid < kKeyTile) mask_piece(va, 64 * piece, cq, nvalid);
 #pragma unroll
-                        for (int i = 0; i < 128; ++i)
-                            if (i >= nvalid) v[i] = 0xff800000u;   // -inf
+                        for (int k = 0; k < 8; ++k) {
+                            ta = max3(ta, as_f(va[4 * k]), as_f(va[4 * k + 1]));
+                            tb = max3(tb, as_f(va[4 * k + 2]), as_f(va[4 * k + 3]));
+                        }
                     }
-                    float mc[4];
+                    tmem_ld_16x256b_x8(t_s, va);               // first piece of pass 2, in flight during the shuffles
+                    ta = fmaxf(ta, __shfl_xor_sync(0xffffffffu, ta, 1));
+                    tb = fmaxf(tb, __shfl_xor_sync(0xffffffffu, tb, 1));
+                    ta = fmaxf(ta, __shfl_xor_sync(0xffffffffu, ta, 2)) * c;
+                    tb = fmaxf(tb, __shfl_xor_sync(0xffffffffu, tb, 2)) * c;
+                    if (j == s.kt0) {
+                        m_a = ta;
+                        m_b = tb;
+                    } else {
+                        const bool grow_a = ta > m_a + kRescaleThreshold, grow_b = tb > m_b + kRescaleThreshold;
+                        if (__any_sync(0xffffffffu, grow_a || grow_b)) {
+                            // rescale the running sums and the O rows; PV of tile j-1 has completed
+                            // (the commit that released S_j covers it) and PV of tile j is not issued yet
+                            const float al_a = grow_a ? ex2(m_a - ta) : 1.f, al_b = grow_b ? ex2(m_b - tb) : 1.f;
+                            if (grow_a) m_a = ta;
+                            if (grow_b) m_b = tb;
+                            acc_a = fma2(acc_a, pack2(al_a, al_a), 0ull);
+                            acc_b = fma2(acc_b, pack2(al_b, al_b), 0ull);
+                            tmem_wait_ld();
+#pragma unroll 1
+                            for (int ch = 0; ch < C::kOChunks; ++ch) {
+                                uint32_t o[32];
+                                tmem_ld_16x256b_x8(t_o + 64 * ch, o);
+                                tmem_wait_ld();
 #pragma unroll
-                    for (int ch = 0; ch < 4; ++ch) {
-                        mc[ch] = fmaxf(__uint_as_float(v[32 * ch]), __uint_as_float(v[32 * ch + 1]));
-#pragma unroll
-                        for (int i = 2; i < 32; i += 2)
-                            mc[ch] = max3(mc[ch], __uint_as_float(v[32 * ch + i]), __uint_as_float(v[32 * ch + i + 1]));
+                                for (int k = 0; k < 8; ++k) {
+                                    o[4 * k] = as_u(as_f(o[4 * k]) * al_a);
+                                    o[4 * k + 1] = as_u(as_f(o[4 * k + 1]) * al_a);
+                                    o[4 * k + 2] = as_u(as_f(o[4 * k + 2]) * al_b);
+                                    o[4 * k + 3] = as_u(as_f(o[4 * k + 3]) * al_b);
+                                }
+                                tmem_st_16x256b_x8(t_o + 64 * ch, o);
+                            }
+                        }
                     }
-                    m_tile = max3(mc[0], mc[1], fmaxf(mc[2], mc[3])) * c;
+                    // ---- pass 2: p = 2^(s*c - m) in two 64-key pieces; each piece's P (bf16, 32
+                    //      packed columns) lands on S columns this warp no longer needs ----
+                    const uint64_t na2 = pack2(-m_a, -m_a), nb2 = pack2(-m_b, -m_b);
+#pragma unroll
+                    for (int piece = 0; piece < 2; ++piece) {
+                        tmem_wait_ld();
+                        if (nvalid < kKeyTile) mask_piece(va, 64 * piece, cq, nvalid);
+                        uint32_t pk[16];
+#pragma unroll
+                        for (int k = 0; k < 8; ++k) {
+                            const uint64_t xa = fma2(pack2(as_f(va[4 * k]), as_f(va[4 * k + 1])), c2, na2);
+                            const uint64_t xb = fma2(pack2(as_f(va[4 * k + 2]), as_f(va[4 * k + 3])), c2, nb2);
+                            uint64_t pa, pb;
+                            if ((kPolyMask >> (8 * piece + k)) & 1u) {
+                                pa = exp2_poly2(xa);
+                                pb = exp2_poly2(xb);
+                            } else {
+                                pa = exp2_sfu2(xa);
+                                pb = exp2_sfu2(xb);
+                            }
+                            acc_a = add2(acc_a, pa);
+                            acc_b = add2(acc_b, pb);
+                            float a0, a1, b0, b1;
+                            unpack2(pa, a0, a1);
+                            unpack2(pb, b0, b1);
+                            pk[2 * k] = cvt_bf16x2(a0, a1);            // key 8k + cq in the low half
+                            pk[2 * k + 1] = cvt_bf16x2(b0, b1);
+                        }
+                        if (piece == 0) tmem_ld_16x256b_x8(t_s + 64, va);   // S columns 64..127
+                        tmem_st_16x128b_x8(t_s + 32 * piece, pk);
+                    }
+                    tmem_wait_st();
+                    tc_fence_before_sync();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(bar(kPFull + w));
                 }
-                if (j == 0) {
-                    m = m_tile;
-                } else {
-                    const bool grow = m_tile > m + kRescaleThreshold;
-                    if (__any_sync(0xffffffffu, grow)) {
-                        // rescale the running sum and the O row; PV of tile j-1 has completed
-                        // (the commit that released S_j covers it) and PV of tile j is not issued yet
-                        const float alpha = grow ? ex2(m - m_tile) : 1.f;
-                        if (grow) m = m_tile;
-                        l *= alpha;
+
+                // ---- the column's (or this part's) O rows are complete ----
+                if (!__all_sync(0xffffffffu, wait(kOFull + w, oc, s.kt1))) return;
+                tc_fence_after_sync();
+                float l_a, l_b;
+                {
+                    float x0, x1;
+                    unpack2(acc_a, x0, x1);
+                    l_a = x0 + x1;
+                    unpack2(acc_b, x0, x1);
+                    l_b = x0 + x1;
+                    l_a += __shfl_xor_sync(0xffffffffu, l_a, 1);
+                    l_b += __shfl_xor_sync(0xffffffffu, l_b, 1);
+                    l_a += __shfl_xor_sync(0xffffffffu, l_a, 2);
+                    l_b += __shfl_xor_sync(0xffffffffu, l_b, 2);
+                }
+                const int row = 128 * w + row_a;               // row inside the column
+                const bool live_a = row < s.rows_valid, live_b = row + 8 < s.rows_valid;
+                ll_bf16 *dst_a = p.out + ((size_t)(s.q0 + row) * p.heads + s.head) * D;
+                ll_bf16 *dst_b = dst_a + (size_t)8 * p.heads * D;
+                float *lse_a = p.lse ? p.lse + (size_t)s.head * p.nq_total + s.q0 + row : nullptr;
+
+                bool finish = true;            // this warp writes the output rows
+                int i0 = 0, n_parts = 1;
+                const bool whole = s.kt0 == 0 && s.kt1 == G.n_kt;
+                const size_t slot_floats = (size_t)kQTileRows * (D + 2);
+                if (!whole) {
+                    // leave this part in its slot and count the arrival
+                    i0 = cta_of_step(p, s.col_begin);
+                    n_parts = cta_of_step(p, s.col_begin + G.n_kt - 1) - i0 + 1;
+                    float *slot = p.partial + (size_t)(2 * cta + (s.kt0 == 0 ? 1 : 0)) * slot_floats;
+#pragma unroll 1
+                    for (int ch = 0; ch < C::kOChunks; ++ch) {
+                        uint32_t o[32];
+                        tmem_ld_16x256b_x8(t_o + 64 * ch, o);
+                        tmem_wait_ld();
 #pragma unroll
-                        for (int i = 0; i < D / 32; ++i) {
-                            uint32_t o[32];
-                            tmem_ld32(t_o + 32 * i, o);
+                        for (int k = 0; k < 8; ++k) {
+                            float2 *dst = reinterpret_cast<float2 *>(slot) +
+                                          ((size_t)(slab * (D / 8) + 8 * ch + k) * 2) * 32 + lane;
+                            dst[0] = make_float2(as_f(o[4 * k]), as_f(o[4 * k + 1]));
+                            dst[32] = make_float2(as_f(o[4 * k + 2]), as_f(o[4 * k + 3]));
+                        }
+                    }
+                    if ((lane & 3) == 0) {
+                        float2 *ml = reinterpret_cast<float2 *>(slot + (size_t)kQTileRows * D) + slab * 16 + (lane >> 2);
+                        ml[0] = make_float2(m_a, l_a);
+                        ml[8] = make_float2(m_b, l_b);
+                    }
+                    __threadfence();
+                    __syncwarp();
+                    uint32_t arrived = 0;
+                    if (lane == 0) arrived = atomicAdd(p.counters + i0 * kSlabs + slab, 1u);
+                    arrived = __shfl_sync(0xffffffffu, arrived, 0);
+                    finish = arrived == (uint32_t)(n_parts - 1);
+                    if (finish) {
+                        if (lane == 0) p.counters[i0 * kSlabs + slab] = 0;    // ready for the next launch
+                        __threadfence();
+                    }
+                }
+                if (finish) {
+                    // the slot of part i, and this thread's two (max, sum) pairs in it
+                    auto part_slot = [&](int i) -> const float * {
+                        return p.partial + (size_t)(2 * i + (i == i0 ? 1 : 0)) * slot_floats;
+                    };
+                    auto part_ml = [&](const float *slot) -> const float2 * {
+                        return reinterpret_cast<const float2 *>(slot + (size_t)kQTileRows * D) + slab * 16 + (lane >> 2);
+                    };
+                    // Reference maximum and sum over all parts.  A split column is merged from the
+                    // slots alone, the own part included, in the order of the parts, so the result
+                    // does not depend on which part happened to arrive last.
+                    float mm_a = m_a, mm_b = m_b, ll_a = l_a, ll_b = l_b;
+                    if (!whole) {
+                        for (int i = i0; i < i0 + n_parts; ++i) {
+                            const float2 *ml = part_ml(part_slot(i));
+                            mm_a = fmaxf(mm_a, __ldcg(ml).x);
+                            mm_b = fmaxf(mm_b, __ldcg(ml + 8).x);
+                        }
+                        ll_a = ll_b = 0.f;
+                        for (int i = i0; i < i0 + n_parts; ++i) {
+                            const float2 *ml = part_ml(part_slot(i));
+                            const float2 pa = __ldcg(ml), pb = __ldcg(ml + 8);
+                            ll_a = fmaf(pa.y, ex2(pa.x - mm_a), ll_a);
+                            ll_b = fmaf(pb.y, ex2(pb.x - mm_b), ll_b);
+                        }
+                    }
+                    const float inv_a = 1.f / ll_a, inv_b = 1.f / ll_b;
+#pragma unroll 1
+                    for (int ch = 0; ch < C::kOChunks; ++ch) {
+                        uint32_t o[32];
+                        if (whole) {
+                            tmem_ld_16x256b_x8(t_o + 64 * ch, o);
                             tmem_wait_ld();
 #pragma unroll
-                            for (int u = 0; u < 32; ++u) o[u] = __float_as_uint(__uint_as_float(o[u]) * alpha);
-                            tmem_st32(t_o + 32 * i, o);
+                            for (int k = 0; k < 8; ++k) {
+                                o[4 * k] = as_u(as_f(o[4 * k]) * inv_a);
+                                o[4 * k + 1] = as_u(as_f(o[4 * k + 1]) * inv_a);
+                                o[4 * k + 2] = as_u(as_f(o[4 * k + 2]) * inv_b);
+                                o[4 * k + 3] = as_u(as_f(o[4 * k + 3]) * inv_b);
+                            }
+                        } else {
+#pragma unroll
+                            for (int k = 0; k < 32; ++k) o[k] = 0u;
+                            for (int i = i0; i < i0 + n_parts; ++i) {
+                                const float *slot = part_slot(i);
+                                const float2 *ml = part_ml(slot);
+                                const float wa = ex2(__ldcg(ml).x - mm_a) * inv_a, wb = ex2(__ldcg(ml + 8).x - mm_b) * inv_b;
+#pragma unroll
+                                for (int k = 0; k < 8; ++k) {
+                                    const float2 *src = reinterpret_cast<const float2 *>(slot) +
+                                                        ((size_t)(slab * (D / 8) + 8 * ch + k) * 2) * 32 + lane;
+                                    const float2 xa = __ldcg(src), xb = __ldcg(src + 32);
+                                    o[4 * k] = as_u(fmaf(xa.x, wa, as_f(o[4 * k])));
+                                    o[4 * k + 1] = as_u(fmaf(xa.y, wa, as_f(o[4 * k + 1])));
+                                    o[4 * k + 2] = as_u(fmaf(xb.x, wb, as_f(o[4 * k + 2])));
+                                    o[4 * k + 3] = as_u(fmaf(xb.y, wb, as_f(o[4 * k + 3])));
+                                }
+                            }
+                        }
+#pragma unroll
+                        for (int k = 0; k < 8; ++k) {
+                            const int col = 64 * ch + 8 * k + cq;
+                            if (live_a)
+                                *reinterpret_cast<uint32_t *>(dst_a + col) = cvt_bf16x2(as_f(o[4 * k]), as_f(o[4 * k + 1]));
+                            if (live_b)
+                                *reinterpret_cast<uint32_t *>(dst_b + col) = cvt_bf16x2(as_f(o[4 * k + 2]), as_f(o[4 * k + 3]));
                         }
                     }
-                }
-                // ---- pass 2: p = 2^(s*c - m) in 32-key chunks; P chunk k (16 packed columns)
-                //      lands on S columns that chunks <= k no longer need ----
-                const uint64_t c2 = pack2(c, c);
-                const uint64_t nm2 = pack2(-m, -m);
-                uint64_t acc[2] = {0ull, 0ull};
-#pragma unroll
-                for (int k = 0; k < 4; ++k) {
-                    uint32_t *cur = (k & 1) ? cb : ca;
-                    uint32_t *nxt = (k & 1) ? ca : cb;
-                    tmem_wait_ld();
-                    if (k < 3) tmem_ld32(t_s + 32 * (k + 1), nxt);
-                    if (nvalid < kKeyTile) {
-#pragma unroll
-                        for (int i = 0; i < 32; ++i)
-                            if (32 * k + i >= nvalid) cur[i] = 0xff800000u;
+                    if (lse_a && (lane & 3) == 0) {
+                        if (live_a) lse_a[0] = (mm_a + log2f(ll_a)) * 0.6931471805599453f;
+                        if (live_b) lse_a[8] = (mm_b + log2f(ll_b)) * 0.6931471805599453f;
                     }
-                    uint32_t pk[16];
-#pragma unroll
-                    for (int i = 0; i < 16; ++i) {
-                        const uint64_t t2 = fma2(pack2(__uint_as_float(cur[2 * i]), __uint_as_float(cur[2 * i + 1])), c2, nm2);
-                        float t0, t1;
-                        unpack2(t2, t0, t1);
-                        const float p0 = ex2(t0), p1 = ex2(t1);
-                        acc[i & 1] = add2(acc[i & 1], pack2(p0, p1));
-                        pk[i] = pack_bf16(p0, p1);         // key 2i in the low half
-                    }
-                    tmem_st16(t_s + 16 * k, pk);
                 }
-                float sum0, sum1;
-                unpack2(add2(acc[0], acc[1]), sum0, sum1);
-                l += sum0 + sum1;
-                tmem_wait_st();
+                // the O columns may be overwritten by the next column's first PV
                 tc_fence_before_sync();
-                mbar_arrive(bar(kPFull + w));
+                __syncwarp();
+                if (lane == 0) mbar_arrive(bar(kOEmpty + w));
+                ++oc;
             }
-            // ---- epilogue: O / l -> bf16 -> global ---------------------------
-            if (ok) ok = __all_sync(0xffffffffu, wait_bar(bar(kOFull + w), 0, ctx, kOFull + w, n_kt));
-            if (ok) {
-                tc_fence_after_sync();
-                const int row = 128 * w + r;
-                const bool live = row < rows_valid;
-                const float inv_l = 1.f / l;
-                ll_bf16 *dst = p.out + ((size_t)(q0 + row) * p.heads + head) * D;
-#pragma unroll
-                for (int i = 0; i < D / 32; ++i) {
-                    uint32_t o[32];
-                    tmem_ld32(t_o + 32 * i, o);
-                    tmem_wait_ld();
-                    if (live) {
-#pragma unroll
-                        for (int u = 0; u < 4; ++u) {
-                            uint4 pk;
-                            pk.x = pack_bf16(__uint_as_float(o[8 * u + 0]) * inv_l, __uint_as_float(o[8 * u + 1]) * inv_l);
-                            pk.y = pack_bf16(__uint_as_float(o[8 * u + 2]) * inv_l, __uint_as_float(o[8 * u + 3]) * inv_l);
-                            pk.z = pack_bf16(__uint_as_float(o[8 * u + 4]) * inv_l, __uint_as_float(o[8 * u + 5]) * inv_l);
-                            pk.w = pack_bf16(__uint_as_float(o[8 * u + 6]) * inv_l, __uint_as_float(o[8 * u + 7]) * inv_l);
-                            *reinterpret_cast<uint4 *>(dst + 32 * i + 8 * u) = pk;
-                        }
-                    }
-                }
-                if (live && p.lse)
-                    p.lse[(size_t)head * p.nq_total + q0 + row] = (m + log2f(l)) * 0.6931471805599453f;
-            }
-        }
+        }();
     }
 
     // ---- common exit -------------------------------------------------------------
@@ -423,8 +679,14 @@ attn_sm100_kernel(const __grid_constant__ AttnParams p, const __grid_constant__ 
 cudaError_t launch_attn_sm100(const AttnParams &p, int head_dim, const CUtensorMap &qmap, const CUtensorMap &kmap,
                               const CUtensorMap &vmap, cudaStream_t stream)
 {
-    dim3 grid((unsigned)p.total_qtiles, (unsigned)p.heads);
+    if (p.n_ctas <= 0) return cudaSuccess;
+    dim3 grid((unsigned)p.n_ctas);
     cudaError_t e;
+    // the in-kernel register reallocation assumes the launch allocation it was sized for
+    cudaFuncAttributes fa;
+    e = head_dim == 128 ? cudaFuncGetAttributes(&fa, attn_sm100_kernel<128>) : cudaFuncGetAttributes(&fa, attn_sm100_kernel<64>);
+    if (e != cudaSuccess) return e;
+    if (fa.numRegs != kLaunchRegs) return cudaErrorLaunchOutOfResources;
     if (head_dim == 128) {
         e = cudaFuncSetAttribute(attn_sm100_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg<128>::kSmemBytes);
         if (e != cudaSuccess) return e;

@@ -185,23 +185,34 @@ int build_attn_params(ll_cache *c, int layer, const ll_bf16 *q, ll_bf16 *out, fl
     p->kbase = reinterpret_cast<const ll_bf16 *>(c->storage ? layer_k(c, layer) : nullptr);
     p->vbase = reinterpret_cast<const ll_bf16 *>(c->storage ? layer_v(c, layer) : nullptr);
     p->status = reinterpret_cast<uint32_t *>(c->storage ? c->storage + c->off_status : nullptr);
+    p->partial = reinterpret_cast<float *>(c->storage ? c->storage + c->off_partial : nullptr);
+    p->counters = reinterpret_cast<uint32_t *>(c->storage ? c->storage + c->off_counters : nullptr);
     const int rows_per_group = c->C * c->P;
-    int tile = 0;
+    long long steps = 0;
     for (int g = 0; g < n_groups; ++g) {
         ll::AttnGroup &G = p->g[g];
         G.q_begin = g * rows_per_group;
         G.q_rows = rows_per_group;
-        G.tile_begin = tile;
-        tile += (rows_per_group + ll::kQTileRows - 1) / ll::kQTileRows;
+        G.tiles = (rows_per_group + ll::kQTileRows - 1) / ll::kQTileRows;
         int64_t starts[LL_MAX_RANGES], lens[LL_MAX_RANGES];
         int n = 0;
         int st = visible_ranges(c, layer, group_frame_start[g], lo_floor, starts, lens, &n);
         if (st != LL_OK) return st;
         G.n_ranges = n;
-        for (int r = 0; r < n; ++r) { G.k_start[r] = (int)starts[r]; G.k_len[r] = (int)lens[r]; }
+        G.n_kt = 0;
+        for (int r = 0; r < n; ++r) {
+            G.k_start[r] = (int)starts[r];
+            G.k_len[r] = (int)lens[r];
+            G.n_kt += (int)((lens[r] + ll::kKeyTile - 1) / ll::kKeyTile);
+        }
+        G.step_begin = steps;
+        steps += (long long)c->H * G.tiles * G.n_kt;
     }
     p->nq_total = n_groups * rows_per_group;
-    p->total_qtiles = tile;
+    p->total_steps = steps;
+    // one persistent CTA per SM, each taking an equal share of the steps
+    const int sms = c->sm_count > 0 ? c->sm_count : 148;
+    p->n_ctas = (int)std::min<long long>(std::min(sms, ll::kMaxCtas), steps);
     return LL_OK;
 }
 
@@ -293,7 +304,9 @@ int ll_cache_create(int layers, int heads, int head_dim, int tokens_per_frame, i
     c->off_ttab = align_up(ll::kStatusWords * sizeof(uint32_t), 256);
     c->off_hwtab = align_up(c->off_ttab + (size_t)ll::kTTabFrames * n_t * sizeof(float2), 256);
     // grid_h + grid_w <= tokens_per_frame + 1 for any grid with grid_h*grid_w == tokens_per_frame
-    c->aux_bytes = align_up(c->off_hwtab + (size_t)(tokens_per_frame + 1) * n_h * sizeof(float2), 1024);
+    c->off_counters = align_up(c->off_hwtab + (size_t)(tokens_per_frame + 1) * n_h * sizeof(float2), 256);
+    c->off_partial = align_up(c->off_counters + (size_t)ll::kMaxCtas * ll::kSlabs * sizeof(uint32_t), 1024);
+    c->aux_bytes = align_up(c->off_partial + 2 * (size_t)ll::kMaxCtas * ll::attn_slot_bytes(head_dim), 1024);
     c->kv_bytes = (size_t)heads * rows * head_dim * sizeof(ll_bf16);
     *out = c;
     return LL_OK;
@@ -316,6 +329,12 @@ int ll_cache_bind_storage(ll_cache *c, void *dev, size_t bytes, ll_stream stream
     if (c->dry_run) return fail(LL_ERR_INVALID_ARG, "handle is in bookkeeping-only mode");
     cudaError_t e = cudaMemsetAsync(dev, 0, ll_cache_storage_bytes(c), (cudaStream_t)stream);
     if (e != cudaSuccess) return cuda_fail(e, "cudaMemsetAsync(storage)");
+    cudaPointerAttributes attr;
+    int sms = 0;
+    e = cudaPointerGetAttributes(&attr, dev);
+    if (e == cudaSuccess) e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, attr.device);
+    if (e != cudaSuccess) return cuda_fail(e, "query of the storage's device");
+    c->sm_count = sms;
     std::vector<CUtensorMap> km(c->L), vm(c->L);
     char *base = static_cast<char *>(dev) + c->aux_bytes;
     for (int l = 0; l < c->L; ++l) {

@@ -16,8 +16,10 @@ constexpr int kMaxGroups = 24;        // query groups (chunks) one attention lau
 constexpr int kTTabFrames = 256;      // frames covered by the resident t-axis RoPE table
 constexpr int kTTabAlign = 128;       // table base is a multiple of this many frames
 constexpr int kStatusWords = 64;      // uint32 words at the head of the aux block
-constexpr int kQTileRows = 256;       // query rows one CTA owns (two 128-row MMA tiles)
+constexpr int kQTileRows = 256;       // query rows of one work column (two 128-row MMA tiles)
 constexpr int kKeyTile = 128;         // keys per MMA tile
+constexpr int kMaxCtas = 160;         // persistent CTAs one attention launch may use
+constexpr int kSlabs = 16;            // 16-row warp slabs in a work column (2 tiles x 8)
 
 // status word 0 is non-zero when a kernel abandoned a wait; words 1.. hold details
 enum StatusCode : uint32_t {
@@ -31,21 +33,31 @@ struct LayerState {
     int64_t n_appends = 0, n_overwrites = 0, n_evictions = 0, n_recaches = 0, n_attn = 0;
 };
 
-// One group of query rows that share a visible key set.
+// One group of query rows that share a visible key set.  The group's work is
+// heads x tiles columns (a column = kQTileRows query rows of one head), each
+// n_kt steps long (a step = one kKeyTile-key tile); columns are numbered
+// head-major and their steps laid end to end after those of earlier groups.
 struct AttnGroup {
     int q_begin;                      // first query row of the group in the q tensor
     int q_rows;                       // rows in the group
-    int tile_begin;                   // index of the group's first query tile in the grid
+    int tiles;                        // query tiles of kQTileRows rows
+    int n_kt;                         // key tiles (steps) per column
+    long long step_begin;             // steps of all earlier groups
     int n_ranges;
     int k_start[LL_MAX_RANGES];       // visible cache-row runs
     int k_len[LL_MAX_RANGES];
 };
 
+// Bytes of one partial-result slot: both tiles' unnormalised O rows in fp32 plus
+// (reference max, sum) per row.
+inline size_t attn_slot_bytes(int head_dim) { return (size_t)kQTileRows * (head_dim + 2) * sizeof(float); }
+
 struct AttnParams {
     int n_groups;
     int heads;
     int nq_total;                     // rows of q / out
-    int total_qtiles;                 // grid.x
+    int n_ctas;                       // grid.x: persistent CTAs sharing total_steps evenly
+    long long total_steps;            // steps of all groups
     int64_t rows_per_head;            // (S+W)*P
     float scale_log2;                 // log2(e) / sqrt(D)
     const ll_bf16 *q;                 // [nq_total, H, D]
@@ -54,6 +66,8 @@ struct AttnParams {
     const ll_bf16 *kbase;             // layer K: [H][rows][D]
     const ll_bf16 *vbase;             // layer V
     uint32_t *status;                 // aux status words
+    float *partial;                   // 2 * kMaxCtas slots of attn_slot_bytes
+    uint32_t *counters;               // kMaxCtas * kSlabs arrival counters, zero between launches
     AttnGroup g[kMaxGroups];
 };
 
@@ -95,7 +109,8 @@ struct ll_cache {
     char *storage = nullptr;
     size_t storage_bytes = 0;
     // aux block layout (byte offsets from storage)
-    size_t off_status = 0, off_ttab = 0, off_hwtab = 0, aux_bytes = 0;
+    size_t off_status = 0, off_ttab = 0, off_hwtab = 0, off_counters = 0, off_partial = 0, aux_bytes = 0;
+    int sm_count = 0;                 // of the device the storage lives on
     size_t kv_bytes = 0;              // one K (or V) matrix set of one layer: H*rows*D*2
     std::vector<CUtensorMap> kmap, vmap;
 

@@ -13,14 +13,16 @@
 // Inside a CTA (640 threads):
 //   warp 16 (one lane)  TMA producer: the column's Q tiles, then K_j V_j K_j+1 ...
 //                       into a ring of 128-byte-swizzled shared-memory stages
-//   warp 17 (one lane)  MMA issuer: S_w = Q_w K_j^T (operands in shared memory,
-//                       accumulator in TMEM), O_w += P_w V_j (P read from TMEM)
+//   warps 17, 18        MMA issuers of lane 0 and lane 1 (one thread each):
+//                       S_w = Q_w K_j^T (operands in shared memory, accumulator in
+//                       TMEM), O_w += P_w V_j (P read from TMEM)
 //   warps 0-15          softmax: warp (w, q, h) owns the 16 rows 32q + 16h .. of
 //                       lane w; its threads read S with the 16x256b TMEM shape, so
 //                       a row lives in the four threads of a quad and the row
 //                       maximum and sum are two shuffles away.  P (bf16) is
-//                       written back over S; O is rescaled in TMEM only when a
-//                       row's maximum moved by more than 2^8.
+//                       written back over S.  The rows' reference maxima move, and
+//                       O is rescaled in TMEM, only when a weight computed against
+//                       the old reference would have been large.
 //   While the softmax warps of one lane work, the tensor pipe runs the other
 //   lane's MMAs.  A share of the exponentials is evaluated with a cubic on the
 //   FMA pipe instead of the special-function unit, which both lanes would
@@ -50,7 +52,8 @@ constexpr int kSoftmaxWarps = 16;
 constexpr int kTmaWarp = 16;
 constexpr int kMmaWarp = 17;
 constexpr uint64_t kWaitLimitNs = 2000000000ull;    // 2 s
-constexpr float kRescaleThreshold = 8.f;            // log2 units
+// a piece's 16 weights per thread and row were safe to compute if they sum to at most this
+constexpr float kSafeSum = 256.f;
 // Register reallocation draws on what the CTA was launched with: 640 threads x 96
 // registers = (16 softmax warps x 104 + 4 producer-group warps x 64) x 32.  A
 // request beyond that total would block forever.
@@ -82,7 +85,7 @@ struct Cfg {
 // barrier indices inside the shared barrier array (+ lane or + stage)
 enum Bar {
     kQFull = 0, kQEmpty = 2, kSFull = 4, kPFull = 6, kOFull = 8, kOEmpty = 10,
-    kKvFull = 12, kKvEmpty = 20, kNumBars = 28
+    kKvFull = 12, kKvEmpty = 20, kTurn = 28, kNumBars = 30
 };
 
 // Walks the visible key tiles of a group: runs in order, 128 rows at a time.
@@ -205,14 +208,15 @@ __device__ __forceinline__ uint64_t exp2_sfu2(uint64_t x2)
 // 2^x for two values on the FMA pipe: x = n + f with n = floor(x) taken from the
 // low mantissa bits of x + 1.5 * 2^23 (rounded down), 2^f by a cubic with maximum
 // relative error 7.5e-5 on [0, 1), and n added to the result's exponent field.
-// Inputs below -126 are treated as -126 (a weight of 2^-126 instead of less).
+// Inputs are clamped to [-126, 127]: below, a weight of 2^-126 instead of less; above, a
+// huge finite weight that the caller's safety check on the sums catches (NaN stays NaN).
 __device__ __forceinline__ uint64_t exp2_poly2(uint64_t x2)
 {
     constexpr float kMagic = 12582912.f;
     float x0, x1;
     unpack2(x2, x0, x1);
-    x0 = fmaxf(x0, -126.f);
-    x1 = fmaxf(x1, -126.f);
+    x0 = fminf(fmaxf(x0, -126.f), 127.f);
+    x1 = fminf(fmaxf(x1, -126.f), 127.f);
     x2 = pack2(x0, x1);
     const uint64_t r2 = add2_rm(x2, pack2(kMagic, kMagic));
     const uint64_t n2 = add2(r2, pack2(-kMagic, -kMagic));                  // floor(x), exact
@@ -254,7 +258,9 @@ attn_sm100_kernel(const __grid_constant__ AttnParams p, const __grid_constant__ 
     volatile int *abort_flag = reinterpret_cast<volatile int *>(tmem_slot + 1);
     auto bar = [&](int i) -> uint32_t { return bars + 8u * (uint32_t)i; };
 
-    const int warp = threadIdx.x >> 5;
+    // (the shuffle tells the compiler that the warp index is the same in all lanes, which
+    // keeps the role code of the MMA warps on the uniform datapath)
+    const int warp = __shfl_sync(0xffffffffu, (int)(threadIdx.x >> 5), 0);
     const int lane = threadIdx.x & 31;
     const int cta = blockIdx.x;
 
@@ -263,6 +269,7 @@ attn_sm100_kernel(const __grid_constant__ AttnParams p, const __grid_constant__ 
         for (int i = 0; i < kNumBars; ++i) {
             uint32_t count = 1;
             if (i == kPFull || i == kPFull + 1 || i == kOEmpty || i == kOEmpty + 1) count = kSoftmaxWarps / 2;
+            if (i == kQEmpty || (i >= kKvEmpty && i < kTurn)) count = 2;       // both MMA warps release Q and every K/V stage
             mbar_init(bar(i), count);
         }
         // an earlier CTA already gave up on a wait: this one does not start (flag value 2)
@@ -327,78 +334,122 @@ attn_sm100_kernel(const __grid_constant__ AttnParams p, const __grid_constant__ 
                     }
                 }
             }();
-        } else if (warp == kMmaWarp && lane == 0) {
-            // ============================ MMA issuer ============================
+        } else if (warp == kMmaWarp || warp == kMmaWarp + 1) {
+            // ====================== MMA issuer of lane w = warp - kMmaWarp ======================
+            // One issuing warp per lane: each runs its own waits and bookkeeping while the
+            // tensor pipe works on the other lane's products.  Both walk the same K/V ring and
+            // both release every stage (a lane that sits a column out releases it unused).
+            // All 32 lanes walk the loops and the waits, so that addresses and descriptors are
+            // warp-uniform values; one elected lane issues the MMAs, commits and arrivals.
             [&]() {
+                const int w = warp - kMmaWarp;
+                const bool elected = elect_one();
                 constexpr uint32_t idesc_qk = idesc_bf16_f32(128, 128, 0, 0);
                 constexpr uint32_t idesc_pv = idesc_bf16_f32(128, D, 0, 1);
+                constexpr uint32_t hi = smem_desc_hi_sw128(1024);
+                const uint32_t t_sw = tmem + C::kColS + 128 * w, t_ow = tmem + C::kColO + D * w;
                 // S_w = Q_w K^T: both operands K-major, 64-element atoms, 16 elements (32 bytes) per MMA
-                auto issue_qk = [&](int w, int stage) {
-                    const uint32_t qa = q_smem + w * C::kTileBytes;
-                    const uint32_t kb = kv_smem + stage * C::kTileBytes;
-#pragma unroll
-                    for (int kk = 0; kk < D / 16; ++kk) {
-                        const uint32_t off = (kk / 4) * C::kAtomBytes + (kk % 4) * 32;
-                        mma_ss(tmem + C::kColS + 128 * w, smem_desc_sw128(qa + off, 16, 1024),
-                               smem_desc_sw128(kb + off, 16, 1024), idesc_qk, kk > 0);
-                    }
-                };
+                const uint32_t q_lo = smem_desc_lo(q_smem + w * C::kTileBytes, 16);
+                const uint32_t k_lo0 = smem_desc_lo(kv_smem, 16);
                 // O_w += P_w V: P from TMEM (16 keys = 8 packed columns per MMA); V is MN-major:
                 // 8-key groups 1024 bytes apart, 64-wide d atoms kAtomBytes apart
-                auto issue_pv = [&](int w, int stage, bool first) {
-                    const uint32_t vb = kv_smem + stage * C::kTileBytes;
+                const uint32_t v_lo0 = smem_desc_lo(kv_smem, C::kAtomBytes);
+                auto issue_qk = [&](uint32_t stage) {
+                    const uint32_t k_lo = k_lo0 + stage * (C::kTileBytes >> 4);
+                    if (elected) {
 #pragma unroll
-                    for (int kk = 0; kk < kKeyTile / 16; ++kk) {
-                        mma_ts(tmem + C::kColO + D * w, tmem + C::kColS + 128 * w + 8 * kk,
-                               smem_desc_sw128(vb + kk * 2048, C::kAtomBytes, 1024), idesc_pv,
-                               (!first || kk > 0) ? 1u : 0u);
+                        for (int kk = 0; kk < D / 16; ++kk) {
+                            const uint32_t off = ((kk / 4) * C::kAtomBytes + (kk % 4) * 32) >> 4;
+                            mma_ss(t_sw, smem_desc_join(q_lo + off, hi), smem_desc_join(k_lo + off, hi), idesc_qk, kk > 0);
+                        }
                     }
+                    __syncwarp();
                 };
-                uint32_t n = 0;                 // K/V tiles consumed so far
-                uint32_t sc[2] = {0, 0};        // steps lane w has been through
-                uint32_t oc[2] = {0, 0};        // columns lane w took part in so far
-                Segment s;
-                for (WorkIter it(p, cta); it.next(s);) {
-                    const int n_steps = s.kt1 - s.kt0;
-                    for (int w = 0; w < s.n_sub; ++w)
-                        if (!wait(kQFull + w, oc[w], 0)) return;
-                    if (!wait(kKvFull + n % C::kStages, n / C::kStages, (int)n)) return;
-                    tc_fence_after_sync();
-                    for (int w = 0; w < s.n_sub; ++w) {
-                        issue_qk(w, n % C::kStages);
-                        tc_commit(bar(kSFull + w));
+                auto issue_pv = [&](uint32_t stage, bool first) {
+                    const uint32_t v_lo = v_lo0 + stage * (C::kTileBytes >> 4);
+                    if (elected) {
+#pragma unroll
+                        for (int kk = 0; kk < kKeyTile / 16; ++kk)
+                            mma_ts(t_ow, t_sw + 8 * kk, smem_desc_join(v_lo + ((kk * 2048) >> 4), hi), idesc_pv,
+                                   (!first || kk > 0) ? 1u : 0u);
                     }
-                    tc_commit(bar(kKvEmpty + n % C::kStages));
-                    ++n;
-                    if (n_steps == 1) tc_commit(bar(kQEmpty));
-                    for (int j = 0; j < n_steps; ++j) {
-                        const bool more = j + 1 < n_steps;
-                        const int sv = n % C::kStages, sk = (n + 1) % C::kStages;
-                        if (!wait(kKvFull + sv, n / C::kStages, (int)n)) return;
-                        if (more && !wait(kKvFull + sk, (n + 1) / C::kStages, (int)n + 1)) return;
-                        for (int w = 0; w < s.n_sub; ++w) {
-                            if (!wait(kPFull + w, sc[w], (int)sc[w])) return;
-                            ++sc[w];
-                            // the previous column's O rows must have been read out
-                            if (j == 0 && oc[w] > 0 && !wait(kOEmpty + w, oc[w] - 1, (int)oc[w])) return;
-                            tc_fence_after_sync();
-                            issue_pv(w, sv, j == 0);
-                            if (more) {
-                                issue_qk(w, sk);
-                                tc_commit(bar(kSFull + w));
-                            } else {
-                                tc_commit(bar(kOFull + w));
+                    __syncwarp();
+                };
+                auto commit = [&](int bar_id) { if (elected) tc_commit(bar(bar_id)); };
+                auto arrive = [&](int bar_id) { if (elected) mbar_arrive(bar(bar_id)); };
+                uint32_t stage = 0, phase = 0;  // ring position of the next K/V tile and its use count parity
+                auto advance = [&]() { if (++stage == (uint32_t)C::kStages) { stage = 0; phase ^= 1u; } };
+                // The two lanes' product groups (PV of one step and QK of the next) alternate on
+                // the tensor pipe, lane 0 first: while one lane's group runs, the other lane's
+                // softmax warps work.  Left to themselves the lanes drift into step with each
+                // other and the pipe idles during both softmaxes.
+                uint32_t bc = 0;                // groups this lane has issued (or passed on)
+                auto take_turn = [&]() -> bool {
+                    if (w == 0) return bc == 0 || wait(kTurn + 0, bc - 1, (int)bc);
+                    return wait(kTurn + 1, bc, (int)bc);
+                };
+                auto pass_turn = [&]() { arrive(kTurn + (w ^ 1)); ++bc; };
+                uint32_t n = 0;                 // K/V tiles consumed so far (for the status record only)
+                uint32_t sc = 0;                // steps this lane has been through
+                uint32_t oc = 0;                // columns this lane took part in so far
+                uint32_t seg = 0;
+                Segment s;
+                for (WorkIter it(p, cta); it.next(s); ++seg) {
+                    const int n_steps = s.kt1 - s.kt0;
+                    if (w >= s.n_sub) {
+                        // not this lane's column: pass every stage on once its tile has landed, and
+                        // the Q buffers once the previous column's release is complete
+                        for (int t = 0; t < 2 * n_steps; ++t, ++n) {
+                            if (!wait(kKvFull + stage, phase, (int)n)) return;
+                            arrive(kKvEmpty + stage);
+                            advance();
+                            if (t & 1) {
+                                // and the turn, as if this lane had issued the step's products
+                                if (!take_turn()) return;
+                                pass_turn();
                             }
                         }
-                        tc_commit(bar(kKvEmpty + sv));
+                        if (seg > 0 && !wait(kQEmpty, seg - 1, (int)seg)) return;
+                        arrive(kQEmpty);
+                        continue;
+                    }
+                    if (!wait(kQFull + w, oc, 0)) return;
+                    if (!wait(kKvFull + stage, phase, (int)n)) return;
+                    tc_fence_after_sync();
+                    issue_qk(stage);
+                    commit(kSFull + w);
+                    commit(kKvEmpty + stage);
+                    advance();
+                    ++n;
+                    if (n_steps == 1) commit(kQEmpty);
+                    for (int j = 0; j < n_steps; ++j, ++sc) {
+                        const bool more = j + 1 < n_steps;
+                        const uint32_t sv = stage, pv = phase;
+                        advance();
+                        const uint32_t sk = stage, pk = phase;
+                        if (!wait(kKvFull + sv, pv, (int)n)) return;
+                        if (more && !wait(kKvFull + sk, pk, (int)n + 1)) return;
+                        if (!take_turn()) return;
+                        // the previous column's O rows must have been read out
+                        if (j == 0 && oc > 0 && !wait(kOEmpty + w, oc - 1, (int)oc)) return;
+                        if (!wait(kPFull + w, sc, (int)sc)) return;
+                        tc_fence_after_sync();
+                        issue_pv(sv, j == 0);
+                        commit(kKvEmpty + sv);
+                        if (more) issue_qk(sk);
+                        pass_turn();
                         ++n;
                         if (more) {
-                            tc_commit(bar(kKvEmpty + sk));
+                            commit(kSFull + w);
+                            commit(kKvEmpty + sk);
+                            advance();
                             ++n;
+                        } else {
+                            commit(kOFull + w);
                         }
-                        if (j + 2 == n_steps) tc_commit(bar(kQEmpty));   // the column's last QK is in the pipe
+                        if (j + 2 == n_steps) commit(kQEmpty);   // the column's last QK is in the pipe
                     }
-                    for (int w = 0; w < s.n_sub; ++w) ++oc[w];
+                    ++oc;
                 }
             }();
         }
@@ -429,85 +480,119 @@ attn_sm100_kernel(const __grid_constant__ AttnParams p, const __grid_constant__ 
                     if (!__all_sync(0xffffffffu, wait(kSFull + w, sc, j))) return;
                     tc_fence_after_sync();
                     const int nvalid = kit.valid();
-                    // ---- pass 1: row maxima of the tile: 32 columns per thread, then across the
-                    //      quad (the values are fetched again below) ----
-                    float ta = -INFINITY, tb = -INFINITY;
-                    uint32_t va[32];
+                    // The tile is taken in two 64-key pieces.  A piece's exponentials are computed
+                    // against the rows' current reference maxima straight away; its sums then tell
+                    // whether that was safe (no weight can exceed the sum).  Only when some sum in
+                    // the warp is large or not finite - always on a column's first piece, where the
+                    // references are -inf - are the exact row maxima taken, the references moved,
+                    // what has been accumulated rescaled, and the piece redone.
 #pragma unroll
                     for (int piece = 0; piece < 2; ++piece) {
-                        tmem_ld_16x256b_x8(t_s + 64 * piece, va);
+                        uint32_t v[32];
+                        tmem_ld_16x256b_x8(t_s + 64 * piece, v);
                         tmem_wait_ld();
-                        if (nvalid < kKeyTile) mask_piece(va, 64 * piece, cq, nvalid);
+                        if (nvalid < kKeyTile) mask_piece(v, 64 * piece, cq, nvalid);
+                        uint32_t pk[16];
+                        uint64_t ts_a = 0ull, ts_b = 0ull;         // the piece's sums, two partials per row
+                        {
+                            const uint64_t na2 = pack2(-m_a, -m_a), nb2 = pack2(-m_b, -m_b);
 #pragma unroll
-                        for (int k = 0; k < 8; ++k) {
-                            ta = max3(ta, as_f(va[4 * k]), as_f(va[4 * k + 1]));
-                            tb = max3(tb, as_f(va[4 * k + 2]), as_f(va[4 * k + 3]));
+                            for (int k = 0; k < 8; ++k) {
+                                const uint64_t xa = fma2(pack2(as_f(v[4 * k]), as_f(v[4 * k + 1])), c2, na2);
+                                const uint64_t xb = fma2(pack2(as_f(v[4 * k + 2]), as_f(v[4 * k + 3])), c2, nb2);
+                                uint64_t pa, pb;
+                                if ((kPolyMask >> (8 * piece + k)) & 1u) {
+                                    pa = exp2_poly2(xa);
+                                    pb = exp2_poly2(xb);
+                                } else {
+                                    pa = exp2_sfu2(xa);
+                                    pb = exp2_sfu2(xb);
+                                }
+                                ts_a = add2(ts_a, pa);
+                                ts_b = add2(ts_b, pb);
+                                float a0, a1, b0, b1;
+                                unpack2(pa, a0, a1);
+                                unpack2(pb, b0, b1);
+                                pk[2 * k] = cvt_bf16x2(a0, a1);        // key 8k + cq in the low half
+                                pk[2 * k + 1] = cvt_bf16x2(b0, b1);
+                            }
                         }
-                    }
-                    tmem_ld_16x256b_x8(t_s, va);               // first piece of pass 2, in flight during the shuffles
-                    ta = fmaxf(ta, __shfl_xor_sync(0xffffffffu, ta, 1));
-                    tb = fmaxf(tb, __shfl_xor_sync(0xffffffffu, tb, 1));
-                    ta = fmaxf(ta, __shfl_xor_sync(0xffffffffu, ta, 2)) * c;
-                    tb = fmaxf(tb, __shfl_xor_sync(0xffffffffu, tb, 2)) * c;
-                    if (j == s.kt0) {
-                        m_a = ta;
-                        m_b = tb;
-                    } else {
-                        const bool grow_a = ta > m_a + kRescaleThreshold, grow_b = tb > m_b + kRescaleThreshold;
-                        if (__any_sync(0xffffffffu, grow_a || grow_b)) {
-                            // rescale the running sums and the O rows; PV of tile j-1 has completed
-                            // (the commit that released S_j covers it) and PV of tile j is not issued yet
-                            const float al_a = grow_a ? ex2(m_a - ta) : 1.f, al_b = grow_b ? ex2(m_b - tb) : 1.f;
-                            if (grow_a) m_a = ta;
-                            if (grow_b) m_b = tb;
+                        float sa, sb;
+                        {
+                            float x0, x1;
+                            unpack2(ts_a, x0, x1);
+                            sa = x0 + x1;
+                            unpack2(ts_b, x0, x1);
+                            sb = x0 + x1;
+                        }
+                        if (__any_sync(0xffffffffu, !(sa <= kSafeSum) || !(sb <= kSafeSum))) {
+                            // exact maxima of the piece's rows: 16 columns per thread, then across the quad
+                            float ta = fmaxf(as_f(v[0]), as_f(v[1])), tb = fmaxf(as_f(v[2]), as_f(v[3]));
+#pragma unroll
+                            for (int k = 1; k < 8; ++k) {
+                                ta = max3(ta, as_f(v[4 * k]), as_f(v[4 * k + 1]));
+                                tb = max3(tb, as_f(v[4 * k + 2]), as_f(v[4 * k + 3]));
+                            }
+                            ta = fmaxf(ta, __shfl_xor_sync(0xffffffffu, ta, 1));
+                            tb = fmaxf(tb, __shfl_xor_sync(0xffffffffu, tb, 1));
+                            ta = fmaxf(ta, __shfl_xor_sync(0xffffffffu, ta, 2)) * c;
+                            tb = fmaxf(tb, __shfl_xor_sync(0xffffffffu, tb, 2)) * c;
+                            const bool fresh = j == s.kt0 && piece == 0;     // nothing accumulated yet
+                            const float new_a = fresh ? ta : fmaxf(m_a, ta), new_b = fresh ? tb : fmaxf(m_b, tb);
+                            const float al_a = fresh ? 0.f : ex2(m_a - new_a), al_b = fresh ? 0.f : ex2(m_b - new_b);
+                            m_a = new_a;
+                            m_b = new_b;
                             acc_a = fma2(acc_a, pack2(al_a, al_a), 0ull);
                             acc_b = fma2(acc_b, pack2(al_b, al_b), 0ull);
-                            tmem_wait_ld();
+                            if (j != s.kt0) {
+                                // the O rows; PV of tile j-1 has completed (the commit that released S_j
+                                // covers it) and PV of tile j is not issued yet
 #pragma unroll 1
-                            for (int ch = 0; ch < C::kOChunks; ++ch) {
-                                uint32_t o[32];
-                                tmem_ld_16x256b_x8(t_o + 64 * ch, o);
+                                for (int ch = 0; ch < C::kOChunks; ++ch) {
+                                    uint32_t o[32];
+                                    tmem_ld_16x256b_x8(t_o + 64 * ch, o);
+                                    tmem_wait_ld();
+#pragma unroll
+                                    for (int k = 0; k < 8; ++k) {
+                                        o[4 * k] = as_u(as_f(o[4 * k]) * al_a);
+                                        o[4 * k + 1] = as_u(as_f(o[4 * k + 1]) * al_a);
+                                        o[4 * k + 2] = as_u(as_f(o[4 * k + 2]) * al_b);
+                                        o[4 * k + 3] = as_u(as_f(o[4 * k + 3]) * al_b);
+                                    }
+                                    tmem_st_16x256b_x8(t_o + 64 * ch, o);
+                                }
+                            }
+                            if (piece == 1) {
+                                // the first piece's P, already in TMEM but not yet handed over
+                                uint32_t p0[16];
+                                tmem_ld_16x128b_x8(t_s, p0);
                                 tmem_wait_ld();
 #pragma unroll
                                 for (int k = 0; k < 8; ++k) {
-                                    o[4 * k] = as_u(as_f(o[4 * k]) * al_a);
-                                    o[4 * k + 1] = as_u(as_f(o[4 * k + 1]) * al_a);
-                                    o[4 * k + 2] = as_u(as_f(o[4 * k + 2]) * al_b);
-                                    o[4 * k + 3] = as_u(as_f(o[4 * k + 3]) * al_b);
+                                    p0[2 * k] = cvt_bf16x2(as_f(p0[2 * k] << 16) * al_a, as_f(p0[2 * k] & 0xffff0000u) * al_a);
+                                    p0[2 * k + 1] = cvt_bf16x2(as_f(p0[2 * k + 1] << 16) * al_b, as_f(p0[2 * k + 1] & 0xffff0000u) * al_b);
                                 }
-                                tmem_st_16x256b_x8(t_o + 64 * ch, o);
+                                tmem_st_16x128b_x8(t_s, p0);
+                            }
+                            // the piece again, against the new references
+                            const uint64_t na2 = pack2(-m_a, -m_a), nb2 = pack2(-m_b, -m_b);
+                            ts_a = ts_b = 0ull;
+#pragma unroll
+                            for (int k = 0; k < 8; ++k) {
+                                const uint64_t pa = exp2_sfu2(fma2(pack2(as_f(v[4 * k]), as_f(v[4 * k + 1])), c2, na2));
+                                const uint64_t pb = exp2_sfu2(fma2(pack2(as_f(v[4 * k + 2]), as_f(v[4 * k + 3])), c2, nb2));
+                                ts_a = add2(ts_a, pa);
+                                ts_b = add2(ts_b, pb);
+                                float a0, a1, b0, b1;
+                                unpack2(pa, a0, a1);
+                                unpack2(pb, b0, b1);
+                                pk[2 * k] = cvt_bf16x2(a0, a1);
+                                pk[2 * k + 1] = cvt_bf16x2(b0, b1);
                             }
                         }
-                    }
-                    // ---- pass 2: p = 2^(s*c - m) in two 64-key pieces; each piece's P (bf16, 32
-                    //      packed columns) lands on S columns this warp no longer needs ----
-                    const uint64_t na2 = pack2(-m_a, -m_a), nb2 = pack2(-m_b, -m_b);
-#pragma unroll
-                    for (int piece = 0; piece < 2; ++piece) {
-                        tmem_wait_ld();
-                        if (nvalid < kKeyTile) mask_piece(va, 64 * piece, cq, nvalid);
-                        uint32_t pk[16];
-#pragma unroll
-                        for (int k = 0; k < 8; ++k) {
-                            const uint64_t xa = fma2(pack2(as_f(va[4 * k]), as_f(va[4 * k + 1])), c2, na2);
-                            const uint64_t xb = fma2(pack2(as_f(va[4 * k + 2]), as_f(va[4 * k + 3])), c2, nb2);
-                            uint64_t pa, pb;
-                            if ((kPolyMask >> (8 * piece + k)) & 1u) {
-                                pa = exp2_poly2(xa);
-                                pb = exp2_poly2(xb);
-                            } else {
-                                pa = exp2_sfu2(xa);
-                                pb = exp2_sfu2(xb);
-                            }
-                            acc_a = add2(acc_a, pa);
-                            acc_b = add2(acc_b, pb);
-                            float a0, a1, b0, b1;
-                            unpack2(pa, a0, a1);
-                            unpack2(pb, b0, b1);
-                            pk[2 * k] = cvt_bf16x2(a0, a1);            // key 8k + cq in the low half
-                            pk[2 * k + 1] = cvt_bf16x2(b0, b1);
-                        }
-                        if (piece == 0) tmem_ld_16x256b_x8(t_s + 64, va);   // S columns 64..127
+                        acc_a = add2(acc_a, ts_a);
+                        acc_b = add2(acc_b, ts_b);
+                        // P (bf16, 32 packed columns) lands on S columns this warp has already read
                         tmem_st_16x128b_x8(t_s + 32 * piece, pk);
                     }
                     tmem_wait_st();

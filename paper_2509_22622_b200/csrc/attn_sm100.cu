@@ -2,10 +2,13 @@
 //
 // Work decomposition.  A *column* is up to 256 query rows of one head (two
 // 128-row MMA tiles, "lanes" 0 and 1) and a *step* is one 128-key tile of that
-// column's visible cache rows.  All steps of all columns are laid end to end and
-// cut into equal shares, one per persistent CTA (one CTA per SM), so every SM
-// gets the same number of steps whatever the number of columns.  A column whose
-// steps fall into several CTAs is finished by whichever of them arrives last:
+// column's visible cache rows.  One persistent CTA runs per SM.  As long as there
+// is a column for every CTA, columns are handed out whole: the CTAs of a head
+// then walk the keys in step and each K/V tile is fetched from HBM once and
+// shared through L2.  The steps of the columns left over are laid end to end and
+// cut into equal shares, so every SM does the same amount of work whatever the
+// number of columns.  A column whose steps fall into several CTAs is finished by
+// whichever of them arrives last:
 // every part leaves its unnormalised O rows, reference maxima and sums in a
 // scratch slot, bumps the column's arrival counter, and the last one merges the
 // parts and writes the output.  Nothing waits on another CTA.
@@ -116,44 +119,64 @@ struct Segment {
     int q0;                 // first query row of the column
     int rows_valid;         // live rows of the 256
     int n_sub;              // live 128-row tiles
-    long long col_begin;    // global index of the column's first step
+    long long col_begin;    // shared-step index of the column's first step (split columns only)
 };
 
-// First global step of CTA `cta`'s share (the next CTA's is one past its last).
+// First shared step of CTA `cta`'s share (the next CTA's is one past its last).
 __device__ __forceinline__ long long share_begin(const AttnParams &p, int cta)
 {
     return p.total_steps * cta / p.n_ctas;
 }
 
-// The CTA whose share holds global step u.
+// The CTA whose share holds shared step u.
 __device__ __forceinline__ int cta_of_step(const AttnParams &p, long long u)
 {
     return (int)(((u + 1) * p.n_ctas - 1) / p.total_steps);
 }
 
+// A CTA's work in order: its whole columns, group by group and wave by wave, then its
+// share of the steps that are left.  Every role of the CTA walks the same sequence.
 struct WorkIter {
     const AttnParams &p;
+    int cta, g, wave;
     long long u, end;
-    __device__ WorkIter(const AttnParams &prm, int cta)
-        : p(prm), u(share_begin(prm, cta)), end(share_begin(prm, cta + 1)) {}
-    __device__ bool next(Segment &s)
+    __device__ WorkIter(const AttnParams &prm, int cta_)
+        : p(prm), cta(cta_), g(0), wave(0), u(share_begin(prm, cta_)), end(share_begin(prm, cta_ + 1)) {}
+    __device__ void fill(Segment &s, int grp, int col, int kt0, int kt1) const
     {
-        if (u >= end) return false;
-        int g = 0;
-        while (g + 1 < p.n_groups && u >= p.g[g + 1].step_begin) ++g;
-        const AttnGroup &G = p.g[g];
-        const long long off = u - G.step_begin;
-        const int col = (int)(off / G.n_kt);
-        s.g = g;
+        const AttnGroup &G = p.g[grp];
+        s.g = grp;
         s.head = col / G.tiles;
         s.tile = col - s.head * G.tiles;
-        s.kt0 = (int)(off - (long long)col * G.n_kt);
-        s.kt1 = (int)min((long long)G.n_kt, s.kt0 + (end - u));
+        s.kt0 = kt0;
+        s.kt1 = kt1;
         s.q0 = G.q_begin + s.tile * kQTileRows;
         s.rows_valid = min(kQTileRows, G.q_rows - s.tile * kQTileRows);
         s.n_sub = s.rows_valid > 128 ? 2 : 1;
-        s.col_begin = u - s.kt0;
-        u += s.kt1 - s.kt0;
+    }
+    __device__ bool next(Segment &s)
+    {
+        while (g < p.n_groups) {
+            if ((wave + 1) * p.n_ctas <= p.g[g].wave_cols) {
+                fill(s, g, wave * p.n_ctas + cta, 0, p.g[g].n_kt);
+                s.col_begin = 0;
+                ++wave;
+                return true;
+            }
+            ++g;
+            wave = 0;
+        }
+        if (u >= end) return false;
+        int gg = 0;
+        while (gg + 1 < p.n_groups && u >= p.g[gg + 1].step_begin) ++gg;
+        const AttnGroup &G = p.g[gg];
+        const long long off = u - G.step_begin;
+        const int col = (int)(off / G.n_kt);
+        const int kt0 = (int)(off - (long long)col * G.n_kt);
+        const int kt1 = (int)min((long long)G.n_kt, kt0 + (end - u));
+        fill(s, gg, G.wave_cols + col, kt0, kt1);
+        s.col_begin = u - kt0;
+        u += kt1 - kt0;
         return true;
     }
 };

@@ -188,7 +188,13 @@ int build_attn_params(ll_cache *c, int layer, const ll_bf16 *q, ll_bf16 *out, fl
     p->partial = reinterpret_cast<float *>(c->storage ? c->storage + c->off_partial : nullptr);
     p->counters = reinterpret_cast<uint32_t *>(c->storage ? c->storage + c->off_counters : nullptr);
     const int rows_per_group = c->C * c->P;
-    long long steps = 0;
+    // One persistent CTA per SM.  While a group still has a CTA's worth of columns they go
+    // out whole, one per CTA and wave (CTAs on the same head then walk the keys in step and
+    // share each K/V tile through L2); what is left over is cut into equal shares of steps.
+    const int sms = std::min(c->sm_count > 0 ? c->sm_count : 148, ll::kMaxCtas);
+    const long long cols_per_group = (long long)c->H * ((rows_per_group + ll::kQTileRows - 1) / ll::kQTileRows);
+    const bool waves = cols_per_group >= sms;
+    long long steps = 0, all_steps = 0;
     for (int g = 0; g < n_groups; ++g) {
         ll::AttnGroup &G = p->g[g];
         G.q_begin = g * rows_per_group;
@@ -205,14 +211,14 @@ int build_attn_params(ll_cache *c, int layer, const ll_bf16 *q, ll_bf16 *out, fl
             G.k_len[r] = (int)lens[r];
             G.n_kt += (int)((lens[r] + ll::kKeyTile - 1) / ll::kKeyTile);
         }
+        G.wave_cols = waves ? (int)(cols_per_group / sms * sms) : 0;
         G.step_begin = steps;
-        steps += (long long)c->H * G.tiles * G.n_kt;
+        steps += (cols_per_group - G.wave_cols) * G.n_kt;
+        all_steps += cols_per_group * G.n_kt;
     }
     p->nq_total = n_groups * rows_per_group;
     p->total_steps = steps;
-    // one persistent CTA per SM, each taking an equal share of the steps
-    const int sms = c->sm_count > 0 ? c->sm_count : 148;
-    p->n_ctas = (int)std::min<long long>(std::min(sms, ll::kMaxCtas), steps);
+    p->n_ctas = waves ? sms : (int)std::min<long long>(sms, all_steps);
     return LL_OK;
 }
 

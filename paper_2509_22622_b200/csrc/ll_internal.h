@@ -34,15 +34,19 @@ struct LayerState {
 };
 
 // One group of query rows that share a visible key set.  The group's work is
-// heads x tiles columns (a column = kQTileRows query rows of one head), each
-// n_kt steps long (a step = one kKeyTile-key tile); columns are numbered
-// head-major and their steps laid end to end after those of earlier groups.
+// heads x tiles columns (a column = kQTileRows query rows of one head, numbered
+// head-major), each n_kt steps long (a step = one kKeyTile-key tile).  The first
+// wave_cols columns (a multiple of the CTA count) are handed out whole, CTA i
+// taking columns i, i + n_ctas, ...; the steps of the remaining columns are
+// laid end to end after those of earlier groups' remainders and cut into equal
+// shares.
 struct AttnGroup {
     int q_begin;                      // first query row of the group in the q tensor
     int q_rows;                       // rows in the group
     int tiles;                        // query tiles of kQTileRows rows
     int n_kt;                         // key tiles (steps) per column
-    long long step_begin;             // steps of all earlier groups
+    int wave_cols;                    // columns handed out whole
+    long long step_begin;             // shared steps of all earlier groups
     int n_ranges;
     int k_start[LL_MAX_RANGES];       // visible cache-row runs
     int k_len[LL_MAX_RANGES];
@@ -56,8 +60,8 @@ struct AttnParams {
     int n_groups;
     int heads;
     int nq_total;                     // rows of q / out
-    int n_ctas;                       // grid.x: persistent CTAs sharing total_steps evenly
-    long long total_steps;            // steps of all groups
+    int n_ctas;                       // grid.x: persistent CTAs
+    long long total_steps;            // shared steps of all groups (cut evenly across the CTAs)
     int64_t rows_per_head;            // (S+W)*P
     float scale_log2;                 // log2(e) / sqrt(D)
     const ll_bf16 *q;                 // [nq_total, H, D]

@@ -16,25 +16,26 @@
 // Inside a CTA (640 threads):
 //   warp 16 (one lane)  TMA producer: the column's Q tiles, then K_j V_j K_j+1 ...
 //                       into a ring of 128-byte-swizzled shared-memory stages
-//   warps 17, 18        MMA issuers of lane 0 and lane 1 (one thread each):
-//                       S_w = Q_w K_j^T (operands in shared memory, accumulator in
-//                       TMEM), O_w += P_w V_j (P read from TMEM)
+//   warps 17, 18        MMA issuers of lane 0 and lane 1 (one elected thread each):
+//                       S_w = Q_w K_j^T and O_w += P_w V_j, all operands in shared
+//                       memory, accumulators in TMEM
 //   warps 0-15          softmax: warp (w, q, h) owns the 16 rows 32q + 16h .. of
 //                       lane w; its threads read S with the 16x256b TMEM shape, so
-//                       a row lives in the four threads of a quad and the row
-//                       maximum and sum are two shuffles away.  P (bf16) is
-//                       written back over S.  The rows' reference maxima move, and
-//                       O is rescaled in TMEM, only when a weight computed against
-//                       the old reference would have been large.
-//   While the softmax warps of one lane work, the tensor pipe runs the other
-//   lane's MMAs.  A share of the exponentials is evaluated with a cubic on the
-//   FMA pipe instead of the special-function unit, which both lanes would
-//   otherwise keep saturated.
+//                       a row lives in the four threads of a quad.  P (bf16) goes to
+//                       a swizzled shared-memory tile, 64 keys at a time.  The rows'
+//                       reference maxima move, and O is rescaled in TMEM, only when
+//                       a weight computed against the old reference would have been
+//                       large.
+//   P does not go back over S: a lane's S buffer is free as soon as its softmax
+//   warps hold the tile in registers, so the MMA warp issues QK of step j+1 while
+//   the softmax of step j is still running, and the softmax warps find the next S
+//   waiting.  The tensor pipe then sees, per lane and step, PV(first half), QK(next),
+//   PV(second half), whenever their inputs arrive.  A share of the exponentials is
+//   evaluated with a cubic on the FMA pipe instead of the special-function unit.
 //
-// TMEM columns: S_0 | S_1 | O_0 | O_1 (fp32); P_w aliases the first half of S_w.
-// The visible keys are a short list of contiguous cache-row runs (sink, ring,
-// wrapped ring); softmax does not care about key order, so the only masking is
-// the ragged last tile of each run.
+// TMEM columns: S_0 | S_1 | O_0 | O_1 (fp32).  The visible keys are a short list of
+// contiguous cache-row runs (sink, ring, wrapped ring); softmax does not care about
+// key order, so the only masking is the ragged last tile of each run.
 //
 // Every mbarrier wait is bounded: a role that waits longer than kWaitLimitNs
 // records a status word, raises the CTA's abort flag, and all roles drain to the
@@ -76,8 +77,9 @@ struct Cfg {
     static constexpr int kAtoms = D / 64;                   // 128-byte swizzle atoms per row
     static constexpr int kAtomBytes = 128 * 128;            // 128 rows x 128 bytes
     static constexpr int kTileBytes = kAtoms * kAtomBytes;  // one 128-row tile of Q, K or V
-    static constexpr int kStages = (D == 128) ? 5 : 8;
-    static constexpr int kSmemTiles = (2 + kStages) * kTileBytes;
+    static constexpr int kPBytes = 2 * kAtomBytes;          // one lane's P: 128 rows x 128 keys
+    static constexpr int kStages = (D == 128) ? 3 : 8;
+    static constexpr int kSmemTiles = 2 * kTileBytes + 2 * kPBytes + kStages * kTileBytes;
     static constexpr int kSmemBytes = kSmemTiles + 1024 /*barriers*/ + 1024 /*alignment slack*/;
     static constexpr int kTmemCols = 512;
     static constexpr int kColS = 0;                         // S_w at kColS + 128 w
@@ -87,8 +89,8 @@ struct Cfg {
 
 // barrier indices inside the shared barrier array (+ lane or + stage)
 enum Bar {
-    kQFull = 0, kQEmpty = 2, kSFull = 4, kPFull = 6, kOFull = 8, kOEmpty = 10,
-    kKvFull = 12, kKvEmpty = 20, kTurn = 28, kNumBars = 30
+    kQFull = 0, kQEmpty = 2, kSFull = 4, kSEmpty = 6, kPFull = 8, kPEmpty = 10, kOFull = 12, kOEmpty = 14,
+    kKvFull = 16, kKvEmpty = 24, kNumBars = 32
 };
 
 // Walks the visible key tiles of a group: runs in order, 128 rows at a time.
@@ -275,7 +277,8 @@ attn_sm100_kernel(const __grid_constant__ AttnParams p, const __grid_constant__ 
     const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     uint8_t *smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));
     const uint32_t q_smem = smem_base;                                  // 2 tiles
-    const uint32_t kv_smem = smem_base + 2 * C::kTileBytes;             // kStages tiles
+    const uint32_t p_smem = smem_base + 2 * C::kTileBytes;              // one 64-key P tile per lane
+    const uint32_t kv_smem = p_smem + 2 * C::kPBytes;                   // kStages tiles
     const uint32_t bars = smem_base + C::kSmemTiles;                    // kNumBars x 8 bytes
     uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(smem_gen + C::kSmemTiles + kNumBars * 8);
     volatile int *abort_flag = reinterpret_cast<volatile int *>(tmem_slot + 1);
@@ -291,8 +294,9 @@ attn_sm100_kernel(const __grid_constant__ AttnParams p, const __grid_constant__ 
     if (threadIdx.x == 0) {
         for (int i = 0; i < kNumBars; ++i) {
             uint32_t count = 1;
-            if (i == kPFull || i == kPFull + 1 || i == kOEmpty || i == kOEmpty + 1) count = kSoftmaxWarps / 2;
-            if (i == kQEmpty || (i >= kKvEmpty && i < kTurn)) count = 2;       // both MMA warps release Q and every K/V stage
+            if ((i >= kSEmpty && i < kSEmpty + 2) || (i >= kPFull && i < kPFull + 2) || (i >= kOEmpty && i < kOEmpty + 2))
+                count = kSoftmaxWarps / 2;                                     // one arrival per softmax warp of the lane
+            if (i == kQEmpty || i >= kKvEmpty) count = 2;                      // both MMA warps release Q and every K/V stage
             mbar_init(bar(i), count);
         }
         // an earlier CTA already gave up on a wait: this one does not start (flag value 2)
@@ -330,20 +334,23 @@ attn_sm100_kernel(const __grid_constant__ AttnParams p, const __grid_constant__ 
                 uint32_t seg = 0;
                 Segment s;
                 for (WorkIter it(p, cta); it.next(s); ++seg) {
-                    KeyIter kit(&p.g[s.g], s.kt0);
-                    auto load_kv = [&](const CUtensorMap *m) -> bool {
+                    // Tile order K_0, K_1, V_0, K_2, V_1, ... : the QK of a step is issued a whole
+                    // softmax ahead of the step's PV, so K runs one step ahead of V and three stages
+                    // (the V in use, the K in use, one in flight) keep both fed.
+                    KeyIter kit_k(&p.g[s.g], s.kt0), kit_v(&p.g[s.g], s.kt0);
+                    auto load_kv = [&](const CUtensorMap *m, int row) -> bool {
                         const int stage = n % C::kStages;
                         if (!wait(kKvEmpty + stage, (n / C::kStages) ^ 1u, (int)n)) return false;
                         mbar_arrive_expect_tx(bar(kKvFull + stage), C::kTileBytes);
                         for (int a = 0; a < C::kAtoms; ++a)
                             tma_load_3d(kv_smem + stage * C::kTileBytes + a * C::kAtomBytes, m,
-                                        bar(kKvFull + stage), a * 64, kit.row(), s.head);
+                                        bar(kKvFull + stage), a * 64, row, s.head);
                         ++n;
                         return true;
                     };
                     // the first key tile goes out before Q: it needs no Q buffer and is in
                     // flight while the previous column's last products drain
-                    if (!load_kv(&kmap) || !load_kv(&vmap)) return;
+                    if (!load_kv(&kmap, kit_k.row())) return;
                     if (seg > 0 && !wait(kQEmpty, seg - 1, (int)seg)) return;
                     for (int w = 0; w < s.n_sub; ++w) {
                         mbar_arrive_expect_tx(bar(kQFull + w), C::kTileBytes);
@@ -351,19 +358,22 @@ attn_sm100_kernel(const __grid_constant__ AttnParams p, const __grid_constant__ 
                             tma_load_3d(q_smem + w * C::kTileBytes + a * C::kAtomBytes, &qmap, bar(kQFull + w),
                                         a * 64, s.head, s.q0 + 128 * w);
                     }
-                    for (int j = s.kt0 + 1; j < s.kt1; ++j) {
-                        kit.next();
-                        if (!load_kv(&kmap) || !load_kv(&vmap)) return;
+                    for (int j = s.kt0; j < s.kt1; ++j) {
+                        if (j + 1 < s.kt1) {
+                            kit_k.next();
+                            if (!load_kv(&kmap, kit_k.row())) return;
+                        }
+                        if (!load_kv(&vmap, kit_v.row())) return;
+                        kit_v.next();
                     }
                 }
             }();
         } else if (warp == kMmaWarp || warp == kMmaWarp + 1) {
             // ====================== MMA issuer of lane w = warp - kMmaWarp ======================
-            // One issuing warp per lane: each runs its own waits and bookkeeping while the
-            // tensor pipe works on the other lane's products.  Both walk the same K/V ring and
-            // both release every stage (a lane that sits a column out releases it unused).
-            // All 32 lanes walk the loops and the waits, so that addresses and descriptors are
-            // warp-uniform values; one elected lane issues the MMAs, commits and arrivals.
+            // One issuing warp per lane.  Both walk the same K/V ring and both release every
+            // stage (a lane that sits a column out releases it unused).  All 32 lanes walk the
+            // loops and the waits, so that addresses and descriptors are warp-uniform values;
+            // one elected lane issues the MMAs, commits and arrivals.
             [&]() {
                 const int w = warp - kMmaWarp;
                 const bool elected = elect_one();
@@ -374,8 +384,9 @@ attn_sm100_kernel(const __grid_constant__ AttnParams p, const __grid_constant__ 
                 // S_w = Q_w K^T: both operands K-major, 64-element atoms, 16 elements (32 bytes) per MMA
                 const uint32_t q_lo = smem_desc_lo(q_smem + w * C::kTileBytes, 16);
                 const uint32_t k_lo0 = smem_desc_lo(kv_smem, 16);
-                // O_w += P_w V: P from TMEM (16 keys = 8 packed columns per MMA); V is MN-major:
+                // O_w += P_w V: P K-major (one 64-key atom, 16 keys = 32 bytes per MMA); V is MN-major:
                 // 8-key groups 1024 bytes apart, 64-wide d atoms kAtomBytes apart
+                const uint32_t p_lo = smem_desc_lo(p_smem + w * C::kPBytes, 16);
                 const uint32_t v_lo0 = smem_desc_lo(kv_smem, C::kAtomBytes);
                 auto issue_qk = [&](uint32_t stage) {
                     const uint32_t k_lo = k_lo0 + stage * (C::kTileBytes >> 4);
@@ -393,26 +404,16 @@ attn_sm100_kernel(const __grid_constant__ AttnParams p, const __grid_constant__ 
                     if (elected) {
 #pragma unroll
                         for (int kk = 0; kk < kKeyTile / 16; ++kk)
-                            mma_ts(t_ow, t_sw + 8 * kk, smem_desc_join(v_lo + ((kk * 2048) >> 4), hi), idesc_pv,
-                                   (!first || kk > 0) ? 1u : 0u);
+                            mma_ss(t_ow, smem_desc_join(p_lo + (((kk / 4) * C::kAtomBytes + (kk % 4) * 32) >> 4), hi),
+                                   smem_desc_join(v_lo + ((kk * 2048) >> 4), hi), idesc_pv, (!first || kk > 0) ? 1u : 0u);
                     }
                     __syncwarp();
                 };
                 auto commit = [&](int bar_id) { if (elected) tc_commit(bar(bar_id)); };
                 auto arrive = [&](int bar_id) { if (elected) mbar_arrive(bar(bar_id)); };
-                uint32_t stage = 0, phase = 0;  // ring position of the next K/V tile and its use count parity
-                auto advance = [&]() { if (++stage == (uint32_t)C::kStages) { stage = 0; phase ^= 1u; } };
-                // The two lanes' product groups (PV of one step and QK of the next) alternate on
-                // the tensor pipe, lane 0 first: while one lane's group runs, the other lane's
-                // softmax warps work.  Left to themselves the lanes drift into step with each
-                // other and the pipe idles during both softmaxes.
-                uint32_t bc = 0;                // groups this lane has issued (or passed on)
-                auto take_turn = [&]() -> bool {
-                    if (w == 0) return bc == 0 || wait(kTurn + 0, bc - 1, (int)bc);
-                    return wait(kTurn + 1, bc, (int)bc);
-                };
-                auto pass_turn = [&]() { arrive(kTurn + (w ^ 1)); ++bc; };
-                uint32_t n = 0;                 // K/V tiles consumed so far (for the status record only)
+                // tile n of the producer's sequence K_0, K_1, V_0, K_2, V_1, ... sits in stage n % kStages
+                auto kv_wait = [&](uint32_t n) -> bool { return wait(kKvFull + n % C::kStages, n / C::kStages, (int)n); };
+                uint32_t n0 = 0;                // producer index of the column's first tile
                 uint32_t sc = 0;                // steps this lane has been through
                 uint32_t oc = 0;                // columns this lane took part in so far
                 uint32_t seg = 0;
@@ -422,56 +423,49 @@ attn_sm100_kernel(const __grid_constant__ AttnParams p, const __grid_constant__ 
                     if (w >= s.n_sub) {
                         // not this lane's column: pass every stage on once its tile has landed, and
                         // the Q buffers once the previous column's release is complete
-                        for (int t = 0; t < 2 * n_steps; ++t, ++n) {
-                            if (!wait(kKvFull + stage, phase, (int)n)) return;
-                            arrive(kKvEmpty + stage);
-                            advance();
-                            if (t & 1) {
-                                // and the turn, as if this lane had issued the step's products
-                                if (!take_turn()) return;
-                                pass_turn();
-                            }
+                        for (int t = 0; t < 2 * n_steps; ++t) {
+                            if (!kv_wait(n0 + t)) return;
+                            arrive(kKvEmpty + (n0 + t) % C::kStages);
                         }
+                        n0 += 2 * n_steps;
                         if (seg > 0 && !wait(kQEmpty, seg - 1, (int)seg)) return;
                         arrive(kQEmpty);
                         continue;
                     }
                     if (!wait(kQFull + w, oc, 0)) return;
-                    if (!wait(kKvFull + stage, phase, (int)n)) return;
+                    // QK of the column's first step: its S buffer was read out by the last softmax
+                    if (!kv_wait(n0)) return;
+                    if (sc > 0 && !wait(kSEmpty + w, sc - 1, (int)sc)) return;
                     tc_fence_after_sync();
-                    issue_qk(stage);
+                    issue_qk(n0 % C::kStages);
                     commit(kSFull + w);
-                    commit(kKvEmpty + stage);
-                    advance();
-                    ++n;
+                    commit(kKvEmpty + n0 % C::kStages);
                     if (n_steps == 1) commit(kQEmpty);
                     for (int j = 0; j < n_steps; ++j, ++sc) {
                         const bool more = j + 1 < n_steps;
-                        const uint32_t sv = stage, pv = phase;
-                        advance();
-                        const uint32_t sk = stage, pk = phase;
-                        if (!wait(kKvFull + sv, pv, (int)n)) return;
-                        if (more && !wait(kKvFull + sk, pk, (int)n + 1)) return;
-                        if (!take_turn()) return;
+                        const uint32_t nk = n0 + 2 * j + 1;                     // K_j+1 (if any)
+                        const uint32_t nv = more ? nk + 1 : nk;                 // V_j
+                        // QK of the next step as soon as the softmax warps hold S_j in registers
+                        if (more) {
+                            if (!kv_wait(nk)) return;
+                            if (!wait(kSEmpty + w, sc, (int)sc)) return;
+                            tc_fence_after_sync();
+                            issue_qk(nk % C::kStages);
+                            commit(kSFull + w);
+                            commit(kKvEmpty + nk % C::kStages);
+                            if (j + 2 == n_steps) commit(kQEmpty);               // the column's last QK is in the pipe
+                        }
+                        if (!kv_wait(nv)) return;
                         // the previous column's O rows must have been read out
                         if (j == 0 && oc > 0 && !wait(kOEmpty + w, oc - 1, (int)oc)) return;
                         if (!wait(kPFull + w, sc, (int)sc)) return;
                         tc_fence_after_sync();
-                        issue_pv(sv, j == 0);
-                        commit(kKvEmpty + sv);
-                        if (more) issue_qk(sk);
-                        pass_turn();
-                        ++n;
-                        if (more) {
-                            commit(kSFull + w);
-                            commit(kKvEmpty + sk);
-                            advance();
-                            ++n;
-                        } else {
-                            commit(kOFull + w);
-                        }
-                        if (j + 2 == n_steps) commit(kQEmpty);   // the column's last QK is in the pipe
+                        issue_pv(nv % C::kStages, j == 0);
+                        commit(kPEmpty + w);
+                        commit(kKvEmpty + nv % C::kStages);
+                        if (!more) commit(kOFull + w);
                     }
+                    n0 += 2 * n_steps;
                     ++oc;
                 }
             }();
@@ -489,6 +483,12 @@ attn_sm100_kernel(const __grid_constant__ AttnParams p, const __grid_constant__ 
             const int row_a = 32 * q + 16 * h + (lane >> 2);   // row of registers 4k+{0,1}; 4k+{2,3} are row_a + 8
             const int cq = 2 * (lane & 3);                     // first of this thread's two columns in each group of 8
             const int slab = w * 8 + q * 2 + h;
+            // P goes to shared memory with stmatrix: of the warp's 16 rows x 64 keys, one call
+            // stores four 8-row x 8-key blocks (a block row = one 16-byte chunk); lane 8m + r gives the
+            // address of row r of the block holding chunk m, which sits at chunk position m ^ r.
+            // Chunks 4..7 are at the same address ^ 64, the second eight rows 1024 bytes on.
+            const uint32_t p_at = p_smem + w * C::kPBytes + (uint32_t)(32 * q + 16 * h + (lane & 7)) * 128 +
+                                  ((uint32_t)((lane >> 3) ^ (lane & 7)) << 4);
             const float c = p.scale_log2;
             const uint64_t c2 = pack2(c, c);
             uint32_t sc = 0, oc = 0;
@@ -509,13 +509,20 @@ attn_sm100_kernel(const __grid_constant__ AttnParams p, const __grid_constant__ 
                     // the warp is large or not finite - always on a column's first piece, where the
                     // references are -inf - are the exact row maxima taken, the references moved,
                     // what has been accumulated rescaled, and the piece redone.
+                    uint32_t pk[32];                               // P of both pieces, handed over together
 #pragma unroll
                     for (int piece = 0; piece < 2; ++piece) {
                         uint32_t v[32];
                         tmem_ld_16x256b_x8(t_s + 64 * piece, v);
                         tmem_wait_ld();
+                        if (piece == 1) {
+                            // the whole tile is in registers now: the S buffer may take the next QK
+                            tc_fence_before_sync();
+                            __syncwarp();
+                            if (lane == 0) mbar_arrive(bar(kSEmpty + w));
+                        }
                         if (nvalid < kKeyTile) mask_piece(v, 64 * piece, cq, nvalid);
-                        uint32_t pk[16];
+                        uint32_t *pp = pk + 16 * piece;
                         uint64_t ts_a = 0ull, ts_b = 0ull;         // the piece's sums, two partials per row
                         {
                             const uint64_t na2 = pack2(-m_a, -m_a), nb2 = pack2(-m_b, -m_b);
@@ -536,8 +543,8 @@ attn_sm100_kernel(const __grid_constant__ AttnParams p, const __grid_constant__ 
                                 float a0, a1, b0, b1;
                                 unpack2(pa, a0, a1);
                                 unpack2(pb, b0, b1);
-                                pk[2 * k] = cvt_bf16x2(a0, a1);        // key 8k + cq in the low half
-                                pk[2 * k + 1] = cvt_bf16x2(b0, b1);
+                                pp[2 * k] = cvt_bf16x2(a0, a1);        // key 8k + cq in the low half
+                                pp[2 * k + 1] = cvt_bf16x2(b0, b1);
                             }
                         }
                         float sa, sb;
@@ -567,9 +574,20 @@ attn_sm100_kernel(const __grid_constant__ AttnParams p, const __grid_constant__ 
                             m_b = new_b;
                             acc_a = fma2(acc_a, pack2(al_a, al_a), 0ull);
                             acc_b = fma2(acc_b, pack2(al_b, al_b), 0ull);
+                            if (piece == 1) {
+                                // the first piece's P, still in registers
+#pragma unroll
+                                for (int k = 0; k < 8; ++k) {
+                                    pk[2 * k] = cvt_bf16x2(as_f(pk[2 * k] << 16) * al_a, as_f(pk[2 * k] & 0xffff0000u) * al_a);
+                                    pk[2 * k + 1] = cvt_bf16x2(as_f(pk[2 * k + 1] << 16) * al_b, as_f(pk[2 * k + 1] & 0xffff0000u) * al_b);
+                                }
+                            }
                             if (j != s.kt0) {
-                                // the O rows; PV of tile j-1 has completed (the commit that released S_j
-                                // covers it) and PV of tile j is not issued yet
+                                // The O rows hold every earlier tile of the column: once the last PV issued
+                                // (the previous step's) has completed they can be rescaled; this step's PV
+                                // waits for this step's P.
+                                if (!__all_sync(0xffffffffu, wait(kPEmpty + w, sc - 1, (int)sc))) return;
+                                tc_fence_after_sync();
 #pragma unroll 1
                                 for (int ch = 0; ch < C::kOChunks; ++ch) {
                                     uint32_t o[32];
@@ -584,18 +602,8 @@ attn_sm100_kernel(const __grid_constant__ AttnParams p, const __grid_constant__ 
                                     }
                                     tmem_st_16x256b_x8(t_o + 64 * ch, o);
                                 }
-                            }
-                            if (piece == 1) {
-                                // the first piece's P, already in TMEM but not yet handed over
-                                uint32_t p0[16];
-                                tmem_ld_16x128b_x8(t_s, p0);
-                                tmem_wait_ld();
-#pragma unroll
-                                for (int k = 0; k < 8; ++k) {
-                                    p0[2 * k] = cvt_bf16x2(as_f(p0[2 * k] << 16) * al_a, as_f(p0[2 * k] & 0xffff0000u) * al_a);
-                                    p0[2 * k + 1] = cvt_bf16x2(as_f(p0[2 * k + 1] << 16) * al_b, as_f(p0[2 * k + 1] & 0xffff0000u) * al_b);
-                                }
-                                tmem_st_16x128b_x8(t_s, p0);
+                                tmem_wait_st();
+                                tc_fence_before_sync();
                             }
                             // the piece again, against the new references
                             const uint64_t na2 = pack2(-m_a, -m_a), nb2 = pack2(-m_b, -m_b);
@@ -609,17 +617,28 @@ attn_sm100_kernel(const __grid_constant__ AttnParams p, const __grid_constant__ 
                                 float a0, a1, b0, b1;
                                 unpack2(pa, a0, a1);
                                 unpack2(pb, b0, b1);
-                                pk[2 * k] = cvt_bf16x2(a0, a1);
-                                pk[2 * k + 1] = cvt_bf16x2(b0, b1);
+                                pp[2 * k] = cvt_bf16x2(a0, a1);
+                                pp[2 * k + 1] = cvt_bf16x2(b0, b1);
                             }
                         }
                         acc_a = add2(acc_a, ts_a);
                         acc_b = add2(acc_b, ts_b);
-                        // P (bf16, 32 packed columns) lands on S columns this warp has already read
-                        tmem_st_16x128b_x8(t_s + 32 * piece, pk);
                     }
-                    tmem_wait_st();
-                    tc_fence_before_sync();
+                    // P (bf16) into the lane's shared-memory tile, once the PV that read the previous
+                    // step's P from it has completed.  The tile is the K-major, 128-byte-swizzled A
+                    // operand of PV: one 64-key atom per piece, row r at r * 128 bytes, its 16-byte
+                    // chunk k (8 keys) at chunk position k ^ (r % 8).
+                    if (sc > 0 && !__all_sync(0xffffffffu, wait(kPEmpty + w, sc - 1, (int)sc))) return;
+#pragma unroll
+                    for (int piece = 0; piece < 2; ++piece) {
+                        const uint32_t *pp = pk + 16 * piece;
+                        const uint32_t at = p_at + piece * C::kAtomBytes;
+                        stmatrix_x4(at, pp[0], pp[2], pp[4], pp[6]);                       // rows a, chunks 0..3
+                        stmatrix_x4(at ^ 64u, pp[8], pp[10], pp[12], pp[14]);               // rows a, chunks 4..7
+                        stmatrix_x4(at + 8 * 128, pp[1], pp[3], pp[5], pp[7]);              // rows a + 8
+                        stmatrix_x4((at ^ 64u) + 8 * 128, pp[9], pp[11], pp[13], pp[15]);
+                    }
+                    fence_proxy_async_smem();                      // the stores above are read by the tensor pipe
                     __syncwarp();
                     if (lane == 0) mbar_arrive(bar(kPFull + w));
                 }

@@ -83,9 +83,13 @@ int ll_cache_create(int layers, int heads, int head_dim, int tokens_per_frame,
 /* Frees the handle (host memory only; bound storage stays the caller's). */
 void ll_cache_destroy(ll_cache *cache);
 
-/* Bytes of device memory the caller must provide: a small aux block (status
- * words, RoPE tables) followed by, per layer, K then V as
- * [heads][(S+W)*tokens_per_frame rows][head_dim] bf16, sink rows first. */
+/* Bytes of device memory the caller must provide: an aux block (status words,
+ * RoPE tables, and the scratch of the attention kernel: arrival counters and
+ * 320 partial-result slots of 256 x (head_dim + 2) floats, 42.6 MB at head_dim
+ * 128) followed by, per layer, K then V as
+ * [heads][(S+W)*tokens_per_frame rows][head_dim] bf16, sink rows first.
+ * The scratch is shared by all layers of the handle: one more reason why calls
+ * on one handle must be ordered. */
 size_t ll_cache_storage_bytes(const ll_cache *cache);
 
 /* Attach caller-owned device memory (`dev`, >= ll_cache_storage_bytes, 1024-byte
@@ -130,7 +134,8 @@ int ll_rope_append_kv(ll_cache *cache, int layer, const ll_bf16 *q, const ll_bf1
  *   lse_out   device, float [heads, n_q_frames*tokens_per_frame], nullable:
  *             natural-log softmax denominators.
  * QK^T and PV run on tcgen05 tensor cores with fp32 accumulation in TMEM; the
- * softmax is fp32. */
+ * softmax is fp32 (weights rounded to bf16 for the PV product, the denominator
+ * summed from the unrounded values).  The result is run-to-run deterministic. */
 int ll_sink_window_attn(ll_cache *cache, int layer, const ll_bf16 *q_roped,
                         int64_t q_frame_start, int n_q_frames, ll_bf16 *out,
                         float *lse_out, ll_stream stream);
@@ -219,6 +224,30 @@ int ll_cache_device_status(ll_cache *cache, ll_stream stream);
 int ll_debug_attn_simt(ll_cache *cache, int layer, const ll_bf16 *q_roped,
                        int64_t q_frame_start, int n_q_frames, ll_bf16 *out,
                        float *lse_out, ll_stream stream);
+
+/* How the attention kernel would divide the work of a call, given the current
+ * state (host-only; for tests and tuning).  recache = 0: ll_sink_window_attn of
+ * the newest chunk; recache = 1: ll_recache of the resident window.  sm_count > 0
+ * overrides the SM count of the storage's device (148 when no storage is bound).
+ * Per query group g: tiles[g] query tiles of 256 rows per head (so heads *
+ * tiles[g] columns), n_kt[g] key tiles (steps) per column, the first
+ * wave_cols[g] columns handed out whole (CTA i takes columns i, i + n_ctas, ...),
+ * the steps of the others laid end to end from step_begin[g] and cut, with all
+ * groups', into n_ctas equal shares: CTA i takes shared steps
+ * [shared_steps * i / n_ctas, shared_steps * (i + 1) / n_ctas). */
+#define LL_MAX_GROUPS 24
+typedef struct ll_attn_plan {
+    int32_t n_ctas;
+    int32_t n_groups;
+    int32_t heads;
+    int32_t reserved;
+    int64_t shared_steps;
+    int32_t tiles[LL_MAX_GROUPS];
+    int32_t n_kt[LL_MAX_GROUPS];
+    int32_t wave_cols[LL_MAX_GROUPS];
+    int64_t step_begin[LL_MAX_GROUPS];
+} ll_attn_plan;
+int ll_debug_attn_plan(ll_cache *cache, int layer, int recache, int sm_count, ll_attn_plan *out);
 
 /* Kernel launches made by this process through the library so far. */
 int64_t ll_launch_count(void);

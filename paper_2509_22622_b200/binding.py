@@ -40,6 +40,23 @@ class ll_state(C.Structure):
     ]
 
 
+LL_MAX_GROUPS = 24
+
+
+class ll_attn_plan(C.Structure):
+    _fields_ = [
+        ("n_ctas", C.c_int32),
+        ("n_groups", C.c_int32),
+        ("heads", C.c_int32),
+        ("reserved", C.c_int32),
+        ("shared_steps", C.c_int64),
+        ("tiles", C.c_int32 * LL_MAX_GROUPS),
+        ("n_kt", C.c_int32 * LL_MAX_GROUPS),
+        ("wave_cols", C.c_int32 * LL_MAX_GROUPS),
+        ("step_begin", C.c_int64 * LL_MAX_GROUPS),
+    ]
+
+
 class LLError(RuntimeError):
     def __init__(self, code: int, message: str):
         super().__init__("llattn error %d: %s" % (code, message))
@@ -72,6 +89,7 @@ SIGNATURES = {
     "ll_cache_device_status": (C.c_int, [C.c_void_p, C.c_void_p]),
     "ll_debug_attn_simt": (C.c_int, [C.c_void_p, C.c_int, C.c_void_p, C.c_int64, C.c_int, C.c_void_p,
                                      C.c_void_p, C.c_void_p]),
+    "ll_debug_attn_plan": (C.c_int, [C.c_void_p, C.c_int, C.c_int, C.c_int, C.POINTER(ll_attn_plan)]),
     "ll_launch_count": (C.c_int64, []),
     "ll_last_error": (C.c_char_p, []),
     "ll_version": (C.c_char_p, []),
@@ -197,6 +215,12 @@ def ll_cache_set_dry_run(h, on: bool):
 
 def ll_cache_device_status(h, stream=None):
     _check(lib().ll_cache_device_status(h, _stream(stream)))
+
+
+def ll_debug_attn_plan(h, layer=0, recache=False, sm_count=0) -> ll_attn_plan:
+    plan = ll_attn_plan()
+    _check(lib().ll_debug_attn_plan(h, layer, int(recache), sm_count, C.byref(plan)))
+    return plan
 
 
 def ll_launch_count() -> int:

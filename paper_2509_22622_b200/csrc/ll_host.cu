@@ -467,6 +467,44 @@ int ll_recache(ll_cache *c, int layer, const ll_bf16 *q, const ll_bf16 *k, const
     return LL_OK;
 }
 
+int ll_debug_attn_plan(ll_cache *c, int layer, int recache, int sm_count, ll_attn_plan *out)
+{
+    if (!layer_ok(c, layer) || !out) return fail(LL_ERR_INVALID_ARG, "bad argument to ll_debug_attn_plan");
+    static_assert(LL_MAX_GROUPS == ll::kMaxGroups, "header and kernel disagree on the group limit");
+    const ll::LayerState &st = c->layers[layer];
+    int n_groups = 1;
+    int64_t gstart[ll::kMaxGroups];
+    int64_t lo_floor = 0;
+    if (recache) {
+        const int64_t r0 = std::max<int64_t>(c->S, st.end - c->W);
+        n_groups = (int)(std::max<int64_t>(0, st.end - r0) / c->C);
+        for (int g = 0; g < n_groups; ++g) gstart[g] = r0 + (int64_t)g * c->C;
+        lo_floor = r0;
+    } else {
+        if (st.end < c->C) return fail(LL_ERR_BAD_POSITION, "no chunk has been appended yet");
+        gstart[0] = st.end - c->C;
+    }
+    memset(out, 0, sizeof *out);
+    if (n_groups == 0) return LL_OK;
+    const int saved = c->sm_count;
+    if (sm_count > 0) c->sm_count = sm_count;
+    ll::AttnParams p;
+    const int s = build_attn_params(c, layer, nullptr, nullptr, nullptr, n_groups, gstart, lo_floor, &p);
+    c->sm_count = saved;
+    if (s != LL_OK) return s;
+    out->n_ctas = p.n_ctas;
+    out->n_groups = p.n_groups;
+    out->heads = p.heads;
+    out->shared_steps = p.total_steps;
+    for (int g = 0; g < p.n_groups; ++g) {
+        out->tiles[g] = p.g[g].tiles;
+        out->n_kt[g] = p.g[g].n_kt;
+        out->wave_cols[g] = p.g[g].wave_cols;
+        out->step_begin[g] = p.g[g].step_begin;
+    }
+    return LL_OK;
+}
+
 int ll_cache_reset(ll_cache *c)
 {
     if (!c) return fail(LL_ERR_INVALID_ARG, "null handle");

@@ -185,6 +185,41 @@ def test_sink_window_attn_outliers(oracle_mod):
     stream_and_check(oracle_mod, wl, B.ll_sink_window_attn, relative=True, faithful=True)
 
 
+def test_sink_window_attn_with_growing_scores(oracle_mod):
+    """Keys whose norm grows with the token index and from chunk to chunk: the row
+    maxima jump by far more than the kernel's safety margin between tiles and
+    between the two halves of a tile, so the references have to be moved (and
+    everything accumulated so far rescaled) at many steps, not only on the first.
+    Same reference and error measure as the outlier test, for the same reason."""
+    wl = dataclasses.replace(MEDIUM, name="medium_growing", seed=15, n_chunks=6)
+    cache = new_cache(wl)
+    orc = oracle_for(oracle_mod, wl, faithful=True)
+    orc_abs = oracle_for(oracle_mod, wl, faithful=True)
+    C, P = wl.chunk_frames, wl.tokens_per_frame
+    nq = C * P
+    for chunk in range(wl.n_chunks):
+        q, k, v = synth.chunk_qkv(wl, chunk)
+        ramp = (1.0 + 2.0 * chunk) * (1.0 + 3.0 * np.arange(nq, dtype=np.float32) / nq)
+        k = synth.f32_to_bf16_bits(synth.bf16_bits_to_f32(k) * ramp[:, None, None])
+        dq, dk, dv = dev(q), dev(k), dev(v)
+        q_out = torch.empty_like(dq)
+        out = torch.full_like(dq, float("nan"))
+        lse = torch.full((wl.heads, nq), float("nan"), device="cuda", dtype=torch.float32)
+        cache.rope_append_kv(0, dq, dk, dv, chunk * C, wl.grid_h, wl.grid_w, wl.rope_theta, q_out)
+        B.ll_sink_window_attn(cache.h, 0, q_out, chunk * C, C, out, lse)
+        cache.check_device()
+        kf, vf = synth.bf16_bits_to_f64(k), synth.bf16_bits_to_f64(v)
+        orc.append(0, kf, vf, chunk * C, wl.grid_h, wl.grid_w, wl.rope_theta)
+        orc_abs.append(0, kf, np.abs(vf), chunk * C, wl.grid_h, wl.grid_w, wl.rope_theta)
+        qr = orc.rope_q(synth.bf16_bits_to_f64(q), chunk * C, wl.grid_h, wl.grid_w, wl.rope_theta)
+        want, want_lse = orc.attn(0, qr, chunk * C)
+        scale = orc_abs.attn(0, qr, chunk * C)[0]
+        check_attn(f64(out), want, scale=scale)
+        got_lse = lse.cpu().numpy().T.astype(np.float64)
+        assert np.abs(got_lse - want_lse).max() <= 2e-2 * max(1.0, np.abs(want_lse).max() / 16)
+    cache.close()
+
+
 def test_sink_window_attn_is_deterministic():
     wl = MEDIUM
     cache = new_cache(wl)

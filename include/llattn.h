@@ -225,6 +225,14 @@ int ll_debug_attn_simt(ll_cache *cache, int layer, const ll_bf16 *q_roped,
                        int64_t q_frame_start, int n_q_frames, ll_bf16 *out,
                        float *lse_out, ll_stream stream);
 
+/* Test-only: exercise the bounded-wait machinery the kernels share.  Enqueues a
+ * one-warp kernel that waits on a barrier nobody completes, gives up after
+ * limit_ms (1..1000), records the time-out in the status words and returns
+ * normally; the next ll_cache_device_status then reports
+ * LL_ERR_DEVICE_TIMEOUT (barrier 99, iteration 7) and clears the record.
+ * Attention launches enqueued while the record stands skip their work. */
+int ll_debug_wait_timeout(ll_cache *cache, int limit_ms, ll_stream stream);
+
 /* How the attention kernel would divide the work of a call, given the current
  * state (host-only; for tests and tuning).  recache = 0: ll_sink_window_attn of
  * the newest chunk; recache = 1: ll_recache of the resident window.  sm_count > 0

@@ -89,6 +89,7 @@ SIGNATURES = {
     "ll_cache_device_status": (C.c_int, [C.c_void_p, C.c_void_p]),
     "ll_debug_attn_simt": (C.c_int, [C.c_void_p, C.c_int, C.c_void_p, C.c_int64, C.c_int, C.c_void_p,
                                      C.c_void_p, C.c_void_p]),
+    "ll_debug_wait_timeout": (C.c_int, [C.c_void_p, C.c_int, C.c_void_p]),
     "ll_debug_attn_plan": (C.c_int, [C.c_void_p, C.c_int, C.c_int, C.c_int, C.POINTER(ll_attn_plan)]),
     "ll_launch_count": (C.c_int64, []),
     "ll_last_error": (C.c_char_p, []),
@@ -215,6 +216,10 @@ def ll_cache_set_dry_run(h, on: bool):
 
 def ll_cache_device_status(h, stream=None):
     _check(lib().ll_cache_device_status(h, _stream(stream)))
+
+
+def ll_debug_wait_timeout(h, limit_ms=20, stream=None):
+    _check(lib().ll_debug_wait_timeout(h, limit_ms, _stream(stream)))
 
 
 def ll_debug_attn_plan(h, layer=0, recache=False, sm_count=0) -> ll_attn_plan:

@@ -42,6 +42,7 @@
 // common exit where TMEM is released.
 #include <cuda_bf16.h>
 
+#include "bounded_wait.cuh"
 #include "ll_internal.h"
 #include "ptx.cuh"
 
@@ -55,7 +56,6 @@ constexpr int kThreads = 640;
 constexpr int kSoftmaxWarps = 16;
 constexpr int kTmaWarp = 16;
 constexpr int kMmaWarp = 17;
-constexpr uint64_t kWaitLimitNs = 2000000000ull;    // 2 s
 // a piece's 16 weights per thread and row were safe to compute if they sum to at most this
 constexpr float kSafeSum = 256.f;
 // Register reallocation draws on what the CTA was launched with: 640 threads x 96
@@ -182,42 +182,6 @@ struct WorkIter {
         return true;
     }
 };
-
-struct WaitCtx {
-    volatile int *abort_flag;
-    uint32_t *status;
-    int role;
-};
-
-// Bounded wait on an mbarrier phase.  Returns false when the CTA is aborting.
-__device__ __forceinline__ bool wait_slow(uint32_t bar, uint32_t parity, const WaitCtx &ctx, int bar_id, int iter)
-{
-    const uint64_t t0 = globaltimer_ns();
-    uint32_t spins = 0;
-    while (true) {
-        if (mbar_try_wait(bar, parity)) return true;
-        if ((++spins & 63u) == 0) {
-            if (*ctx.abort_flag) return false;
-            if (globaltimer_ns() - t0 > kWaitLimitNs) {
-                *ctx.abort_flag = 1;
-                if (atomicCAS(ctx.status, 0u, (uint32_t)kStatusTimeout) == 0u) {
-                    ctx.status[1] = (uint32_t)ctx.role;
-                    ctx.status[2] = (uint32_t)bar_id;
-                    ctx.status[3] = (uint32_t)iter;
-                    ctx.status[4] = blockIdx.x; ctx.status[5] = blockIdx.y; ctx.status[6] = blockIdx.z;
-                    __threadfence();
-                }
-                return false;
-            }
-        }
-    }
-}
-
-__device__ __forceinline__ bool wait_bar(uint32_t bar, uint32_t parity, const WaitCtx &ctx, int bar_id, int iter)
-{
-    if (mbar_try_wait(bar, parity)) return true;
-    return wait_slow(bar, parity, ctx, bar_id, iter);
-}
 
 __device__ __forceinline__ float as_f(uint32_t u) { return __uint_as_float(u); }
 __device__ __forceinline__ uint32_t as_u(float f) { return __float_as_uint(f); }
@@ -801,7 +765,30 @@ attn_sm100_kernel(const __grid_constant__ AttnParams p, const __grid_constant__ 
     }
 }
 
+// The bounded-wait machinery on its own: one warp waits on a barrier that nobody will ever
+// complete, gives up after limit_ns, leaves the record and returns normally.
+__global__ void wait_probe_kernel(uint32_t *status, unsigned long long limit_ns)
+{
+    __shared__ uint64_t never;
+    __shared__ int abort_flag;
+    if (threadIdx.x == 0) {
+        mbar_init(smem_u32(&never), 1);
+        abort_flag = 0;
+        fence_mbar_init();
+    }
+    __syncthreads();
+    WaitCtx ctx{&abort_flag, status, (int)(threadIdx.x >> 5)};
+    wait_bar(smem_u32(&never), 0, ctx, kProbeBarrierId, kProbeIteration, limit_ns);
+}
+
 }  // namespace
+
+cudaError_t launch_wait_probe(uint32_t *status, uint64_t limit_ns, cudaStream_t stream)
+{
+    wait_probe_kernel<<<1, 32, 0, stream>>>(status, (unsigned long long)limit_ns);
+    count_launch();
+    return cudaGetLastError();
+}
 
 cudaError_t launch_attn_sm100(const AttnParams &p, int head_dim, const CUtensorMap &qmap, const CUtensorMap &kmap,
                               const CUtensorMap &vmap, cudaStream_t stream)

@@ -505,6 +505,17 @@ int ll_debug_attn_plan(ll_cache *c, int layer, int recache, int sm_count, ll_att
     return LL_OK;
 }
 
+int ll_debug_wait_timeout(ll_cache *c, int limit_ms, ll_stream stream)
+{
+    if (!c) return fail(LL_ERR_INVALID_ARG, "null handle");
+    if (limit_ms < 1 || limit_ms > 1000) return fail(LL_ERR_INVALID_ARG, "limit_ms must be in [1, 1000]");
+    int s = need_storage(c);
+    if (s != LL_OK) return s;
+    cudaError_t e = ll::launch_wait_probe(reinterpret_cast<uint32_t *>(c->storage + c->off_status),
+                                          (uint64_t)limit_ms * 1000000ull, (cudaStream_t)stream);
+    return e == cudaSuccess ? LL_OK : cuda_fail(e, "wait probe kernel");
+}
+
 int ll_cache_reset(ll_cache *c)
 {
     if (!c) return fail(LL_ERR_INVALID_ARG, "null handle");

@@ -97,6 +97,10 @@ cudaError_t launch_attn_sm100(const AttnParams &p, int head_dim, const CUtensorM
                               const CUtensorMap &kmap, const CUtensorMap &vmap,
                               cudaStream_t stream);
 cudaError_t launch_attn_simt(const AttnParams &p, int head_dim, cudaStream_t stream);
+// what the probe of the bounded-wait machinery records as barrier and iteration
+constexpr int kProbeBarrierId = 99;
+constexpr int kProbeIteration = 7;
+cudaError_t launch_wait_probe(uint32_t *status, uint64_t limit_ns, cudaStream_t stream);
 
 void count_launch(int n = 1);
 void set_last_error(const char *msg);     // what ll_last_error() returns on this thread

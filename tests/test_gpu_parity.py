@@ -330,6 +330,38 @@ def test_recache_matches_oracle(oracle_mod, wl, at_chunks):
 # error paths on a live device
 # ---------------------------------------------------------------------------
 
+def test_a_wait_that_runs_out_is_reported_and_the_context_stays_usable(oracle_mod):
+    """No fault, no hang: a one-warp kernel waits 20 ms on a barrier nobody completes,
+    gives up, and leaves the record the host decodes.  An attention launch enqueued
+    while the record stands does no work; after the record is read (and cleared)
+    the same call works again and matches the oracle."""
+    wl = MEDIUM
+    cache = new_cache(wl)
+    orc = oracle_for(oracle_mod, wl)
+    C = wl.chunk_frames
+    q, k, v = synth.chunk_qkv(wl, 0)
+    dq, dk, dv = dev(q), dev(k), dev(v)
+    q_out = torch.empty_like(dq)
+    cache.rope_append_kv(0, dq, dk, dv, 0, wl.grid_h, wl.grid_w, wl.rope_theta, q_out)
+    orc.append(0, synth.bf16_bits_to_f64(k), synth.bf16_bits_to_f64(v), 0, wl.grid_h, wl.grid_w, wl.rope_theta)
+    cache.check_device()
+    B.ll_debug_wait_timeout(cache.h, 20)
+    skipped = torch.full_like(dq, 7.0)
+    B.ll_sink_window_attn(cache.h, 0, q_out, 0, C, skipped)         # enqueued behind the time-out: skips
+    with pytest.raises(B.LLError) as e:
+        cache.check_device()
+    assert e.value.code == B.LL_ERR_DEVICE_TIMEOUT
+    assert "barrier 99" in str(e.value) and "iteration 7" in str(e.value)
+    assert bool((skipped == 7.0).all())
+    cache.check_device()                                            # the record is gone
+    out = torch.full_like(dq, float("nan"))
+    B.ll_sink_window_attn(cache.h, 0, q_out, 0, C, out)
+    cache.check_device()
+    want, _ = orc.attn(0, orc.rope_q(synth.bf16_bits_to_f64(q), 0, wl.grid_h, wl.grid_w, wl.rope_theta), 0)
+    check_attn(f64(out), want)
+    cache.close()
+
+
 def test_errors_leave_state_unchanged():
     wl = MEDIUM
     cache = new_cache(wl)

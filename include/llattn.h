@@ -140,6 +140,28 @@ int ll_sink_window_attn(ll_cache *cache, int layer, const ll_bf16 *q_roped,
                         int64_t q_frame_start, int n_q_frames, ll_bf16 *out,
                         float *lse_out, ll_stream stream);
 
+/* The same for several independent streams in ONE launch (serving: the streams
+ * of a batch sit at different positions, with windows filled to different
+ * degrees and possibly of different sizes; Sec. 3.3's attention per stream is
+ * unchanged).  Each item is one ll_sink_window_attn call's arguments; the
+ * caches must agree in heads and head_dim and may differ in everything else,
+ * no (cache, layer) may appear twice, n_items <= LL_MAX_BATCH.  The kernel
+ * divides the work of all items between the SMs together, so small or
+ * partly filled windows do not leave SMs idle.  The scratch of items[0].cache
+ * is used; the usual rule (calls on a handle are ordered) extends to every
+ * handle named.  On error nothing is launched and no state changes. */
+#define LL_MAX_BATCH 8
+typedef struct ll_attn_item {
+    ll_cache *cache;
+    int32_t layer;
+    int32_t n_q_frames;                 /* must equal the cache's chunk_frames */
+    const ll_bf16 *q_roped;
+    int64_t q_frame_start;              /* must equal end - chunk_frames */
+    ll_bf16 *out;
+    float *lse_out;                     /* nullable */
+} ll_attn_item;
+int ll_sink_window_attn_batched(const ll_attn_item *items, int n_items, ll_stream stream);
+
 /* KV-recache (Sec. 3.1; Sec. 3.3 last paragraph: only the most recent W frames
  * are rebuilt; the sink is left alone).  q, k, v hold fresh activations for the
  * resident window frames [r0, end), r0 = max(S, end - W), oldest first.
@@ -241,14 +263,15 @@ int ll_debug_wait_timeout(ll_cache *cache, int limit_ms, ll_stream stream);
  * tiles[g] columns), n_kt[g] key tiles (steps) per column, the first
  * wave_cols[g] columns handed out whole (CTA i takes columns i, i + n_ctas, ...),
  * the steps of the others laid end to end from step_begin[g] and cut, with all
- * groups', into n_ctas equal shares: CTA i takes shared steps
- * [shared_steps * i / n_ctas, shared_steps * (i + 1) / n_ctas). */
+ * groups', into share_ctas = min(n_ctas, shared_steps) equal shares: CTA i <
+ * share_ctas takes shared steps [shared_steps * i / share_ctas,
+ * shared_steps * (i + 1) / share_ctas), the other CTAs none. */
 #define LL_MAX_GROUPS 24
 typedef struct ll_attn_plan {
     int32_t n_ctas;
     int32_t n_groups;
     int32_t heads;
-    int32_t reserved;
+    int32_t share_ctas;
     int64_t shared_steps;
     int32_t tiles[LL_MAX_GROUPS];
     int32_t n_kt[LL_MAX_GROUPS];

@@ -48,12 +48,27 @@ class ll_attn_plan(C.Structure):
         ("n_ctas", C.c_int32),
         ("n_groups", C.c_int32),
         ("heads", C.c_int32),
-        ("reserved", C.c_int32),
+        ("share_ctas", C.c_int32),
         ("shared_steps", C.c_int64),
         ("tiles", C.c_int32 * LL_MAX_GROUPS),
         ("n_kt", C.c_int32 * LL_MAX_GROUPS),
         ("wave_cols", C.c_int32 * LL_MAX_GROUPS),
         ("step_begin", C.c_int64 * LL_MAX_GROUPS),
+    ]
+
+
+LL_MAX_BATCH = 8
+
+
+class ll_attn_item(C.Structure):
+    _fields_ = [
+        ("cache", C.c_void_p),
+        ("layer", C.c_int32),
+        ("n_q_frames", C.c_int32),
+        ("q_roped", C.c_void_p),
+        ("q_frame_start", C.c_int64),
+        ("out", C.c_void_p),
+        ("lse_out", C.c_void_p),
     ]
 
 
@@ -76,6 +91,7 @@ SIGNATURES = {
                                     C.c_int, C.c_int, C.c_int, C.c_float, C.c_void_p, C.c_void_p]),
     "ll_sink_window_attn": (C.c_int, [C.c_void_p, C.c_int, C.c_void_p, C.c_int64, C.c_int, C.c_void_p,
                                       C.c_void_p, C.c_void_p]),
+    "ll_sink_window_attn_batched": (C.c_int, [C.POINTER(ll_attn_item), C.c_int, C.c_void_p]),
     "ll_recache": (C.c_int, [C.c_void_p, C.c_int, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int, C.c_int,
                              C.c_int, C.c_float, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]),
     "ll_rope_q_static": (C.c_int, [C.c_void_p, C.c_void_p, C.c_int, C.c_int, C.c_int64, C.c_int, C.c_int, C.c_int,
@@ -169,6 +185,17 @@ def ll_rope_append_kv(h, layer, q, k, v, frame_start, n_frames, grid_h, grid_w, 
 def ll_sink_window_attn(h, layer, q_roped, q_frame_start, n_q_frames, out, lse_out=None, stream=None):
     _check(lib().ll_sink_window_attn(h, layer, _ptr(q_roped), q_frame_start, n_q_frames, _ptr(out),
                                      _ptr(lse_out), _stream(stream)))
+
+
+def ll_sink_window_attn_batched(items, stream=None):
+    """items: sequence of (handle, layer, q_roped, q_frame_start, n_q_frames, out, lse_out or None)."""
+    def addr(t):
+        return None if t is None else t.data_ptr()
+    arr = (ll_attn_item * max(len(items), 1))()
+    for i, (h, layer, q_roped, q_frame_start, n_q_frames, out, lse_out) in enumerate(items):
+        arr[i] = ll_attn_item(h.value if isinstance(h, C.c_void_p) else h, layer, n_q_frames, addr(q_roped),
+                              q_frame_start, addr(out), addr(lse_out))
+    _check(lib().ll_sink_window_attn_batched(arr, len(items), _stream(stream)))
 
 
 def ll_debug_attn_simt(h, layer, q_roped, q_frame_start, n_q_frames, out, lse_out=None, stream=None):
@@ -291,6 +318,12 @@ class Cache:
 
     def sink_window_attn(self, layer, q_roped, q_frame_start, out, lse_out=None, stream=None):
         ll_sink_window_attn(self.h, layer, q_roped, q_frame_start, self.C, out, lse_out, stream)
+
+    @staticmethod
+    def sink_window_attn_batched(items, stream=None):
+        """items: (Cache, layer, q_roped, q_frame_start, out, lse_out or None) per stream, one launch."""
+        ll_sink_window_attn_batched([(c.h, layer, q, f0, c.C, out, lse) for c, layer, q, f0, out, lse in items],
+                                    stream)
 
     def recache(self, layer, q, k, v, n_frames, grid_h, grid_w, theta, q_out, out, lse_out=None, stream=None):
         ll_recache(self.h, layer, q, k, v, n_frames, grid_h, grid_w, theta, q_out, out, lse_out, stream)

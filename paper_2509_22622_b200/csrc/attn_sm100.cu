@@ -127,13 +127,13 @@ struct Segment {
 // First shared step of CTA `cta`'s share (the next CTA's is one past its last).
 __device__ __forceinline__ long long share_begin(const AttnParams &p, int cta)
 {
-    return p.total_steps * cta / p.n_ctas;
+    return p.total_steps * min(cta, p.share_ctas) / p.share_ctas;
 }
 
 // The CTA whose share holds shared step u.
 __device__ __forceinline__ int cta_of_step(const AttnParams &p, long long u)
 {
-    return (int)(((u + 1) * p.n_ctas - 1) / p.total_steps);
+    return (int)(((u + 1) * p.share_ctas - 1) / p.total_steps);
 }
 
 // A CTA's work in order: its whole columns, group by group and wave by wave, then its
@@ -233,8 +233,7 @@ __device__ __forceinline__ void mask_piece(uint32_t *v, int col0, int cq, int nv
 
 template <int D>
 __global__ void __launch_bounds__(kThreads, 1)
-attn_sm100_kernel(const __grid_constant__ AttnParams p, const __grid_constant__ CUtensorMap qmap,
-                  const __grid_constant__ CUtensorMap kmap, const __grid_constant__ CUtensorMap vmap)
+attn_sm100_kernel(const __grid_constant__ AttnParams p, const __grid_constant__ AttnMaps maps)
 {
     using C = Cfg<D>;
     extern __shared__ uint8_t smem_raw[];
@@ -291,9 +290,11 @@ attn_sm100_kernel(const __grid_constant__ AttnParams p, const __grid_constant__ 
         } else if (warp == kTmaWarp && lane == 0) {
             // =========================== TMA producer ===========================
             [&]() {
-                prefetch_tensormap(&qmap);
-                prefetch_tensormap(&kmap);
-                prefetch_tensormap(&vmap);
+                for (int i = 0; i < p.n_items; ++i) {
+                    prefetch_tensormap(&maps.q[i]);
+                    prefetch_tensormap(&maps.k[i]);
+                    prefetch_tensormap(&maps.v[i]);
+                }
                 uint32_t n = 0;                 // K/V tiles issued so far
                 uint32_t seg = 0;
                 Segment s;
@@ -302,6 +303,8 @@ attn_sm100_kernel(const __grid_constant__ AttnParams p, const __grid_constant__ 
                     // softmax ahead of the step's PV, so K runs one step ahead of V and three stages
                     // (the V in use, the K in use, one in flight) keep both fed.
                     KeyIter kit_k(&p.g[s.g], s.kt0), kit_v(&p.g[s.g], s.kt0);
+                    const int item = p.g[s.g].item;
+                    const CUtensorMap *qmap = &maps.q[item], *kmap = &maps.k[item], *vmap = &maps.v[item];
                     auto load_kv = [&](const CUtensorMap *m, int row) -> bool {
                         const int stage = n % C::kStages;
                         if (!wait(kKvEmpty + stage, (n / C::kStages) ^ 1u, (int)n)) return false;
@@ -314,20 +317,20 @@ attn_sm100_kernel(const __grid_constant__ AttnParams p, const __grid_constant__ 
                     };
                     // the first key tile goes out before Q: it needs no Q buffer and is in
                     // flight while the previous column's last products drain
-                    if (!load_kv(&kmap, kit_k.row())) return;
+                    if (!load_kv(kmap, kit_k.row())) return;
                     if (seg > 0 && !wait(kQEmpty, seg - 1, (int)seg)) return;
                     for (int w = 0; w < s.n_sub; ++w) {
                         mbar_arrive_expect_tx(bar(kQFull + w), C::kTileBytes);
                         for (int a = 0; a < C::kAtoms; ++a)
-                            tma_load_3d(q_smem + w * C::kTileBytes + a * C::kAtomBytes, &qmap, bar(kQFull + w),
+                            tma_load_3d(q_smem + w * C::kTileBytes + a * C::kAtomBytes, qmap, bar(kQFull + w),
                                         a * 64, s.head, s.q0 + 128 * w);
                     }
                     for (int j = s.kt0; j < s.kt1; ++j) {
                         if (j + 1 < s.kt1) {
                             kit_k.next();
-                            if (!load_kv(&kmap, kit_k.row())) return;
+                            if (!load_kv(kmap, kit_k.row())) return;
                         }
-                        if (!load_kv(&vmap, kit_v.row())) return;
+                        if (!load_kv(vmap, kit_v.row())) return;
                         kit_v.next();
                     }
                 }
@@ -624,9 +627,10 @@ attn_sm100_kernel(const __grid_constant__ AttnParams p, const __grid_constant__ 
                 }
                 const int row = 128 * w + row_a;               // row inside the column
                 const bool live_a = row < s.rows_valid, live_b = row + 8 < s.rows_valid;
-                ll_bf16 *dst_a = p.out + ((size_t)(s.q0 + row) * p.heads + s.head) * D;
+                const AttnItem &item = p.item[G.item];
+                ll_bf16 *dst_a = item.out + ((size_t)(s.q0 + row) * p.heads + s.head) * D;
                 ll_bf16 *dst_b = dst_a + (size_t)8 * p.heads * D;
-                float *lse_a = p.lse ? p.lse + (size_t)s.head * p.nq_total + s.q0 + row : nullptr;
+                float *lse_a = item.lse ? item.lse + (size_t)s.head * item.nq_total + s.q0 + row : nullptr;
 
                 bool finish = true;            // this warp writes the output rows
                 int i0 = 0, n_parts = 1;
@@ -790,8 +794,7 @@ cudaError_t launch_wait_probe(uint32_t *status, uint64_t limit_ns, cudaStream_t 
     return cudaGetLastError();
 }
 
-cudaError_t launch_attn_sm100(const AttnParams &p, int head_dim, const CUtensorMap &qmap, const CUtensorMap &kmap,
-                              const CUtensorMap &vmap, cudaStream_t stream)
+cudaError_t launch_attn_sm100(const AttnParams &p, int head_dim, const AttnMaps &maps, cudaStream_t stream)
 {
     if (p.n_ctas <= 0) return cudaSuccess;
     dim3 grid((unsigned)p.n_ctas);
@@ -804,11 +807,11 @@ cudaError_t launch_attn_sm100(const AttnParams &p, int head_dim, const CUtensorM
     if (head_dim == 128) {
         e = cudaFuncSetAttribute(attn_sm100_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg<128>::kSmemBytes);
         if (e != cudaSuccess) return e;
-        attn_sm100_kernel<128><<<grid, kThreads, Cfg<128>::kSmemBytes, stream>>>(p, qmap, kmap, vmap);
+        attn_sm100_kernel<128><<<grid, kThreads, Cfg<128>::kSmemBytes, stream>>>(p, maps);
     } else {
         e = cudaFuncSetAttribute(attn_sm100_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg<64>::kSmemBytes);
         if (e != cudaSuccess) return e;
-        attn_sm100_kernel<64><<<grid, kThreads, Cfg<64>::kSmemBytes, stream>>>(p, qmap, kmap, vmap);
+        attn_sm100_kernel<64><<<grid, kThreads, Cfg<64>::kSmemBytes, stream>>>(p, maps);
     }
     count_launch();
     return cudaGetLastError();

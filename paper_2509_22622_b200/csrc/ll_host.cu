@@ -170,74 +170,113 @@ int fill_rope_params(ll_cache *c, int layer, const ll_bf16 *q, const ll_bf16 *k,
     return LL_OK;
 }
 
-// Split a group's rows into query tiles and fill the launch parameters.
-int build_attn_params(ll_cache *c, int layer, const ll_bf16 *q, ll_bf16 *out, float *lse,
-                      int n_groups, const int64_t *group_frame_start, int64_t lo_floor,
-                      ll::AttnParams *p)
+// One (cache, layer, q, out) of an attention launch and the chunks of queries it brings.
+struct AttnCall {
+    ll_cache *c;
+    int layer;
+    const ll_bf16 *q;
+    ll_bf16 *out;
+    float *lse;
+    int n_groups;
+    int64_t group_frame_start[ll::kMaxGroups];
+    int64_t lo_floor;
+};
+
+// Fill the launch parameters of one launch serving `n_calls` calls: every call's query chunks
+// become groups, each split into query tiles, and the work is divided between the CTAs.
+// Scratch and status words are those of the first call's cache.
+int build_attn_params(const AttnCall *calls, int n_calls, ll::AttnParams *p)
 {
-    if (n_groups > ll::kMaxGroups) return fail(LL_ERR_UNSUPPORTED_SHAPE, "more than %d query groups", ll::kMaxGroups);
+    if (n_calls < 1 || n_calls > ll::kMaxItems) return fail(LL_ERR_UNSUPPORTED_SHAPE, "between 1 and %d items per launch", ll::kMaxItems);
+    ll_cache *c0 = calls[0].c;
     memset(p, 0, sizeof *p);
-    p->n_groups = n_groups;
-    p->heads = c->H;
-    p->rows_per_head = c->rows;
-    p->scale_log2 = (float)(1.4426950408889634 / std::sqrt((double)c->D));
-    p->q = q; p->out = out; p->lse = lse;
-    p->kbase = reinterpret_cast<const ll_bf16 *>(c->storage ? layer_k(c, layer) : nullptr);
-    p->vbase = reinterpret_cast<const ll_bf16 *>(c->storage ? layer_v(c, layer) : nullptr);
-    p->status = reinterpret_cast<uint32_t *>(c->storage ? c->storage + c->off_status : nullptr);
-    p->partial = reinterpret_cast<float *>(c->storage ? c->storage + c->off_partial : nullptr);
-    p->counters = reinterpret_cast<uint32_t *>(c->storage ? c->storage + c->off_counters : nullptr);
-    const int rows_per_group = c->C * c->P;
+    p->n_items = n_calls;
+    p->heads = c0->H;
+    p->rows_per_head = c0->rows;
+    p->scale_log2 = (float)(1.4426950408889634 / std::sqrt((double)c0->D));
+    p->q = calls[0].q; p->out = calls[0].out; p->lse = calls[0].lse;
+    p->kbase = reinterpret_cast<const ll_bf16 *>(c0->storage ? layer_k(c0, calls[0].layer) : nullptr);
+    p->vbase = reinterpret_cast<const ll_bf16 *>(c0->storage ? layer_v(c0, calls[0].layer) : nullptr);
+    p->status = reinterpret_cast<uint32_t *>(c0->storage ? c0->storage + c0->off_status : nullptr);
+    p->partial = reinterpret_cast<float *>(c0->storage ? c0->storage + c0->off_partial : nullptr);
+    p->counters = reinterpret_cast<uint32_t *>(c0->storage ? c0->storage + c0->off_counters : nullptr);
     // One persistent CTA per SM.  While a group still has a CTA's worth of columns they go
     // out whole, one per CTA and wave (CTAs on the same head then walk the keys in step and
     // share each K/V tile through L2); what is left over is cut into equal shares of steps.
-    const int sms = std::min(c->sm_count > 0 ? c->sm_count : 148, ll::kMaxCtas);
-    const long long cols_per_group = (long long)c->H * ((rows_per_group + ll::kQTileRows - 1) / ll::kQTileRows);
-    const bool waves = cols_per_group >= sms;
+    const int sms = std::min(c0->sm_count > 0 ? c0->sm_count : 148, ll::kMaxCtas);
+    bool waves = false;
     long long steps = 0, all_steps = 0;
-    for (int g = 0; g < n_groups; ++g) {
-        ll::AttnGroup &G = p->g[g];
-        G.q_begin = g * rows_per_group;
-        G.q_rows = rows_per_group;
-        G.tiles = (rows_per_group + ll::kQTileRows - 1) / ll::kQTileRows;
-        int64_t starts[LL_MAX_RANGES], lens[LL_MAX_RANGES];
-        int n = 0;
-        int st = visible_ranges(c, layer, group_frame_start[g], lo_floor, starts, lens, &n);
-        if (st != LL_OK) return st;
-        G.n_ranges = n;
-        G.n_kt = 0;
-        for (int r = 0; r < n; ++r) {
-            G.k_start[r] = (int)starts[r];
-            G.k_len[r] = (int)lens[r];
-            G.n_kt += (int)((lens[r] + ll::kKeyTile - 1) / ll::kKeyTile);
+    int ng = 0;
+    for (int i = 0; i < n_calls; ++i) {
+        const AttnCall &call = calls[i];
+        ll_cache *c = call.c;
+        if (c->H != c0->H || c->D != c0->D)
+            return fail(LL_ERR_UNSUPPORTED_SHAPE, "the items of one launch must agree in heads and head_dim");
+        if (ng + call.n_groups > ll::kMaxGroups) return fail(LL_ERR_UNSUPPORTED_SHAPE, "more than %d query groups", ll::kMaxGroups);
+        const int rows_per_group = c->C * c->P;
+        const int tiles = (rows_per_group + ll::kQTileRows - 1) / ll::kQTileRows;
+        const long long cols = (long long)c->H * tiles;
+        p->item[i].out = call.out;
+        p->item[i].lse = call.lse;
+        p->item[i].nq_total = call.n_groups * rows_per_group;
+        for (int g = 0; g < call.n_groups; ++g, ++ng) {
+            ll::AttnGroup &G = p->g[ng];
+            G.item = i;
+            G.q_begin = g * rows_per_group;
+            G.q_rows = rows_per_group;
+            G.tiles = tiles;
+            int64_t starts[LL_MAX_RANGES], lens[LL_MAX_RANGES];
+            int n = 0;
+            int st = visible_ranges(c, call.layer, call.group_frame_start[g], call.lo_floor, starts, lens, &n);
+            if (st != LL_OK) return st;
+            G.n_ranges = n;
+            G.n_kt = 0;
+            for (int r = 0; r < n; ++r) {
+                G.k_start[r] = (int)starts[r];
+                G.k_len[r] = (int)lens[r];
+                G.n_kt += (int)((lens[r] + ll::kKeyTile - 1) / ll::kKeyTile);
+            }
+            G.wave_cols = cols >= sms ? (int)(cols / sms * sms) : 0;
+            waves |= G.wave_cols > 0;
+            G.step_begin = steps;
+            steps += (cols - G.wave_cols) * G.n_kt;
+            all_steps += cols * G.n_kt;
         }
-        G.wave_cols = waves ? (int)(cols_per_group / sms * sms) : 0;
-        G.step_begin = steps;
-        steps += (cols_per_group - G.wave_cols) * G.n_kt;
-        all_steps += cols_per_group * G.n_kt;
     }
-    p->nq_total = n_groups * rows_per_group;
+    p->n_groups = ng;
+    p->nq_total = p->item[0].nq_total;
     p->total_steps = steps;
     p->n_ctas = waves ? sms : (int)std::min<long long>(sms, all_steps);
+    // with fewer shared steps than CTAs only the first CTAs take one each, so that the parts
+    // of a split column always sit in consecutive CTAs
+    p->share_ctas = (int)std::max<long long>(1, std::min<long long>(p->n_ctas, steps));
     return LL_OK;
 }
 
-int launch_attention(ll_cache *c, int layer, const ll::AttnParams &p, cudaStream_t stream, bool simt)
+int launch_attention(const AttnCall *calls, int n_calls, const ll::AttnParams &p, cudaStream_t stream, bool simt)
 {
+    ll_cache *c0 = calls[0].c;
     if (simt) {
-        cudaError_t e = ll::launch_attn_simt(p, c->D, stream);
+        cudaError_t e = ll::launch_attn_simt(p, c0->D, stream);
         return e == cudaSuccess ? LL_OK : cuda_fail(e, "simt attention kernel");
     }
-    CUtensorMap qmap;
-    int st = encode_map(&qmap, p.q, (uint64_t)c->D, (uint64_t)c->H, (uint64_t)p.nq_total,
-                        (uint64_t)c->D * 2, (uint64_t)c->H * c->D * 2, 1, 128);
-    if (st != LL_OK) return st;
-    cudaError_t e = ll::launch_attn_sm100(p, c->D, qmap, c->kmap[layer], c->vmap[layer], stream);
+    ll::AttnMaps maps;
+    memset(&maps, 0, sizeof maps);
+    for (int i = 0; i < n_calls; ++i) {
+        ll_cache *c = calls[i].c;
+        int st = encode_map(&maps.q[i], calls[i].q, (uint64_t)c->D, (uint64_t)c->H, (uint64_t)p.item[i].nq_total,
+                            (uint64_t)c->D * 2, (uint64_t)c->H * c->D * 2, 1, 128);
+        if (st != LL_OK) return st;
+        maps.k[i] = c->kmap[calls[i].layer];
+        maps.v[i] = c->vmap[calls[i].layer];
+    }
+    cudaError_t e = ll::launch_attn_sm100(p, c0->D, maps, stream);
     return e == cudaSuccess ? LL_OK : cuda_fail(e, "sink+window attention kernel");
 }
 
-int attn_entry(ll_cache *c, int layer, const ll_bf16 *q_roped, int64_t q_frame_start, int n_q_frames,
-               ll_bf16 *out, float *lse_out, ll_stream stream, bool simt)
+// Checks of one decode item (the newest chunk's queries of one layer of one cache).
+int check_decode_item(ll_cache *c, int layer, const ll_bf16 *q_roped, int64_t q_frame_start, int n_q_frames,
+                      ll_bf16 *out, float *lse_out)
 {
     if (!layer_ok(c, layer)) return fail(LL_ERR_INVALID_ARG, "bad cache handle or layer %d", layer);
     ll::LayerState &st = c->layers[layer];
@@ -252,14 +291,23 @@ int attn_entry(ll_cache *c, int layer, const ll_bf16 *q_roped, int64_t q_frame_s
         int s = need_storage(c);
         if (s != LL_OK) return s;
     }
+    return LL_OK;
+}
+
+int attn_entry(ll_cache *c, int layer, const ll_bf16 *q_roped, int64_t q_frame_start, int n_q_frames,
+               ll_bf16 *out, float *lse_out, ll_stream stream, bool simt)
+{
+    int s = check_decode_item(c, layer, q_roped, q_frame_start, n_q_frames, out, lse_out);
+    if (s != LL_OK) return s;
+    AttnCall call{c, layer, q_roped, out, lse_out, 1, {q_frame_start}, 0};
     ll::AttnParams p;
-    int s = build_attn_params(c, layer, q_roped, out, lse_out, 1, &q_frame_start, 0, &p);
+    s = build_attn_params(&call, 1, &p);
     if (s != LL_OK) return s;
     if (!c->dry_run) {
-        s = launch_attention(c, layer, p, (cudaStream_t)stream, simt);
+        s = launch_attention(&call, 1, p, (cudaStream_t)stream, simt);
         if (s != LL_OK) return s;
     }
-    st.n_attn += 1;
+    c->layers[layer].n_attn += 1;
     return LL_OK;
 }
 
@@ -419,6 +467,34 @@ int ll_sink_window_attn(ll_cache *c, int layer, const ll_bf16 *q_roped, int64_t 
     return attn_entry(c, layer, q_roped, q_frame_start, n_q_frames, out, lse_out, stream, false);
 }
 
+int ll_sink_window_attn_batched(const ll_attn_item *items, int n_items, ll_stream stream)
+{
+    if (!items || n_items < 1) return fail(LL_ERR_INVALID_ARG, "no items");
+    if (n_items > LL_MAX_BATCH) return fail(LL_ERR_UNSUPPORTED_SHAPE, "more than %d items", LL_MAX_BATCH);
+    static_assert(LL_MAX_BATCH == ll::kMaxItems, "header and kernel disagree on the batch limit");
+    AttnCall calls[ll::kMaxItems];
+    for (int i = 0; i < n_items; ++i) {
+        const ll_attn_item &it = items[i];
+        int s = check_decode_item(it.cache, it.layer, it.q_roped, it.q_frame_start, it.n_q_frames, it.out, it.lse_out);
+        if (s != LL_OK) return s;
+        if (it.cache->dry_run != items[0].cache->dry_run)
+            return fail(LL_ERR_INVALID_ARG, "bookkeeping-only and real handles cannot share a launch");
+        for (int j = 0; j < i; ++j)
+            if (items[j].cache == it.cache && items[j].layer == it.layer)
+                return fail(LL_ERR_INVALID_ARG, "items %d and %d name the same layer of the same cache", j, i);
+        calls[i] = AttnCall{it.cache, it.layer, it.q_roped, it.out, it.lse_out, 1, {it.q_frame_start}, 0};
+    }
+    ll::AttnParams p;
+    int s = build_attn_params(calls, n_items, &p);
+    if (s != LL_OK) return s;
+    if (!items[0].cache->dry_run) {
+        s = launch_attention(calls, n_items, p, (cudaStream_t)stream, false);
+        if (s != LL_OK) return s;
+    }
+    for (int i = 0; i < n_items; ++i) items[i].cache->layers[items[i].layer].n_attn += 1;
+    return LL_OK;
+}
+
 int ll_debug_attn_simt(ll_cache *c, int layer, const ll_bf16 *q_roped, int64_t q_frame_start,
                        int n_q_frames, ll_bf16 *out, float *lse_out, ll_stream stream)
 {
@@ -450,8 +526,10 @@ int ll_recache(ll_cache *c, int layer, const ll_bf16 *q, const ll_bf16 *k, const
         int s = need_storage(c);
         if (s != LL_OK) return s;
     }
+    AttnCall call{c, layer, q_out, out, lse_out, n_groups, {}, r0};
+    for (int g = 0; g < n_groups; ++g) call.group_frame_start[g] = gstart[g];
     ll::AttnParams ap;
-    int s = build_attn_params(c, layer, q_out, out, lse_out, n_groups, gstart, r0, &ap);
+    int s = build_attn_params(&call, 1, &ap);
     if (s != LL_OK) return s;
     if (!c->dry_run) {
         s = ensure_tables(c, r0, st.end, grid_h, grid_w, rope_theta, (cudaStream_t)stream);
@@ -460,7 +538,7 @@ int ll_recache(ll_cache *c, int layer, const ll_bf16 *q, const ll_bf16 *k, const
         fill_rope_params(c, layer, q, k, v, q_out, r0, n_frames, grid_w, &rp);
         cudaError_t e = ll::launch_rope_append(rp, c->D, (cudaStream_t)stream);
         if (e != cudaSuccess) return cuda_fail(e, "rope+append kernel (recache)");
-        s = launch_attention(c, layer, ap, (cudaStream_t)stream, false);
+        s = launch_attention(&call, 1, ap, (cudaStream_t)stream, false);
         if (s != LL_OK) return s;
     }
     st.n_recaches += 1;
@@ -488,13 +566,16 @@ int ll_debug_attn_plan(ll_cache *c, int layer, int recache, int sm_count, ll_att
     if (n_groups == 0) return LL_OK;
     const int saved = c->sm_count;
     if (sm_count > 0) c->sm_count = sm_count;
+    AttnCall call{c, layer, nullptr, nullptr, nullptr, n_groups, {}, lo_floor};
+    for (int g = 0; g < n_groups; ++g) call.group_frame_start[g] = gstart[g];
     ll::AttnParams p;
-    const int s = build_attn_params(c, layer, nullptr, nullptr, nullptr, n_groups, gstart, lo_floor, &p);
+    const int s = build_attn_params(&call, 1, &p);
     c->sm_count = saved;
     if (s != LL_OK) return s;
     out->n_ctas = p.n_ctas;
     out->n_groups = p.n_groups;
     out->heads = p.heads;
+    out->share_ctas = p.share_ctas;
     out->shared_steps = p.total_steps;
     for (int g = 0; g < p.n_groups; ++g) {
         out->tiles[g] = p.g[g].tiles;

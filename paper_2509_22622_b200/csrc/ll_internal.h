@@ -13,6 +13,7 @@
 namespace ll {
 
 constexpr int kMaxGroups = 24;        // query groups (chunks) one attention launch can hold
+constexpr int kMaxItems = 8;          // (cache, layer, q, out) tuples one attention launch can serve
 constexpr int kTTabFrames = 256;      // frames covered by the resident t-axis RoPE table
 constexpr int kTTabAlign = 128;       // table base is a multiple of this many frames
 constexpr int kStatusWords = 64;      // uint32 words at the head of the aux block
@@ -41,7 +42,8 @@ struct LayerState {
 // laid end to end after those of earlier groups' remainders and cut into equal
 // shares.
 struct AttnGroup {
-    int q_begin;                      // first query row of the group in the q tensor
+    int item;                         // which (cache, layer, q, out) of the launch the group belongs to
+    int q_begin;                      // first query row of the group in its item's q tensor
     int q_rows;                       // rows in the group
     int tiles;                        // query tiles of kQTileRows rows
     int n_kt;                         // key tiles (steps) per column
@@ -56,12 +58,26 @@ struct AttnGroup {
 // (reference max, sum) per row.
 inline size_t attn_slot_bytes(int head_dim) { return (size_t)kQTileRows * (head_dim + 2) * sizeof(float); }
 
+// What differs between the items of a batched launch (the K/V and Q tensor maps are in AttnMaps).
+struct AttnItem {
+    ll_bf16 *out;                     // [nq_total, H, D]
+    float *lse;                       // [H, nq_total] or null
+    int nq_total;                     // rows of this item's q / out
+    int pad;
+};
+
+struct AttnMaps {
+    CUtensorMap q[kMaxItems], k[kMaxItems], v[kMaxItems];
+};
+
 struct AttnParams {
     int n_groups;
+    int n_items;
     int heads;
-    int nq_total;                     // rows of q / out
+    int nq_total;                     // rows of q / out of item 0 (the triage kernel serves one item)
     int n_ctas;                       // grid.x: persistent CTAs
-    long long total_steps;            // shared steps of all groups (cut evenly across the CTAs)
+    int share_ctas;                   // the first share_ctas CTAs take a share of the shared steps (each >= 1 step)
+    long long total_steps;            // shared steps of all groups (cut evenly across those CTAs)
     int64_t rows_per_head;            // (S+W)*P
     float scale_log2;                 // log2(e) / sqrt(D)
     const ll_bf16 *q;                 // [nq_total, H, D]
@@ -72,6 +88,7 @@ struct AttnParams {
     uint32_t *status;                 // aux status words
     float *partial;                   // 2 * kMaxCtas slots of attn_slot_bytes
     uint32_t *counters;               // kMaxCtas * kSlabs arrival counters, zero between launches
+    AttnItem item[kMaxItems];
     AttnGroup g[kMaxGroups];
 };
 
@@ -93,9 +110,7 @@ cudaError_t launch_rope_tables(float2 *t_tab, int64_t t_base, int n_t_frames, in
                                float2 *h_tab, int grid_h, float2 *w_tab, int grid_w, int n_hw,
                                float theta, bool do_t, bool do_hw, cudaStream_t stream);
 cudaError_t launch_rope_append(const RopeAppendParams &p, int head_dim, cudaStream_t stream);
-cudaError_t launch_attn_sm100(const AttnParams &p, int head_dim, const CUtensorMap &qmap,
-                              const CUtensorMap &kmap, const CUtensorMap &vmap,
-                              cudaStream_t stream);
+cudaError_t launch_attn_sm100(const AttnParams &p, int head_dim, const AttnMaps &maps, cudaStream_t stream);
 cudaError_t launch_attn_simt(const AttnParams &p, int head_dim, cudaStream_t stream);
 // what the probe of the bounded-wait machinery records as barrier and iteration
 constexpr int kProbeBarrierId = 99;

@@ -8,7 +8,7 @@ a column split over several CTAs is split into contiguous parts whose owners
 can be found from the first step alone, and no CTA does more than one step more
 than another."""
 import pytest
-from hypothesis import given, settings, strategies as st
+from hypothesis import example, given, settings, strategies as st
 
 from paper_2509_22622_b200 import binding as B
 
@@ -26,8 +26,9 @@ def cta_work(plan, cta):
     for g in range(plan.n_groups):
         for wave in range(plan.wave_cols[g] // G):
             out.append((g, wave * G + cta, 0, plan.n_kt[g]))
-    u = plan.shared_steps * cta // G
-    end = plan.shared_steps * (cta + 1) // G
+    S = plan.share_ctas
+    u = plan.shared_steps * min(cta, S) // S
+    end = plan.shared_steps * min(cta + 1, S) // S
     while u < end:
         # the group whose shared steps hold u
         g = 0
@@ -42,7 +43,7 @@ def cta_work(plan, cta):
 
 
 def owner_of_shared_step(plan, u):
-    return ((u + 1) * plan.n_ctas - 1) // plan.shared_steps
+    return ((u + 1) * plan.share_ctas - 1) // plan.shared_steps
 
 
 def check_plan(plan):
@@ -100,6 +101,8 @@ def test_plan_of_the_benchmark_layer():
 @given(heads=st.integers(1, 12), P=st.integers(1, 700), C=st.integers(1, 3), s_chunks=st.integers(0, 2),
        w_chunks=st.integers(1, 4), n_chunks=st.integers(1, 12), sms=st.sampled_from([1, 7, 148, 160]),
        recache=st.booleans())
+# fewer shared steps (3) than CTAs (7): the CTAs that take one must still be consecutive
+@example(heads=11, P=86, C=3, s_chunks=0, w_chunks=1, n_chunks=1, sms=7, recache=False)
 def test_every_step_is_done_exactly_once(heads, P, C, s_chunks, w_chunks, n_chunks, sms, recache):
     h = make_cache(heads, P, C, s_chunks * C, w_chunks * C, n_chunks)
     plan = B.ll_debug_attn_plan(h, recache=recache, sm_count=sms)

@@ -229,24 +229,38 @@ def test_config3_long_stream(oracle_mod):
 # config 4: ragged stream positions x window sweep, 1% outliers x20
 # ---------------------------------------------------------------------------
 
+@pytest.mark.parametrize("batched", [False, True], ids=["per_stream", "one_launch"])
 @pytest.mark.parametrize("W", synth.SWEEP_WINDOWS)
-def test_config4_ragged_streams_window_sweep(oracle_mod, W):
+def test_config4_ragged_streams_window_sweep(oracle_mod, W, batched):
+    """Each stream owns a cache and sits at its own position; the attention of the
+    newest chunk runs either as one call per stream or as one launch for all."""
     wl = dataclasses.replace(synth.CONFIGS[4], window_frames=W)
     C, S = wl.chunk_frames, wl.sink_frames
     pool = synth.InputPool(wl)
     dpool = DevicePool(pool)
     positions = synth.SWEEP_POSITIONS if W == 9 else (0, 2, 6, 50)
     nq = wl.chunk_tokens
-    q_out = torch.empty(nq, wl.heads, wl.head_dim, device="cuda", dtype=torch.bfloat16)
-    worst = (0.0, 0.0)
+    caches, q_outs, outs = [], [], []
     for stream, pos in enumerate(positions):
-        cache = new_cache(wl)                       # every stream owns its cache
+        cache = new_cache(wl)
+        q_out = torch.empty(nq, wl.heads, wl.head_dim, device="cuda", dtype=torch.bfloat16)
         for chunk in range(pos + 1):
             dq, dk, dv = dpool.get(chunk, 0, 0, stream)
             cache.rope_append_kv(0, dq, dk, dv, chunk * C, wl.grid_h, wl.grid_w, wl.rope_theta, q_out)
-        out = torch.full_like(q_out, float("nan"))
-        cache.sink_window_attn(0, q_out, pos * C, out)
+        caches.append(cache)
+        q_outs.append(q_out)
+        outs.append(torch.full_like(q_out, float("nan")))
+    if batched:
+        B.Cache.sink_window_attn_batched([(cache, 0, q_out, pos * C, out, None)
+                                          for cache, q_out, out, pos in zip(caches, q_outs, outs, positions)])
+    else:
+        for cache, q_out, out, pos in zip(caches, q_outs, outs, positions):
+            cache.sink_window_attn(0, q_out, pos * C, out)
+    worst = (0.0, 0.0)
+    for stream, pos in enumerate(positions):
+        cache, out = caches[stream], outs[stream]
         cache.check_device()
+        assert cache.state()["attn_calls"] == 1
         # reference: storage-faithful oracle; a twin with |V| gives the error scale sum_j p_j |v_j|
         orc = make_oracle(oracle_mod, wl, faithful=True)
         orc_abs = make_oracle(oracle_mod, wl, faithful=True)
@@ -265,4 +279,5 @@ def test_config4_ragged_streams_window_sweep(oracle_mod, W):
         orc.close()
         orc_abs.close()
         cache.close()
-    print("parity config4 W=%d: worst scaled max %.3e mean %.3e" % (W, worst[0], worst[1]))
+    print("parity config4 W=%d %s: worst scaled max %.3e mean %.3e"
+          % (W, "one launch" if batched else "per stream", worst[0], worst[1]))

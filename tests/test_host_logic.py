@@ -172,3 +172,42 @@ def test_attention_position_checks():
     with pytest.raises(B.LLError):
         B.ll_sink_window_attn(c.h, 0, None, 3, 2, None)
     assert c.state()["attn_calls"] == 1
+
+
+def test_batched_attention_checks_every_item_before_anything_changes():
+    a = B.Cache(2, 2, 64, 2, 3, 3, 9, dry_run=True)
+    b = B.Cache(1, 2, 64, 5, 1, 0, 2, dry_run=True)            # other frame size, chunk, sink, window
+    three_heads = B.Cache(1, 3, 64, 2, 3, 3, 9, dry_run=True)
+    d128 = B.Cache(1, 2, 128, 2, 3, 3, 9, dry_run=True)
+    for c in (a, three_heads, d128):
+        for layer in range(c.L):
+            B.ll_rope_append_kv(c.h, layer, None, None, None, 0, 3, 1, 2)
+    B.ll_rope_append_kv(b.h, 0, None, None, None, 0, 1, 1, 5)
+    B.ll_rope_append_kv(b.h, 0, None, None, None, 1, 1, 1, 5)
+
+    def item(c, layer=0, start=0):
+        return (c.h, layer, None, start, c.C, None, None)
+
+    def calls():
+        return [a.state(0)["attn_calls"], a.state(1)["attn_calls"], b.state()["attn_calls"]]
+
+    B.ll_sink_window_attn_batched([item(a, 0), item(b, 0, 1), item(a, 1)])
+    assert calls() == [1, 1, 1]
+    for bad, code in [([], B.LL_ERR_INVALID_ARG),
+                      ([item(a), item(three_heads)], B.LL_ERR_UNSUPPORTED_SHAPE),
+                      ([item(a), item(d128)], B.LL_ERR_UNSUPPORTED_SHAPE),
+                      ([item(a), item(b, 0, 1), item(a)], B.LL_ERR_INVALID_ARG),          # a layer twice
+                      ([item(a), item(b, 0, 0)], B.LL_ERR_BAD_POSITION),                  # b's newest chunk is frame 1
+                      ([item(a), item(a, 5)], B.LL_ERR_INVALID_ARG)]:                     # no such layer
+        with pytest.raises(B.LLError) as e:
+            B.ll_sink_window_attn_batched(bad)
+        assert e.value.code == code, bad
+        assert calls() == [1, 1, 1]
+    many = [B.Cache(1, 2, 64, 2, 3, 3, 9, dry_run=True) for _ in range(B.LL_MAX_BATCH + 1)]
+    for c in many:
+        B.ll_rope_append_kv(c.h, 0, None, None, None, 0, 3, 1, 2)
+    B.ll_sink_window_attn_batched([item(c) for c in many[:B.LL_MAX_BATCH]])
+    with pytest.raises(B.LLError) as e:
+        B.ll_sink_window_attn_batched([item(c) for c in many])
+    assert e.value.code == B.LL_ERR_UNSUPPORTED_SHAPE
+    assert [c.state()["attn_calls"] for c in many] == [1] * B.LL_MAX_BATCH + [0]

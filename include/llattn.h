@@ -260,25 +260,36 @@ int ll_debug_wait_timeout(ll_cache *cache, int limit_ms, ll_stream stream);
  * the newest chunk; recache = 1: ll_recache of the resident window.  sm_count > 0
  * overrides the SM count of the storage's device (148 when no storage is bound).
  * Per query group g: tiles[g] query tiles of 256 rows per head (so heads *
- * tiles[g] columns), n_kt[g] key tiles (steps) per column, the first
- * wave_cols[g] columns handed out whole (CTA i takes columns i, i + n_ctas, ...),
- * the steps of the others laid end to end from step_begin[g] and cut, with all
- * groups', into share_ctas = min(n_ctas, shared_steps) equal shares: CTA i <
- * share_ctas takes shared steps [shared_steps * i / share_ctas,
- * shared_steps * (i + 1) / share_ctas), the other CTAs none. */
+ * tiles[g] columns), n_kt[g] key tiles (steps) per column.  The columns of all
+ * groups are numbered through (group g's first is col_begin[g]); the first
+ * n_waves * n_ctas go out whole, CTA i taking columns i, i + n_ctas, ... (of
+ * group g these are its first wave_cols[g]).  The steps of the other columns
+ * are laid end to end (group g's from step_begin[g]) and cut into n_shares
+ * shares: CTA i takes shared steps [share_begin[k], share_begin[k + 1]) with
+ * k = share_of_cta[i], or none when that is -1.  Shares are sized so that
+ * whole columns plus share come to the same number of steps on every CTA.
+ * ll_debug_attn_plan_batched: the same for ll_sink_window_attn_batched of the
+ * newest chunk of every item (only cache and layer of an item are read). */
 #define LL_MAX_GROUPS 24
+#define LL_MAX_CTAS 160
 typedef struct ll_attn_plan {
     int32_t n_ctas;
     int32_t n_groups;
     int32_t heads;
-    int32_t share_ctas;
+    int32_t n_waves;
+    int32_t n_shares;
+    int32_t reserved;
     int64_t shared_steps;
     int32_t tiles[LL_MAX_GROUPS];
     int32_t n_kt[LL_MAX_GROUPS];
+    int32_t col_begin[LL_MAX_GROUPS];
     int32_t wave_cols[LL_MAX_GROUPS];
     int64_t step_begin[LL_MAX_GROUPS];
+    int32_t share_begin[LL_MAX_CTAS + 1];
+    int32_t share_of_cta[LL_MAX_CTAS];
 } ll_attn_plan;
 int ll_debug_attn_plan(ll_cache *cache, int layer, int recache, int sm_count, ll_attn_plan *out);
+int ll_debug_attn_plan_batched(const ll_attn_item *items, int n_items, int sm_count, ll_attn_plan *out);
 
 /* Kernel launches made by this process through the library so far. */
 int64_t ll_launch_count(void);

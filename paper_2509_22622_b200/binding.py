@@ -41,6 +41,7 @@ class ll_state(C.Structure):
 
 
 LL_MAX_GROUPS = 24
+LL_MAX_CTAS = 160
 
 
 class ll_attn_plan(C.Structure):
@@ -48,12 +49,17 @@ class ll_attn_plan(C.Structure):
         ("n_ctas", C.c_int32),
         ("n_groups", C.c_int32),
         ("heads", C.c_int32),
-        ("share_ctas", C.c_int32),
+        ("n_waves", C.c_int32),
+        ("n_shares", C.c_int32),
+        ("reserved", C.c_int32),
         ("shared_steps", C.c_int64),
         ("tiles", C.c_int32 * LL_MAX_GROUPS),
         ("n_kt", C.c_int32 * LL_MAX_GROUPS),
+        ("col_begin", C.c_int32 * LL_MAX_GROUPS),
         ("wave_cols", C.c_int32 * LL_MAX_GROUPS),
         ("step_begin", C.c_int64 * LL_MAX_GROUPS),
+        ("share_begin", C.c_int32 * (LL_MAX_CTAS + 1)),
+        ("share_of_cta", C.c_int32 * LL_MAX_CTAS),
     ]
 
 
@@ -107,6 +113,7 @@ SIGNATURES = {
                                      C.c_void_p, C.c_void_p]),
     "ll_debug_wait_timeout": (C.c_int, [C.c_void_p, C.c_int, C.c_void_p]),
     "ll_debug_attn_plan": (C.c_int, [C.c_void_p, C.c_int, C.c_int, C.c_int, C.POINTER(ll_attn_plan)]),
+    "ll_debug_attn_plan_batched": (C.c_int, [C.POINTER(ll_attn_item), C.c_int, C.c_int, C.POINTER(ll_attn_plan)]),
     "ll_launch_count": (C.c_int64, []),
     "ll_last_error": (C.c_char_p, []),
     "ll_version": (C.c_char_p, []),
@@ -252,6 +259,16 @@ def ll_debug_wait_timeout(h, limit_ms=20, stream=None):
 def ll_debug_attn_plan(h, layer=0, recache=False, sm_count=0) -> ll_attn_plan:
     plan = ll_attn_plan()
     _check(lib().ll_debug_attn_plan(h, layer, int(recache), sm_count, C.byref(plan)))
+    return plan
+
+
+def ll_debug_attn_plan_batched(handles_and_layers, sm_count=0) -> ll_attn_plan:
+    arr = (ll_attn_item * len(handles_and_layers))()
+    for i, (h, layer) in enumerate(handles_and_layers):
+        arr[i].cache = h.value if isinstance(h, C.c_void_p) else h
+        arr[i].layer = layer
+    plan = ll_attn_plan()
+    _check(lib().ll_debug_attn_plan_batched(arr, len(handles_and_layers), sm_count, C.byref(plan)))
     return plan
 
 

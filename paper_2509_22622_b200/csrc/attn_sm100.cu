@@ -121,29 +121,23 @@ struct Segment {
     int q0;                 // first query row of the column
     int rows_valid;         // live rows of the 256
     int n_sub;              // live 128-row tiles
-    long long col_begin;    // shared-step index of the column's first step (split columns only)
+    int col_begin;          // shared-step index of the column's first step (split columns only)
 };
 
-// First shared step of CTA `cta`'s share (the next CTA's is one past its last).
-__device__ __forceinline__ long long share_begin(const AttnParams &p, int cta)
-{
-    return p.total_steps * min(cta, p.share_ctas) / p.share_ctas;
-}
-
-// The CTA whose share holds shared step u.
-__device__ __forceinline__ int cta_of_step(const AttnParams &p, long long u)
-{
-    return (int)(((u + 1) * p.share_ctas - 1) / p.total_steps);
-}
-
-// A CTA's work in order: its whole columns, group by group and wave by wave, then its
-// share of the steps that are left.  Every role of the CTA walks the same sequence.
+// A CTA's work in order: its whole columns, wave by wave, then its share of the steps
+// that are left.  Every role of the CTA walks the same sequence.
 struct WorkIter {
     const AttnParams &p;
-    int cta, g, wave;
-    long long u, end;
+    int cta, g, wave, share;
+    int u, end;
     __device__ WorkIter(const AttnParams &prm, int cta_)
-        : p(prm), cta(cta_), g(0), wave(0), u(share_begin(prm, cta_)), end(share_begin(prm, cta_ + 1)) {}
+        : p(prm), cta(cta_), g(0), wave(0), share(prm.share_of_cta[cta_]), u(0), end(0)
+    {
+        if (share >= 0) {
+            u = p.share_begin[share];
+            end = p.share_begin[share + 1];
+        }
+    }
     __device__ void fill(Segment &s, int grp, int col, int kt0, int kt1) const
     {
         const AttnGroup &G = p.g[grp];
@@ -158,24 +152,22 @@ struct WorkIter {
     }
     __device__ bool next(Segment &s)
     {
-        while (g < p.n_groups) {
-            if ((wave + 1) * p.n_ctas <= p.g[g].wave_cols) {
-                fill(s, g, wave * p.n_ctas + cta, 0, p.g[g].n_kt);
-                s.col_begin = 0;
-                ++wave;
-                return true;
-            }
-            ++g;
-            wave = 0;
+        if (wave < p.n_waves) {
+            const int col = wave * p.n_ctas + cta;                  // launch-wide column number
+            while (col >= p.g[g].col_begin + p.heads * p.g[g].tiles) ++g;
+            fill(s, g, col - p.g[g].col_begin, 0, p.g[g].n_kt);
+            s.col_begin = 0;
+            ++wave;
+            return true;
         }
         if (u >= end) return false;
         int gg = 0;
         while (gg + 1 < p.n_groups && u >= p.g[gg + 1].step_begin) ++gg;
         const AttnGroup &G = p.g[gg];
-        const long long off = u - G.step_begin;
-        const int col = (int)(off / G.n_kt);
-        const int kt0 = (int)(off - (long long)col * G.n_kt);
-        const int kt1 = (int)min((long long)G.n_kt, kt0 + (end - u));
+        const int off = u - (int)G.step_begin;
+        const int col = off / G.n_kt;
+        const int kt0 = off - col * G.n_kt;
+        const int kt1 = min(G.n_kt, kt0 + (end - u));
         fill(s, gg, G.wave_cols + col, kt0, kt1);
         s.col_begin = u - kt0;
         u += kt1 - kt0;
@@ -638,9 +630,14 @@ attn_sm100_kernel(const __grid_constant__ AttnParams p, const __grid_constant__ 
                 const size_t slot_floats = (size_t)kQTileRows * (D + 2);
                 if (!whole) {
                     // leave this part in its slot and count the arrival
-                    i0 = cta_of_step(p, s.col_begin);
-                    n_parts = cta_of_step(p, s.col_begin + G.n_kt - 1) - i0 + 1;
-                    float *slot = p.partial + (size_t)(2 * cta + (s.kt0 == 0 ? 1 : 0)) * slot_floats;
+                    // (the parts of a column sit in consecutive shares; i0 = the share with its first step)
+                    const int own = p.share_of_cta[cta];
+                    int i1 = own;
+                    i0 = own;
+                    while (p.share_begin[i0] > s.col_begin) --i0;
+                    while (p.share_begin[i1 + 1] < s.col_begin + G.n_kt) ++i1;
+                    n_parts = i1 - i0 + 1;
+                    float *slot = p.partial + (size_t)(2 * own + (s.kt0 == 0 ? 1 : 0)) * slot_floats;
 #pragma unroll 1
                     for (int ch = 0; ch < C::kOChunks; ++ch) {
                         uint32_t o[32];

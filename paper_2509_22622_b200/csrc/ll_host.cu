@@ -182,6 +182,65 @@ struct AttnCall {
     int64_t lo_floor;
 };
 
+// Divide the columns of all groups between the CTAs (one persistent CTA per SM).  The
+// columns are numbered through, group after group.  While a CTA's worth of them is
+// left they go out whole, one per CTA and wave (CTAs on the same head then walk the keys
+// in step and share each K/V tile through L2).  The steps of the columns left over are
+// laid end to end and cut into shares: a CTA's share is what it lacks to the common
+// level T of steps, after its whole columns; CTAs already above T take none.
+void plan_work(ll::AttnParams *p, int sms, long long all_cols, long long all_steps)
+{
+    const bool waves = all_cols >= sms;
+    p->n_ctas = waves ? sms : (int)std::min<long long>(sms, all_steps);
+    p->n_waves = waves ? (int)(all_cols / sms) : 0;
+    const long long whole_cols = (long long)p->n_waves * p->n_ctas;
+    long long steps = 0;
+    for (int g = 0; g < p->n_groups; ++g) {
+        ll::AttnGroup &G = p->g[g];
+        const long long cols = (long long)p->heads * G.tiles;
+        G.wave_cols = (int)std::min(cols, std::max<long long>(0, whole_cols - G.col_begin));
+        G.step_begin = steps;
+        steps += (cols - G.wave_cols) * G.n_kt;
+    }
+    p->total_steps = steps;
+    // steps each CTA gets as whole columns
+    long long load[ll::kMaxCtas] = {};
+    {
+        int g = 0;
+        for (long long col = 0; col < whole_cols; ++col) {
+            while (col >= p->g[g].col_begin + (long long)p->heads * p->g[g].tiles) ++g;
+            load[col % p->n_ctas] += p->g[g].n_kt;
+        }
+    }
+    // the highest level T that the shared steps can fill: sum over CTAs of max(0, T - load) <= steps
+    auto fill = [&](long long T) {
+        long long need = 0;
+        for (int i = 0; i < p->n_ctas; ++i) need += std::max<long long>(0, T - load[i]);
+        return need;
+    };
+    long long lo = 0, hi = 0;
+    for (int i = 0; i < p->n_ctas; ++i) hi = std::max(hi, load[i]);
+    hi += steps + 1;                                     // fill(hi) > steps
+    while (hi - lo > 1) {
+        const long long mid = lo + (hi - lo) / 2;
+        if (fill(mid) <= steps) lo = mid; else hi = mid;
+    }
+    const long long T = lo;
+    long long extra = steps - fill(T);                   // fewer than the CTAs at or below T: one more step each
+    int k = 0;
+    p->share_begin[0] = 0;
+    for (int i = 0; i < p->n_ctas; ++i) {
+        long long size = std::max<long long>(0, T - load[i]);
+        if (load[i] <= T && extra > 0) { ++size; --extra; }
+        p->share_of_cta[i] = size > 0 ? (short)k : (short)-1;
+        if (size > 0) {
+            p->share_begin[k + 1] = p->share_begin[k] + (int)size;
+            ++k;
+        }
+    }
+    p->n_shares = k;
+}
+
 // Fill the launch parameters of one launch serving `n_calls` calls: every call's query chunks
 // become groups, each split into query tiles, and the work is divided between the CTAs.
 // Scratch and status words are those of the first call's cache.
@@ -200,12 +259,8 @@ int build_attn_params(const AttnCall *calls, int n_calls, ll::AttnParams *p)
     p->status = reinterpret_cast<uint32_t *>(c0->storage ? c0->storage + c0->off_status : nullptr);
     p->partial = reinterpret_cast<float *>(c0->storage ? c0->storage + c0->off_partial : nullptr);
     p->counters = reinterpret_cast<uint32_t *>(c0->storage ? c0->storage + c0->off_counters : nullptr);
-    // One persistent CTA per SM.  While a group still has a CTA's worth of columns they go
-    // out whole, one per CTA and wave (CTAs on the same head then walk the keys in step and
-    // share each K/V tile through L2); what is left over is cut into equal shares of steps.
     const int sms = std::min(c0->sm_count > 0 ? c0->sm_count : 148, ll::kMaxCtas);
-    bool waves = false;
-    long long steps = 0, all_steps = 0;
+    long long all_steps = 0, all_cols = 0;
     int ng = 0;
     for (int i = 0; i < n_calls; ++i) {
         const AttnCall &call = calls[i];
@@ -215,7 +270,6 @@ int build_attn_params(const AttnCall *calls, int n_calls, ll::AttnParams *p)
         if (ng + call.n_groups > ll::kMaxGroups) return fail(LL_ERR_UNSUPPORTED_SHAPE, "more than %d query groups", ll::kMaxGroups);
         const int rows_per_group = c->C * c->P;
         const int tiles = (rows_per_group + ll::kQTileRows - 1) / ll::kQTileRows;
-        const long long cols = (long long)c->H * tiles;
         p->item[i].out = call.out;
         p->item[i].lse = call.lse;
         p->item[i].nq_total = call.n_groups * rows_per_group;
@@ -236,20 +290,15 @@ int build_attn_params(const AttnCall *calls, int n_calls, ll::AttnParams *p)
                 G.k_len[r] = (int)lens[r];
                 G.n_kt += (int)((lens[r] + ll::kKeyTile - 1) / ll::kKeyTile);
             }
-            G.wave_cols = cols >= sms ? (int)(cols / sms * sms) : 0;
-            waves |= G.wave_cols > 0;
-            G.step_begin = steps;
-            steps += (cols - G.wave_cols) * G.n_kt;
-            all_steps += cols * G.n_kt;
+            G.col_begin = (int)all_cols;
+            all_cols += (long long)c->H * tiles;
+            all_steps += (long long)c->H * tiles * G.n_kt;
         }
     }
+    if (all_steps > INT32_MAX) return fail(LL_ERR_UNSUPPORTED_SHAPE, "too much work for one launch");
     p->n_groups = ng;
     p->nq_total = p->item[0].nq_total;
-    p->total_steps = steps;
-    p->n_ctas = waves ? sms : (int)std::min<long long>(sms, all_steps);
-    // with fewer shared steps than CTAs only the first CTAs take one each, so that the parts
-    // of a split column always sit in consecutive CTAs
-    p->share_ctas = (int)std::max<long long>(1, std::min<long long>(p->n_ctas, steps));
+    plan_work(p, sms, all_cols, all_steps);
     return LL_OK;
 }
 
@@ -545,10 +594,55 @@ int ll_recache(ll_cache *c, int layer, const ll_bf16 *q, const ll_bf16 *k, const
     return LL_OK;
 }
 
+namespace {
+void copy_plan(const ll::AttnParams &p, ll_attn_plan *out)
+{
+    memset(out, 0, sizeof *out);
+    out->n_ctas = p.n_ctas;
+    out->n_groups = p.n_groups;
+    out->heads = p.heads;
+    out->n_waves = p.n_waves;
+    out->n_shares = p.n_shares;
+    out->shared_steps = p.total_steps;
+    for (int k = 0; k <= p.n_shares; ++k) out->share_begin[k] = p.share_begin[k];
+    for (int i = 0; i < p.n_ctas; ++i) out->share_of_cta[i] = p.share_of_cta[i];
+    for (int g = 0; g < p.n_groups; ++g) {
+        out->tiles[g] = p.g[g].tiles;
+        out->n_kt[g] = p.g[g].n_kt;
+        out->col_begin[g] = p.g[g].col_begin;
+        out->wave_cols[g] = p.g[g].wave_cols;
+        out->step_begin[g] = p.g[g].step_begin;
+    }
+}
+}  // namespace
+
+int ll_debug_attn_plan_batched(const ll_attn_item *items, int n_items, int sm_count, ll_attn_plan *out)
+{
+    if (!items || !out || n_items < 1 || n_items > LL_MAX_BATCH)
+        return fail(LL_ERR_INVALID_ARG, "bad argument to ll_debug_attn_plan_batched");
+    AttnCall calls[ll::kMaxItems];
+    for (int i = 0; i < n_items; ++i) {
+        const ll_attn_item &it = items[i];
+        if (!layer_ok(it.cache, it.layer)) return fail(LL_ERR_INVALID_ARG, "bad cache handle or layer in item %d", i);
+        const ll::LayerState &st = it.cache->layers[it.layer];
+        if (st.end < it.cache->C) return fail(LL_ERR_BAD_POSITION, "no chunk has been appended yet");
+        calls[i] = AttnCall{it.cache, it.layer, nullptr, nullptr, nullptr, 1, {st.end - it.cache->C}, 0};
+    }
+    ll_cache *c0 = items[0].cache;
+    const int saved = c0->sm_count;
+    if (sm_count > 0) c0->sm_count = sm_count;
+    ll::AttnParams p;
+    const int s = build_attn_params(calls, n_items, &p);
+    c0->sm_count = saved;
+    if (s != LL_OK) return s;
+    copy_plan(p, out);
+    return LL_OK;
+}
+
 int ll_debug_attn_plan(ll_cache *c, int layer, int recache, int sm_count, ll_attn_plan *out)
 {
     if (!layer_ok(c, layer) || !out) return fail(LL_ERR_INVALID_ARG, "bad argument to ll_debug_attn_plan");
-    static_assert(LL_MAX_GROUPS == ll::kMaxGroups, "header and kernel disagree on the group limit");
+    static_assert(LL_MAX_GROUPS == ll::kMaxGroups && LL_MAX_CTAS == ll::kMaxCtas, "header and kernel disagree on a limit");
     const ll::LayerState &st = c->layers[layer];
     int n_groups = 1;
     int64_t gstart[ll::kMaxGroups];
@@ -572,17 +666,7 @@ int ll_debug_attn_plan(ll_cache *c, int layer, int recache, int sm_count, ll_att
     const int s = build_attn_params(&call, 1, &p);
     c->sm_count = saved;
     if (s != LL_OK) return s;
-    out->n_ctas = p.n_ctas;
-    out->n_groups = p.n_groups;
-    out->heads = p.heads;
-    out->share_ctas = p.share_ctas;
-    out->shared_steps = p.total_steps;
-    for (int g = 0; g < p.n_groups; ++g) {
-        out->tiles[g] = p.g[g].tiles;
-        out->n_kt[g] = p.g[g].n_kt;
-        out->wave_cols[g] = p.g[g].wave_cols;
-        out->step_begin[g] = p.g[g].step_begin;
-    }
+    copy_plan(p, out);
     return LL_OK;
 }
 

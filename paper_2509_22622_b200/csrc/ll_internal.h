@@ -36,18 +36,21 @@ struct LayerState {
 
 // One group of query rows that share a visible key set.  The group's work is
 // heads x tiles columns (a column = kQTileRows query rows of one head, numbered
-// head-major), each n_kt steps long (a step = one kKeyTile-key tile).  The first
-// wave_cols columns (a multiple of the CTA count) are handed out whole, CTA i
-// taking columns i, i + n_ctas, ...; the steps of the remaining columns are
-// laid end to end after those of earlier groups' remainders and cut into equal
-// shares.
+// head-major), each n_kt steps long (a step = one kKeyTile-key tile).  The
+// columns of all groups of a launch are numbered through, group after group;
+// the first n_waves * n_ctas of them are handed out whole, CTA i taking columns
+// i, i + n_ctas, ..., and the steps of the columns left over are laid end to
+// end and cut into one share per CTA, sized so that every CTA ends up with the
+// same number of steps (whole columns of groups with different key counts
+// weigh differently).
 struct AttnGroup {
     int item;                         // which (cache, layer, q, out) of the launch the group belongs to
     int q_begin;                      // first query row of the group in its item's q tensor
     int q_rows;                       // rows in the group
     int tiles;                        // query tiles of kQTileRows rows
     int n_kt;                         // key tiles (steps) per column
-    int wave_cols;                    // columns handed out whole
+    int col_begin;                    // launch-wide number of the group's first column
+    int wave_cols;                    // the group's first wave_cols columns are handed out whole
     long long step_begin;             // shared steps of all earlier groups
     int n_ranges;
     int k_start[LL_MAX_RANGES];       // visible cache-row runs
@@ -76,8 +79,9 @@ struct AttnParams {
     int heads;
     int nq_total;                     // rows of q / out of item 0 (the triage kernel serves one item)
     int n_ctas;                       // grid.x: persistent CTAs
-    int share_ctas;                   // the first share_ctas CTAs take a share of the shared steps (each >= 1 step)
-    long long total_steps;            // shared steps of all groups (cut evenly across those CTAs)
+    int n_waves;                      // whole-column waves
+    int n_shares;                     // non-empty shares of the shared steps
+    long long total_steps;            // shared steps of all groups
     int64_t rows_per_head;            // (S+W)*P
     float scale_log2;                 // log2(e) / sqrt(D)
     const ll_bf16 *q;                 // [nq_total, H, D]
@@ -86,10 +90,12 @@ struct AttnParams {
     const ll_bf16 *kbase;             // layer K: [H][rows][D]
     const ll_bf16 *vbase;             // layer V
     uint32_t *status;                 // aux status words
-    float *partial;                   // 2 * kMaxCtas slots of attn_slot_bytes
-    uint32_t *counters;               // kMaxCtas * kSlabs arrival counters, zero between launches
+    float *partial;                   // 2 * kMaxCtas slots of attn_slot_bytes (two per share)
+    uint32_t *counters;               // kMaxCtas * kSlabs arrival counters (per share), zero between launches
     AttnItem item[kMaxItems];
     AttnGroup g[kMaxGroups];
+    int share_begin[kMaxCtas + 1];    // share k = shared steps [share_begin[k], share_begin[k + 1]), k < n_shares
+    short share_of_cta[kMaxCtas];     // the share a CTA takes, -1 for none; shares go to CTAs in rising order
 };
 
 struct RopeAppendParams {

@@ -138,7 +138,7 @@ def test_split_column_with_fewer_shared_steps_than_ctas(oracle_mod):
     cache.check_device()
     plan = B.ll_debug_attn_plan(cache.h)
     if plan.n_ctas == 148:
-        assert plan.wave_cols[0] == 148 and plan.shared_steps == 58 and plan.share_ctas == 58
+        assert plan.wave_cols[0] == 148 and plan.shared_steps == 58 and plan.n_shares == 58
     assert torch.isfinite(out.float()).all()
     orc.append(0, F64(k), F64(v), 0, wl.grid_h, wl.grid_w, wl.rope_theta)
     qr = orc.rope_q(F64(q), 0, wl.grid_h, wl.grid_w, wl.rope_theta)

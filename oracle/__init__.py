@@ -79,6 +79,10 @@ def lib():
             L.llo_recache.argtypes = [C.c_void_p, C.c_int] + [C.POINTER(C.c_double)] * 3 + \
                                      [C.c_int, C.c_int, C.c_int, C.c_double, C.POINTER(C.c_int64), C.c_int64] + \
                                      [C.POINTER(C.c_double)] * 3
+            L.llo_visible_window.argtypes = [C.c_void_p, C.c_int64, C.c_int64, C.c_int]
+            L.llo_clip.argtypes = [C.c_void_p, C.c_int] + [C.POINTER(C.c_double)] * 3 + \
+                                  [C.c_int64, C.c_int, C.c_int, C.c_int, C.c_int, C.c_double,
+                                   C.POINTER(C.c_int64), C.c_int64] + [C.POINTER(C.c_double)] * 3
             L.llo_read_row.argtypes = [C.c_void_p, C.c_int, C.c_int64,
                                        C.POINTER(C.c_double), C.POINTER(C.c_double)]
             L.llo_read_layer.argtypes = [C.c_void_p, C.c_int, C.POINTER(C.c_double), C.POINTER(C.c_double)]
@@ -223,6 +227,26 @@ class Oracle:
         if st != OK:
             raise OracleError(st, "recache")
         return qr, out, lse
+
+    def clip(self, layer, q, k, v, frame_start, n_frames, window, gh, gw, theta=10000.0, rows=None):
+        """A clip of whole chunks appended and attended in one step under a local window of
+        ``window`` frames (Sec. 3.3, training/inference consistency).  Returns (q_roped, out, lse)."""
+        q, k, v = _f64(q), _f64(k), _f64(v)
+        if q.shape != (n_frames * gh * gw, self.H, self.D) or k.shape != q.shape or v.shape != q.shape:
+            raise OracleError(ERR_ARG, "clip shape")
+        r = None if rows is None else np.ascontiguousarray(rows, dtype=np.int64)
+        n_rows = q.shape[0] if r is None else r.shape[0]
+        qr = np.empty_like(q)
+        out = np.empty((n_rows, self.H, self.D), dtype=np.float64)
+        lse = np.empty((n_rows, self.H), dtype=np.float64)
+        st = lib().llo_clip(self._h, layer, _dp(q), _dp(k), _dp(v), frame_start, n_frames, window, gh, gw,
+                            theta, _ip(r), n_rows, _dp(qr), _dp(out), _dp(lse))
+        if st != OK:
+            raise OracleError(st, "clip")
+        return qr, out, lse
+
+    def visible_window(self, fq: int, fk: int, window: int) -> bool:
+        return bool(lib().llo_visible_window(self._h, fq, fk, window))
 
     # -- storage ------------------------------------------------------------
     def read_row(self, layer, cache_row):

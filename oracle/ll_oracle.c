@@ -15,6 +15,11 @@
  *     cache is rebuilt from the most recent W generated frames only.
  *   - Algorithm 2 (interactive inference): every denoising pass of a chunk
  *     attends over the cache; the final clean pass commits the chunk's K/V.
+ *   - Sec. 3.3 "Consistency between Training and Inference": a supervised clip
+ *     of T frames is processed in one step over a resident cache of the S sink
+ *     frames, the last W_a frames of the preceding context and the clip's own
+ *     T frames, under the same sink + local-window rule (llo_clip; forward
+ *     only, gradients are not this library's business).
  *
  * Readings where the paper is silent (the benchmark definition fixes them):
  *   - W counts the current chunk ("9 local + 3 sink = effective window 12").
@@ -234,12 +239,24 @@ int llo_append(llo *o, int layer, const double *k, const double *v,
  * and it is either a sink frame or inside the W-frame window that ends with the
  * query's chunk.  lo_floor additionally hides non-sink frames older than it
  * (recache: frames that no longer exist). */
-int llo_visible(const llo *o, int64_t fq, int64_t fk, int64_t lo_floor)
+static int visible_in_window(const llo *o, int64_t fq, int64_t fk, int64_t lo_floor, int window)
 {
     int64_t hi = (fq / o->C + 1) * o->C;      /* one past the query's chunk */
     if (fk < 0 || fk >= hi) return 0;
     if (fk < o->S) return 1;
-    return fk >= hi - o->W && fk >= lo_floor;
+    return fk >= hi - window && fk >= lo_floor;
+}
+
+int llo_visible(const llo *o, int64_t fq, int64_t fk, int64_t lo_floor)
+{
+    return visible_in_window(o, fq, fk, lo_floor, o->W);
+}
+
+/* The same with a local window of `window` frames that may be shorter than the
+ * resident ring (the clip step below). */
+int llo_visible_window(const llo *o, int64_t fq, int64_t fk, int window)
+{
+    return visible_in_window(o, fq, fk, 0, window);
 }
 
 /* ---- step: attention ------------------------------------------------------ */
@@ -249,9 +266,9 @@ int llo_visible(const llo *o, int64_t fq, int64_t fk, int64_t lo_floor)
  *   rows[n_rows]                 : query row indices to evaluate (NULL = all)
  *   out [n_rows, H, D], lse [n_rows, H] (natural log of the softmax denominator)
  * Per row and head: s_j = q.k_j / sqrt(D), p = softmax(s), o = sum p_j v_j. */
-int llo_attn(const llo *o, int layer, const double *q_roped, int64_t q_frame_start,
-             int n_q_frames, int64_t lo_floor, const int64_t *rows, int64_t n_rows,
-             double *out, double *lse)
+static int attn_in_window(const llo *o, int layer, const double *q_roped, int64_t q_frame_start,
+                          int n_q_frames, int64_t lo_floor, int window, const int64_t *rows, int64_t n_rows,
+                          double *out, double *lse)
 {
     if (!o || layer < 0 || layer >= o->L || !q_roped || !out) return LLO_ERR_ARG;
     int64_t nq = (int64_t)n_q_frames * o->P;
@@ -273,7 +290,7 @@ int llo_attn(const llo *o, int layer, const double *q_roped, int64_t q_frame_sta
         int nvis = 0;
         int *vslot = (int *)malloc(sizeof(int) * (size_t)(o->S + o->W));
         for (int64_t fk = 0; fk < hi; ++fk) {
-            if (!llo_visible(o, fq, fk, lo_floor)) continue;
+            if (!visible_in_window(o, fq, fk, lo_floor, window)) continue;
             int slot = llo_slot_of(o, fk);
             if (sf[slot] != (int32_t)fk || nvis >= o->S + o->W) { status = LLO_ERR_NOT_RESIDENT; nvis = -1; break; }
             vslot[nvis++] = slot;
@@ -308,6 +325,14 @@ int llo_attn(const llo *o, int layer, const double *q_roped, int64_t q_frame_sta
         free(s); free(vslot);
     }
     return status;
+}
+
+int llo_attn(const llo *o, int layer, const double *q_roped, int64_t q_frame_start,
+             int n_q_frames, int64_t lo_floor, const int64_t *rows, int64_t n_rows,
+             double *out, double *lse)
+{
+    if (!o) return LLO_ERR_ARG;
+    return attn_in_window(o, layer, q_roped, q_frame_start, n_q_frames, lo_floor, o->W, rows, n_rows, out, lse);
 }
 
 /* Softmax probabilities of one (row, head) and the cache rows they belong to;
@@ -390,6 +415,37 @@ int llo_recache(llo *o, int layer, const double *q, const double *k, const doubl
     double *qr = q_roped_out ? q_roped_out : (double *)malloc(sizeof(double) * (size_t)nq * re);
     llo_rope(q, qr, nq, o->H, o->D, r0, gh, gw, theta, o->faithful);
     int st = llo_attn(o, layer, qr, r0, n_frames, r0, rows, n_rows, out, lse);
+    if (!q_roped_out) free(qr);
+    return st;
+}
+
+/* ---- step: a clip in one go (Sec. 3.3, "Consistency between Training and Inference") ---- */
+
+/* The clip's n_frames frames (whole chunks, starting at the stream's end) enter
+ * the cache chunk after chunk exactly as in llo_append; then every clip frame's
+ * queries attend over the sink frames and the local window of `window` frames
+ * that ends with their own chunk: the tail of the preceding context and the
+ * clip's earlier chunks.  The ring must be long enough that the first chunk's
+ * window is still resident once the last chunk is in:
+ * W >= window + n_frames - C.  q_roped_out (nullable) receives the roped queries. */
+int llo_clip(llo *o, int layer, const double *q, const double *k, const double *v,
+             int64_t frame_start, int n_frames, int window, int gh, int gw, double theta,
+             const int64_t *rows, int64_t n_rows, double *q_roped_out, double *out, double *lse)
+{
+    if (!o || layer < 0 || layer >= o->L || !q || !k || !v || !out) return LLO_ERR_ARG;
+    if (gh * gw != o->P || n_frames <= 0 || n_frames % o->C) return LLO_ERR_ARG;
+    if (window < o->C || window % o->C || window + n_frames - o->C > o->W) return LLO_ERR_ARG;
+    if (frame_start != o->end[layer]) return LLO_ERR_POSITION;
+    size_t chunk_elems = (size_t)o->C * o->P * row_elems(o);
+    for (int c = 0; c < n_frames / o->C; ++c) {
+        int st = llo_append(o, layer, k + (size_t)c * chunk_elems, v + (size_t)c * chunk_elems,
+                            frame_start + (int64_t)c * o->C, o->C, gh, gw, theta);
+        if (st != LLO_OK) return st;
+    }
+    int64_t nq = (int64_t)n_frames * o->P;
+    double *qr = q_roped_out ? q_roped_out : (double *)malloc(sizeof(double) * (size_t)nq * row_elems(o));
+    llo_rope(q, qr, nq, o->H, o->D, frame_start, gh, gw, theta, o->faithful);
+    int st = attn_in_window(o, layer, qr, frame_start, n_frames, 0, window, rows, n_rows, out, lse);
     if (!q_roped_out) free(qr);
     return st;
 }

@@ -470,3 +470,90 @@ def test_seek_equals_full_replay(oracle_mod):
     assert list(short.state()["slot_frame"]) == list(full.state()["slot_frame"])
     with pytest.raises(oracle_mod.OracleError):
         short.seek(0, 4)                                        # cannot go back
+
+
+# ---------------------------------------------------------------------------
+# a clip in one step (Sec. 3.3, "Consistency between Training and Inference")
+# ---------------------------------------------------------------------------
+
+def clip_flat_reference(oracle_mod, hist_q, hist_k, hist_v, first_clip_chunk, C, S, window, gh, gw):
+    """Library-softmax attention of the clip's queries over the frames Sec. 3.3 keeps for them,
+    written from the text: the sink frames, and of all other frames up to the query's own chunk
+    the last `window` ones.  hist_* hold every chunk of the stream so far, raw."""
+    P = gh * gw
+    D = hist_q[0].shape[-1]
+    keys = np.concatenate([oracle_mod.rope(k, c * C, gh, gw) for c, k in enumerate(hist_k)])
+    vals = np.concatenate(hist_v)
+    outs, lses = [], []
+    for c in range(first_clip_chunk, len(hist_q)):
+        upto = list(range((c + 1) * C))
+        frames = [f for f in upto if f < S] + [f for f in upto[-window:] if f >= S]
+        idx = np.concatenate([np.arange(f * P, (f + 1) * P) for f in frames])
+        qr = oracle_mod.rope(hist_q[c], c * C, gh, gw)
+        s = np.einsum("qhd,khd->hqk", qr, keys[idx]) / np.sqrt(D)
+        outs.append(np.einsum("hqk,khd->qhd", softmax(s, axis=-1), vals[idx]))
+        lses.append(logsumexp(s, axis=-1).T)
+    return np.concatenate(outs), np.concatenate(lses)
+
+
+@pytest.mark.parametrize("C,S,window,clip_chunks,before", [(1, 1, 2, 3, 4), (2, 2, 4, 2, 3), (1, 0, 1, 4, 2),
+                                                            (2, 2, 2, 3, 0), (1, 2, 3, 2, 1)])
+def test_clip_equals_flat_attention_over_sink_context_tail_and_clip(oracle_mod, C, S, window, clip_chunks, before):
+    gh, gw, H, D = 2, 3, 2, 16
+    P = gh * gw
+    T = clip_chunks * C
+    ring = window + T - C                      # resident set of S + (window - C) + T frames: O(W + T + S)
+    o = oracle_mod.Oracle(1, H, D, P, C, S, ring)
+    hq, hk, hv = [], [], []
+    for c in range(before + clip_chunks):
+        q, k, v = (rand((C * P, H, D), 1000 + 10 * c + i) for i in range(3))
+        hq.append(q); hk.append(k); hv.append(v)
+        if c < before:
+            o.append(0, k, v, c * C, gh, gw)
+    q, k, v = (np.concatenate(h[before:]) for h in (hq, hk, hv))
+    qr, out, lse = o.clip(0, q, k, v, before * C, T, window, gh, gw)
+    want, want_lse = clip_flat_reference(oracle_mod, hq, hk, hv, before, C, S, window, gh, gw)
+    np.testing.assert_allclose(out, want, rtol=0, atol=1e-12)
+    np.testing.assert_allclose(lse, want_lse, rtol=0, atol=1e-12)
+    np.testing.assert_array_equal(qr, oracle_mod.rope(q, before * C, gh, gw))
+    assert o.state()["end"] == (before + clip_chunks) * C
+
+
+def test_clip_equals_chunk_by_chunk_decoding_with_that_window(oracle_mod):
+    """Train/inference consistency itself: the clip step gives every chunk exactly what
+    streaming inference with a ring of `window` frames gives it."""
+    C, S, window, gh, gw, H, D = 2, 2, 4, 2, 2, 2, 16
+    P = gh * gw
+    clip_chunks, before = 4, 5
+    T = clip_chunks * C
+    big = oracle_mod.Oracle(1, H, D, P, C, S, window + T - C)
+    small = oracle_mod.Oracle(1, H, D, P, C, S, window)
+    outs = []
+    data = [[rand((C * P, H, D), 2000 + 10 * c + i) for i in range(3)] for c in range(before + clip_chunks)]
+    for c, (q, k, v) in enumerate(data):
+        small.append(0, k, v, c * C, gh, gw)
+        if c < before:
+            big.append(0, k, v, c * C, gh, gw)
+        else:
+            outs.append(small.attn(0, small.rope_q(q, c * C, gh, gw), c * C))
+    q, k, v = (np.concatenate([d[i] for d in data[before:]]) for i in range(3))
+    _, out, lse = big.clip(0, q, k, v, before * C, T, window, gh, gw)
+    np.testing.assert_allclose(out, np.concatenate([x[0] for x in outs]), rtol=0, atol=1e-13)
+    np.testing.assert_allclose(lse, np.concatenate([x[1] for x in outs]), rtol=0, atol=1e-13)
+    # a longer window than the one asked for would see more: the result really depends on it
+    big2 = oracle_mod.Oracle(1, H, D, P, C, S, window + T - C)
+    for c in range(before):
+        big2.append(0, data[c][1], data[c][2], c * C, gh, gw)
+    _, out2, _ = big2.clip(0, q, k, v, before * C, T, window - C, gh, gw)
+    assert np.abs(out2 - out).max() > 1e-6
+
+
+def test_clip_rejects_a_ring_too_short_for_it(oracle_mod):
+    C, S, window = 1, 1, 3
+    o = oracle_mod.Oracle(1, 1, 8, 1, C, S, 4)
+    x = rand((3, 1, 8), 5)
+    with pytest.raises(oracle_mod.OracleError):
+        o.clip(0, x, x, x, 0, 3, window, 1, 1)          # needs 3 + 3 - 1 = 5 ring frames
+    o.clip(0, x[:2], x[:2], x[:2], 0, 2, window, 1, 1)  # 3 + 2 - 1 = 4 fits
+    with pytest.raises(oracle_mod.OracleError):
+        o.clip(0, x[:2], x[:2], x[:2], 0, 2, window, 1, 1)   # not at the stream's end any more

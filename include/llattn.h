@@ -162,6 +162,31 @@ typedef struct ll_attn_item {
 } ll_attn_item;
 int ll_sink_window_attn_batched(const ll_attn_item *items, int n_items, ll_stream stream);
 
+/* A clip of several chunks in one step (Sec. 3.3 "Consistency between Training
+ * and Inference": the resident cache is the S sink frames, the last frames of
+ * the preceding context and the T frames of the current clip, attended under
+ * the same sink + local-window rule as at inference; also the way to prefill a
+ * stream from an existing video).  Forward only.
+ *   q, k, v             [n_frames*tokens_per_frame, heads, head_dim], raw
+ *   frame_start         must equal end; n_frames a positive multiple of
+ *                       chunk_frames, at most 24 chunks
+ *   attn_window_frames  W_a, the local window a chunk attends over (counts the
+ *                       chunk itself), a multiple of chunk_frames.  The ring
+ *                       must hold the first chunk's window until the last chunk
+ *                       is in: window_frames >= W_a + n_frames - chunk_frames,
+ *                       else LL_ERR_UNSUPPORTED_SHAPE.
+ * Appends all n_frames (RoPE on K, slots and eviction as n_frames/chunk_frames
+ * calls of ll_rope_append_kv would), writes RoPE(q) to q_out, then attends: a
+ * query of the chunk ending at frame e sees the sink frames below e and the
+ * frames [max(S, e - W_a), e).  Every chunk gets what chunk-by-chunk decoding
+ * on a cache with window_frames = W_a would give it.  out/lse_out as for
+ * ll_sink_window_attn with n_frames*tokens_per_frame rows.  On error nothing is
+ * launched and no state changes. */
+int ll_clip_append_attn(ll_cache *cache, int layer, const ll_bf16 *q, const ll_bf16 *k,
+                        const ll_bf16 *v, int64_t frame_start, int n_frames,
+                        int attn_window_frames, int grid_h, int grid_w, float rope_theta,
+                        ll_bf16 *q_out, ll_bf16 *out, float *lse_out, ll_stream stream);
+
 /* KV-recache (Sec. 3.1; Sec. 3.3 last paragraph: only the most recent W frames
  * are rebuilt; the sink is left alone).  q, k, v hold fresh activations for the
  * resident window frames [r0, end), r0 = max(S, end - W), oldest first.

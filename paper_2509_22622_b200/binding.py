@@ -98,6 +98,9 @@ SIGNATURES = {
     "ll_sink_window_attn": (C.c_int, [C.c_void_p, C.c_int, C.c_void_p, C.c_int64, C.c_int, C.c_void_p,
                                       C.c_void_p, C.c_void_p]),
     "ll_sink_window_attn_batched": (C.c_int, [C.POINTER(ll_attn_item), C.c_int, C.c_void_p]),
+    "ll_clip_append_attn": (C.c_int, [C.c_void_p, C.c_int, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int64, C.c_int,
+                                      C.c_int, C.c_int, C.c_int, C.c_float, C.c_void_p, C.c_void_p, C.c_void_p,
+                                      C.c_void_p]),
     "ll_recache": (C.c_int, [C.c_void_p, C.c_int, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int, C.c_int,
                              C.c_int, C.c_float, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]),
     "ll_rope_q_static": (C.c_int, [C.c_void_p, C.c_void_p, C.c_int, C.c_int, C.c_int64, C.c_int, C.c_int, C.c_int,
@@ -208,6 +211,13 @@ def ll_sink_window_attn_batched(items, stream=None):
 def ll_debug_attn_simt(h, layer, q_roped, q_frame_start, n_q_frames, out, lse_out=None, stream=None):
     _check(lib().ll_debug_attn_simt(h, layer, _ptr(q_roped), q_frame_start, n_q_frames, _ptr(out),
                                     _ptr(lse_out), _stream(stream)))
+
+
+def ll_clip_append_attn(h, layer, q, k, v, frame_start, n_frames, attn_window_frames, grid_h, grid_w,
+                        rope_theta, q_out, out, lse_out=None, stream=None):
+    _check(lib().ll_clip_append_attn(h, layer, _ptr(q), _ptr(k), _ptr(v), frame_start, n_frames, attn_window_frames,
+                                     grid_h, grid_w, rope_theta, _ptr(q_out), _ptr(out), _ptr(lse_out),
+                                     _stream(stream)))
 
 
 def ll_recache(h, layer, q, k, v, n_frames, grid_h, grid_w, rope_theta, q_out, out, lse_out=None, stream=None):
@@ -341,6 +351,11 @@ class Cache:
         """items: (Cache, layer, q_roped, q_frame_start, out, lse_out or None) per stream, one launch."""
         ll_sink_window_attn_batched([(c.h, layer, q, f0, c.C, out, lse) for c, layer, q, f0, out, lse in items],
                                     stream)
+
+    def clip_append_attn(self, layer, q, k, v, frame_start, n_frames, attn_window_frames, grid_h, grid_w, theta,
+                         q_out, out, lse_out=None, stream=None):
+        ll_clip_append_attn(self.h, layer, q, k, v, frame_start, n_frames, attn_window_frames, grid_h, grid_w,
+                            theta, q_out, out, lse_out, stream)
 
     def recache(self, layer, q, k, v, n_frames, grid_h, grid_w, theta, q_out, out, lse_out=None, stream=None):
         ll_recache(self.h, layer, q, k, v, n_frames, grid_h, grid_w, theta, q_out, out, lse_out, stream)

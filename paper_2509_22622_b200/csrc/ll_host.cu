@@ -179,7 +179,8 @@ struct AttnCall {
     float *lse;
     int n_groups;
     int64_t group_frame_start[ll::kMaxGroups];
-    int64_t lo_floor;
+    int64_t lo_floor;                             // non-sink frames older than this are hidden from every group ...
+    int64_t group_lo_floor[ll::kMaxGroups];       // ... and from group g those older than this (0: no extra limit)
 };
 
 // Divide the columns of all groups between the CTAs (one persistent CTA per SM).  The
@@ -281,7 +282,7 @@ int build_attn_params(const AttnCall *calls, int n_calls, ll::AttnParams *p)
             G.tiles = tiles;
             int64_t starts[LL_MAX_RANGES], lens[LL_MAX_RANGES];
             int n = 0;
-            int st = visible_ranges(c, call.layer, call.group_frame_start[g], call.lo_floor, starts, lens, &n);
+            int st = visible_ranges(c, call.layer, call.group_frame_start[g], std::max(call.lo_floor, call.group_lo_floor[g]), starts, lens, &n);
             if (st != LL_OK) return st;
             G.n_ranges = n;
             G.n_kt = 0;
@@ -591,6 +592,73 @@ int ll_recache(ll_cache *c, int layer, const ll_bf16 *q, const ll_bf16 *k, const
         if (s != LL_OK) return s;
     }
     st.n_recaches += 1;
+    return LL_OK;
+}
+
+int ll_clip_append_attn(ll_cache *c, int layer, const ll_bf16 *q, const ll_bf16 *k, const ll_bf16 *v,
+                        int64_t frame_start, int n_frames, int attn_window_frames, int grid_h, int grid_w,
+                        float rope_theta, ll_bf16 *q_out, ll_bf16 *out, float *lse_out, ll_stream stream)
+{
+    if (!layer_ok(c, layer)) return fail(LL_ERR_INVALID_ARG, "bad cache handle or layer %d", layer);
+    if (grid_h <= 0 || grid_w <= 0 || (int64_t)grid_h * grid_w != c->P)
+        return fail(LL_ERR_INVALID_ARG, "grid %dx%d does not give %d tokens per frame", grid_h, grid_w, c->P);
+    if (!(rope_theta > 0.f)) return fail(LL_ERR_INVALID_ARG, "rope_theta must be positive");
+    if (n_frames <= 0 || n_frames % c->C)
+        return fail(LL_ERR_BAD_POSITION, "n_frames %d is not a positive multiple of chunk_frames %d", n_frames, c->C);
+    const int n_groups = n_frames / c->C;
+    if (n_groups > ll::kMaxGroups) return fail(LL_ERR_UNSUPPORTED_SHAPE, "more than %d chunks in a clip", ll::kMaxGroups);
+    if (attn_window_frames < c->C || attn_window_frames % c->C)
+        return fail(LL_ERR_INVALID_ARG, "attn_window_frames %d is not a positive multiple of chunk_frames", attn_window_frames);
+    if ((int64_t)attn_window_frames + n_frames - c->C > c->W)
+        return fail(LL_ERR_UNSUPPORTED_SHAPE,
+                    "the ring (%d frames) is shorter than attn_window_frames + n_frames - chunk_frames = %lld: the first "
+                    "chunk's window would be evicted before it is read",
+                    c->W, (long long)attn_window_frames + n_frames - c->C);
+    ll::LayerState &st = c->layers[layer];
+    if (frame_start != st.end)
+        return fail(LL_ERR_BAD_POSITION, "frame_start %lld is not the end of the stream (%lld)", (long long)frame_start,
+                    (long long)st.end);
+    if (frame_start + n_frames > INT32_MAX) return fail(LL_ERR_BAD_POSITION, "frame index exceeds int32");
+    if (!c->dry_run) {
+        if (!q || !k || !v || !q_out || !out) return fail(LL_ERR_INVALID_ARG, "null q/k/v/q_out/out");
+        if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(q_out) || !aligned16(out) ||
+            (lse_out && !aligned16(lse_out)))
+            return fail(LL_ERR_INVALID_ARG, "pointers must be 16-byte aligned");
+        int s = need_storage(c);
+        if (s != LL_OK) return s;
+    }
+    // the clip's frames take their slots first (the plan below reads the slot table); undone on error
+    const ll::LayerState saved = st;
+    for (int i = 0; i < n_frames; ++i) {
+        const int64_t f = frame_start + i;
+        const int slot = slot_of(c, f);
+        if (st.slot_frame[slot] >= 0 && st.slot_frame[slot] != (int32_t)f) st.n_evictions += 1;
+        st.slot_frame[slot] = (int32_t)f;
+    }
+    st.end += n_frames;
+    st.n_appends += n_groups;
+    AttnCall call{c, layer, q_out, out, lse_out, n_groups, {}, 0, {}};
+    for (int g = 0; g < n_groups; ++g) {
+        call.group_frame_start[g] = frame_start + (int64_t)g * c->C;
+        call.group_lo_floor[g] = call.group_frame_start[g] + c->C - attn_window_frames;
+    }
+    ll::AttnParams ap;
+    int s = build_attn_params(&call, 1, &ap);
+    if (s == LL_OK && !c->dry_run) {
+        s = ensure_tables(c, frame_start, frame_start + n_frames, grid_h, grid_w, rope_theta, (cudaStream_t)stream);
+        if (s == LL_OK) {
+            ll::RopeAppendParams rp;
+            fill_rope_params(c, layer, q, k, v, q_out, frame_start, n_frames, grid_w, &rp);
+            cudaError_t e = ll::launch_rope_append(rp, c->D, (cudaStream_t)stream);
+            if (e != cudaSuccess) s = cuda_fail(e, "rope+append kernel (clip)");
+        }
+        if (s == LL_OK) s = launch_attention(&call, 1, ap, (cudaStream_t)stream, false);
+    }
+    if (s != LL_OK) {
+        st = saved;
+        return s;
+    }
+    st.n_attn += 1;
     return LL_OK;
 }
 

@@ -211,3 +211,37 @@ def test_batched_attention_checks_every_item_before_anything_changes():
         B.ll_sink_window_attn_batched([item(c) for c in many])
     assert e.value.code == B.LL_ERR_UNSUPPORTED_SHAPE
     assert [c.state()["attn_calls"] for c in many] == [1] * B.LL_MAX_BATCH + [0]
+
+
+def test_clip_step_bookkeeping_matches_the_oracle_and_errors_change_nothing(oracle_mod):
+    C, S, Wa, T = 2, 2, 4, 6
+    ring = Wa + T - C
+    c = B.Cache(1, 1, 64, 1, C, S, ring, dry_run=True)
+    o = oracle_mod.Oracle(1, 1, 2, 1, C, S, ring)
+    x = np.zeros((C, 1, 2))
+    for chunk in range(3):
+        B.ll_rope_append_kv(c.h, 0, None, None, None, chunk * C, C, 1, 1)
+        o.append(0, x, x, chunk * C, 1, 1)
+    before = c.state()
+    for args, code in [((6, T + 1, Wa), B.LL_ERR_BAD_POSITION),            # not whole chunks
+                       ((4, T, Wa), B.LL_ERR_BAD_POSITION),                # not at the end of the stream
+                       ((6, T, Wa + C), B.LL_ERR_UNSUPPORTED_SHAPE),       # the ring cannot keep the first window
+                       ((6, T + C, Wa), B.LL_ERR_UNSUPPORTED_SHAPE),
+                       ((6, T, 3), B.LL_ERR_INVALID_ARG)]:                 # window not whole chunks
+        with pytest.raises(B.LLError) as e:
+            B.ll_clip_append_attn(c.h, 0, None, None, None, args[0], args[1], args[2], 1, 1, 10000.0, None, None)
+        assert e.value.code == code, args
+        assert c.state() == before
+    for rep in range(3):                                                   # three clips in a row: the ring wraps
+        f0 = 6 + rep * T
+        B.ll_clip_append_attn(c.h, 0, None, None, None, f0, T, Wa, 1, 1, 10000.0, None, None)
+        xs = np.zeros((T, 1, 2))
+        o.clip(0, xs, xs, xs, f0, T, Wa, 1, 1)
+        st, ost = c.state(), o.state()
+        assert st["end"] == ost["end"] == f0 + T
+        assert st["slot_frame"] == list(ost["slot_frame"]) and st["evictions"] == ost["evictions"]
+    assert c.state()["appends"] == 3 + 3 * (T // C) and c.state()["attn_calls"] == 3
+    # a shorter window than the ring allows is fine, and decoding goes on afterwards
+    B.ll_clip_append_attn(c.h, 0, None, None, None, 24, C, C, 1, 1, 10000.0, None, None)
+    B.ll_rope_append_kv(c.h, 0, None, None, None, 26, C, 1, 1)
+    B.ll_sink_window_attn(c.h, 0, None, 26, C, None)

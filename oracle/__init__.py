@@ -83,6 +83,9 @@ def lib():
             L.llo_clip.argtypes = [C.c_void_p, C.c_int] + [C.POINTER(C.c_double)] * 3 + \
                                   [C.c_int64, C.c_int, C.c_int, C.c_int, C.c_int, C.c_double,
                                    C.POINTER(C.c_int64), C.c_int64] + [C.POINTER(C.c_double)] * 3
+            L.llo_dense_attn.argtypes = [C.POINTER(C.c_double)] * 3 + [C.c_int64, C.c_int64, C.c_int, C.c_int,
+                                                                       C.POINTER(C.c_int64), C.c_int64,
+                                                                       C.POINTER(C.c_double), C.POINTER(C.c_double)]
             L.llo_read_row.argtypes = [C.c_void_p, C.c_int, C.c_int64,
                                        C.POINTER(C.c_double), C.POINTER(C.c_double)]
             L.llo_read_layer.argtypes = [C.c_void_p, C.c_int, C.POINTER(C.c_double), C.POINTER(C.c_double)]
@@ -121,6 +124,23 @@ def rope(x, frame_start: int, gh: int, gw: int, theta: float = 10000.0, round_bf
     if st != OK:
         raise OracleError(st, "rope")
     return out
+
+
+def dense_attn(q, k, v, rows=None):
+    """Plain softmax attention, every query over every key (cross-attention, Sec. 3.1).
+    q [n_q, H, D], k and v [n_k, H, D].  Returns (out [n_rows, H, D], lse [n_rows, H])."""
+    q, k, v = _f64(q), _f64(k), _f64(v)
+    n_q, H, D = q.shape
+    if k.shape != v.shape or k.shape[1:] != (H, D):
+        raise OracleError(ERR_ARG, "dense_attn shape")
+    r = None if rows is None else np.ascontiguousarray(rows, dtype=np.int64)
+    n_rows = n_q if r is None else r.shape[0]
+    out = np.empty((n_rows, H, D), dtype=np.float64)
+    lse = np.empty((n_rows, H), dtype=np.float64)
+    st = lib().llo_dense_attn(_dp(q), _dp(k), _dp(v), n_q, k.shape[0], H, D, _ip(r), n_rows, _dp(out), _dp(lse))
+    if st != OK:
+        raise OracleError(st, "dense_attn")
+    return out, lse
 
 
 class Oracle:

@@ -20,6 +20,10 @@
  *     frames, the last W_a frames of the preceding context and the clip's own
  *     T frames, under the same sink + local-window rule (llo_clip; forward
  *     only, gradients are not this library's business).
+ *   - Sec. 3.1: cross-attention layers alternate with the self-attention layers
+ *     and inject the prompt; the recache re-encodes the prefix under the new
+ *     prompt through them.  Cross-attention is plain softmax attention of the
+ *     video tokens over the prompt tokens, no mask, no RoPE (llo_dense_attn).
  *
  * Readings where the paper is silent (the benchmark definition fixes them):
  *   - W counts the current chunk ("9 local + 3 sink = effective window 12").
@@ -448,6 +452,49 @@ int llo_clip(llo *o, int layer, const double *q, const double *k, const double *
     int st = attn_in_window(o, layer, qr, frame_start, n_frames, 0, window, rows, n_rows, out, lse);
     if (!q_roped_out) free(qr);
     return st;
+}
+
+/* ---- step: dense attention (cross-attention to the prompt, Sec. 3.1) -------- */
+
+/* o = softmax(q k^T / sqrt(D)) v per head; every query sees every key.
+ *   q [n_q, H, D], k and v [n_k, H, D]; rows[n_rows] selects query rows (NULL = all)
+ *   out [n_rows, H, D], lse [n_rows, H] (nullable). */
+int llo_dense_attn(const double *q, const double *k, const double *v, int64_t n_q, int64_t n_k,
+                   int H, int D, const int64_t *rows, int64_t n_rows, double *out, double *lse)
+{
+    if (!q || !k || !v || !out || n_q <= 0 || n_k <= 0 || H <= 0 || D <= 0) return LLO_ERR_ARG;
+    if (!rows) n_rows = n_q;
+    const double scale = 1.0 / sqrt((double)D);
+    int status = LLO_OK;
+#pragma omp parallel for schedule(dynamic, 1)
+    for (int64_t ri = 0; ri < n_rows; ++ri) {
+        int64_t r = rows ? rows[ri] : ri;
+        if (r < 0 || r >= n_q) { status = LLO_ERR_ARG; continue; }
+        double *s = (double *)malloc(sizeof(double) * (size_t)n_k);
+        for (int h = 0; h < H; ++h) {
+            const double *qv = q + ((size_t)r * H + h) * D;
+            double m = -INFINITY;
+            for (int64_t j = 0; j < n_k; ++j) {
+                const double *kv = k + ((size_t)j * H + h) * D;
+                double dot = 0.0;
+                for (int d = 0; d < D; ++d) dot += qv[d] * kv[d];
+                s[j] = dot * scale;
+                if (s[j] > m) m = s[j];
+            }
+            double denom = 0.0;
+            for (int64_t j = 0; j < n_k; ++j) { s[j] = exp(s[j] - m); denom += s[j]; }
+            double *ov = out + ((size_t)ri * H + h) * D;
+            for (int d = 0; d < D; ++d) ov[d] = 0.0;
+            for (int64_t j = 0; j < n_k; ++j) {
+                double pj = s[j] / denom;
+                const double *vv = v + ((size_t)j * H + h) * D;
+                for (int d = 0; d < D; ++d) ov[d] += pj * vv[d];
+            }
+            if (lse) lse[(size_t)ri * H + h] = m + log(denom);
+        }
+        free(s);
+    }
+    return status;
 }
 
 /* Read back one cache row (slot*P + token) of K and V, [H, D] each. */

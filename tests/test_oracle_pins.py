@@ -557,3 +557,40 @@ def test_clip_rejects_a_ring_too_short_for_it(oracle_mod):
     o.clip(0, x[:2], x[:2], x[:2], 0, 2, window, 1, 1)  # 3 + 2 - 1 = 4 fits
     with pytest.raises(oracle_mod.OracleError):
         o.clip(0, x[:2], x[:2], x[:2], 0, 2, window, 1, 1)   # not at the stream's end any more
+
+
+# ---------------------------------------------------------------------------
+# dense attention (cross-attention to the prompt, Sec. 3.1)
+# ---------------------------------------------------------------------------
+
+def test_dense_attention_equals_library_softmax(oracle_mod):
+    q, k, v = rand((37, 3, 16), 1), rand((29, 3, 16), 2), rand((29, 3, 16), 3)
+    out, lse = oracle_mod.dense_attn(q, k, v)
+    s = np.einsum("qhd,khd->hqk", q, k) / np.sqrt(16)
+    np.testing.assert_allclose(out, np.einsum("hqk,khd->qhd", softmax(s, axis=-1), v), rtol=0, atol=1e-12)
+    np.testing.assert_allclose(lse, logsumexp(s, axis=-1).T, rtol=0, atol=1e-12)
+    rows = np.array([36, 0, 5])
+    out_r, lse_r = oracle_mod.dense_attn(q, k, v, rows=rows)
+    np.testing.assert_array_equal(out_r, out[rows])
+    np.testing.assert_array_equal(lse_r, lse[rows])
+
+
+def test_dense_attention_special_cases(oracle_mod):
+    q, k, v = rand((5, 2, 8), 4), rand((1, 2, 8), 5), rand((1, 2, 8), 6)
+    out, lse = oracle_mod.dense_attn(q, k, v)                       # one key: its value, lse = the score
+    np.testing.assert_array_equal(out, np.broadcast_to(v, out.shape))
+    np.testing.assert_allclose(lse, np.einsum("qhd,hd->qh", q, k[0]) / np.sqrt(8), atol=1e-13)
+    k0 = np.zeros((7, 2, 8)); v7 = rand((7, 2, 8), 7)
+    out, lse = oracle_mod.dense_attn(q, k0, v7)                     # equal scores: the mean of the values
+    np.testing.assert_allclose(out, np.broadcast_to(v7.mean(axis=0), out.shape), atol=1e-14)
+    np.testing.assert_allclose(lse, np.log(7.0), atol=1e-14)
+    # permuting the keys (with their values) changes nothing; heads do not mix
+    k9, v9 = rand((9, 2, 8), 8), rand((9, 2, 8), 9)
+    perm = np.random.default_rng(0).permutation(9)
+    a, _ = oracle_mod.dense_attn(q, k9, v9)
+    b, _ = oracle_mod.dense_attn(q, k9[perm], v9[perm])
+    np.testing.assert_allclose(a, b, atol=1e-13)
+    k9b = k9.copy(); k9b[:, 1] += 1.0
+    c, _ = oracle_mod.dense_attn(q, k9b, v9)
+    np.testing.assert_array_equal(a[:, 0], c[:, 0])
+    assert np.abs(a[:, 1] - c[:, 1]).max() > 1e-6

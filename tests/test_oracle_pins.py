@@ -590,7 +590,7 @@ def test_dense_attention_special_cases(oracle_mod):
     a, _ = oracle_mod.dense_attn(q, k9, v9)
     b, _ = oracle_mod.dense_attn(q, k9[perm], v9[perm])
     np.testing.assert_allclose(a, b, atol=1e-13)
-    k9b = k9.copy(); k9b[:, 1] += 1.0
+    k9b = k9.copy(); k9b[:, 1] *= 2.0
     c, _ = oracle_mod.dense_attn(q, k9b, v9)
     np.testing.assert_array_equal(a[:, 0], c[:, 0])
     assert np.abs(a[:, 1] - c[:, 1]).max() > 1e-6

@@ -162,6 +162,19 @@ typedef struct ll_attn_item {
 } ll_attn_item;
 int ll_sink_window_attn_batched(const ll_attn_item *items, int n_items, ll_stream stream);
 
+/* Dense attention of n_q queries over n_k keys, no mask and no RoPE: the
+ * cross-attention to the prompt that alternates with the self-attention layers
+ * and through which the recache re-encodes the prefix under the new prompt
+ * (Sec. 3.1).  Same kernel as ll_sink_window_attn, reading K and V where the
+ * projection left them.
+ *   q [n_q, heads, head_dim], k and v [n_k, heads, head_dim], bf16, device,
+ *   16-byte aligned; heads and head_dim are the handle's.  The handle lends its
+ *   scratch and status words; its caches and integer state are not touched
+ *   (calls on a handle are ordered by the caller, as everywhere).
+ *   out [n_q, heads, head_dim] bf16; lse_out [heads, n_q] fp32, nullable. */
+int ll_cross_attn(ll_cache *cache, const ll_bf16 *q, int64_t n_q, const ll_bf16 *k, const ll_bf16 *v,
+                  int64_t n_k, ll_bf16 *out, float *lse_out, ll_stream stream);
+
 /* A clip of several chunks in one step (Sec. 3.3 "Consistency between Training
  * and Inference": the resident cache is the S sink frames, the last frames of
  * the preceding context and the T frames of the current clip, attended under

@@ -98,6 +98,8 @@ SIGNATURES = {
     "ll_sink_window_attn": (C.c_int, [C.c_void_p, C.c_int, C.c_void_p, C.c_int64, C.c_int, C.c_void_p,
                                       C.c_void_p, C.c_void_p]),
     "ll_sink_window_attn_batched": (C.c_int, [C.POINTER(ll_attn_item), C.c_int, C.c_void_p]),
+    "ll_cross_attn": (C.c_int, [C.c_void_p, C.c_void_p, C.c_int64, C.c_void_p, C.c_void_p, C.c_int64, C.c_void_p,
+                                C.c_void_p, C.c_void_p]),
     "ll_clip_append_attn": (C.c_int, [C.c_void_p, C.c_int, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int64, C.c_int,
                                       C.c_int, C.c_int, C.c_int, C.c_float, C.c_void_p, C.c_void_p, C.c_void_p,
                                       C.c_void_p]),
@@ -211,6 +213,12 @@ def ll_sink_window_attn_batched(items, stream=None):
 def ll_debug_attn_simt(h, layer, q_roped, q_frame_start, n_q_frames, out, lse_out=None, stream=None):
     _check(lib().ll_debug_attn_simt(h, layer, _ptr(q_roped), q_frame_start, n_q_frames, _ptr(out),
                                     _ptr(lse_out), _stream(stream)))
+
+
+def ll_cross_attn(h, q, k, v, out, lse_out=None, stream=None, n_q=None, n_k=None):
+    n_q = q.shape[0] if n_q is None else n_q
+    n_k = k.shape[0] if n_k is None else n_k
+    _check(lib().ll_cross_attn(h, _ptr(q), n_q, _ptr(k), _ptr(v), n_k, _ptr(out), _ptr(lse_out), _stream(stream)))
 
 
 def ll_clip_append_attn(h, layer, q, k, v, frame_start, n_frames, attn_window_frames, grid_h, grid_w,
@@ -351,6 +359,9 @@ class Cache:
         """items: (Cache, layer, q_roped, q_frame_start, out, lse_out or None) per stream, one launch."""
         ll_sink_window_attn_batched([(c.h, layer, q, f0, c.C, out, lse) for c, layer, q, f0, out, lse in items],
                                     stream)
+
+    def cross_attn(self, q, k, v, out, lse_out=None, stream=None):
+        ll_cross_attn(self.h, q, k, v, out, lse_out, stream)
 
     def clip_append_attn(self, layer, q, k, v, frame_start, n_frames, attn_window_frames, grid_h, grid_w, theta,
                          q_out, out, lse_out=None, stream=None):

@@ -303,7 +303,8 @@ attn_sm100_kernel(const __grid_constant__ AttnParams p, const __grid_constant__ 
                         mbar_arrive_expect_tx(bar(kKvFull + stage), C::kTileBytes);
                         for (int a = 0; a < C::kAtoms; ++a)
                             tma_load_3d(kv_smem + stage * C::kTileBytes + a * C::kAtomBytes, m,
-                                        bar(kKvFull + stage), a * 64, row, s.head);
+                                        bar(kKvFull + stage), a * 64, p.kv_token_major ? s.head : row,
+                                        p.kv_token_major ? row : s.head);
                         ++n;
                         return true;
                     };

@@ -181,6 +181,10 @@ struct AttnCall {
     int64_t group_frame_start[ll::kMaxGroups];
     int64_t lo_floor;                             // non-sink frames older than this are hidden from every group ...
     int64_t group_lo_floor[ll::kMaxGroups];       // ... and from group g those older than this (0: no extra limit)
+    // dense attention (dense_keys > 0): one group of dense_rows queries over all dense_keys rows of the
+    // token-major k/v tensors given here; the cache lends its shape and scratch only
+    int64_t dense_rows, dense_keys;
+    const ll_bf16 *dense_k, *dense_v;
 };
 
 // Divide the columns of all groups between the CTAs (one persistent CTA per SM).  The
@@ -269,8 +273,11 @@ int build_attn_params(const AttnCall *calls, int n_calls, ll::AttnParams *p)
         if (c->H != c0->H || c->D != c0->D)
             return fail(LL_ERR_UNSUPPORTED_SHAPE, "the items of one launch must agree in heads and head_dim");
         if (ng + call.n_groups > ll::kMaxGroups) return fail(LL_ERR_UNSUPPORTED_SHAPE, "more than %d query groups", ll::kMaxGroups);
-        const int rows_per_group = c->C * c->P;
+        const bool dense = call.dense_keys > 0;
+        if (dense && n_calls != 1) return fail(LL_ERR_INVALID_ARG, "dense attention does not share a launch");
+        const int rows_per_group = dense ? (int)call.dense_rows : c->C * c->P;
         const int tiles = (rows_per_group + ll::kQTileRows - 1) / ll::kQTileRows;
+        p->kv_token_major = dense ? 1 : 0;
         p->item[i].out = call.out;
         p->item[i].lse = call.lse;
         p->item[i].nq_total = call.n_groups * rows_per_group;
@@ -282,8 +289,15 @@ int build_attn_params(const AttnCall *calls, int n_calls, ll::AttnParams *p)
             G.tiles = tiles;
             int64_t starts[LL_MAX_RANGES], lens[LL_MAX_RANGES];
             int n = 0;
-            int st = visible_ranges(c, call.layer, call.group_frame_start[g], std::max(call.lo_floor, call.group_lo_floor[g]), starts, lens, &n);
-            if (st != LL_OK) return st;
+            if (dense) {
+                starts[0] = 0;
+                lens[0] = call.dense_keys;
+                n = 1;
+            } else {
+                int st = visible_ranges(c, call.layer, call.group_frame_start[g],
+                                        std::max(call.lo_floor, call.group_lo_floor[g]), starts, lens, &n);
+                if (st != LL_OK) return st;
+            }
             G.n_ranges = n;
             G.n_kt = 0;
             for (int r = 0; r < n; ++r) {
@@ -317,6 +331,16 @@ int launch_attention(const AttnCall *calls, int n_calls, const ll::AttnParams &p
         int st = encode_map(&maps.q[i], calls[i].q, (uint64_t)c->D, (uint64_t)c->H, (uint64_t)p.item[i].nq_total,
                             (uint64_t)c->D * 2, (uint64_t)c->H * c->D * 2, 1, 128);
         if (st != LL_OK) return st;
+        if (calls[i].dense_keys > 0) {
+            // token-major K/V: coordinates (dim, head, token), a tile = 128 tokens of one head
+            st = encode_map(&maps.k[i], calls[i].dense_k, (uint64_t)c->D, (uint64_t)c->H, (uint64_t)calls[i].dense_keys,
+                            (uint64_t)c->D * 2, (uint64_t)c->H * c->D * 2, 1, 128);
+            if (st != LL_OK) return st;
+            st = encode_map(&maps.v[i], calls[i].dense_v, (uint64_t)c->D, (uint64_t)c->H, (uint64_t)calls[i].dense_keys,
+                            (uint64_t)c->D * 2, (uint64_t)c->H * c->D * 2, 1, 128);
+            if (st != LL_OK) return st;
+            continue;
+        }
         maps.k[i] = c->kmap[calls[i].layer];
         maps.v[i] = c->vmap[calls[i].layer];
     }
@@ -592,6 +616,30 @@ int ll_recache(ll_cache *c, int layer, const ll_bf16 *q, const ll_bf16 *k, const
         if (s != LL_OK) return s;
     }
     st.n_recaches += 1;
+    return LL_OK;
+}
+
+int ll_cross_attn(ll_cache *c, const ll_bf16 *q, int64_t n_q, const ll_bf16 *k, const ll_bf16 *v, int64_t n_k,
+                  ll_bf16 *out, float *lse_out, ll_stream stream)
+{
+    if (!c) return fail(LL_ERR_INVALID_ARG, "null handle");
+    if (n_q <= 0 || n_k <= 0) return fail(LL_ERR_INVALID_ARG, "n_q and n_k must be positive");
+    if (n_q > (1ll << 30) || n_k > (1ll << 30)) return fail(LL_ERR_UNSUPPORTED_SHAPE, "more than 2^30 queries or keys");
+    if (!c->dry_run) {
+        if (!q || !k || !v || !out) return fail(LL_ERR_INVALID_ARG, "null q/k/v/out");
+        if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(out) || (lse_out && !aligned16(lse_out)))
+            return fail(LL_ERR_INVALID_ARG, "pointers must be 16-byte aligned");
+        int s = need_storage(c);
+        if (s != LL_OK) return s;
+    }
+    AttnCall call{c, 0, q, out, lse_out, 1, {}, 0, {}, n_q, n_k, k, v};
+    ll::AttnParams p;
+    int s = build_attn_params(&call, 1, &p);
+    if (s != LL_OK) return s;
+    if (!c->dry_run) {
+        s = launch_attention(&call, 1, p, (cudaStream_t)stream, false);
+        if (s != LL_OK) return s;
+    }
     return LL_OK;
 }
 

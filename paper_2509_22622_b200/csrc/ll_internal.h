@@ -79,6 +79,7 @@ struct AttnParams {
     int heads;
     int nq_total;                     // rows of q / out of item 0 (the triage kernel serves one item)
     int n_ctas;                       // grid.x: persistent CTAs
+    int kv_token_major;               // K/V maps are [token][head][dim] (dense attention) instead of [head][row][dim]
     int n_waves;                      // whole-column waves
     int n_shares;                     // non-empty shares of the shared steps
     long long total_steps;            // shared steps of all groups

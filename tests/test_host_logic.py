@@ -245,3 +245,19 @@ def test_clip_step_bookkeeping_matches_the_oracle_and_errors_change_nothing(orac
     B.ll_clip_append_attn(c.h, 0, None, None, None, 24, C, C, 1, 1, 10000.0, None, None)
     B.ll_rope_append_kv(c.h, 0, None, None, None, 26, C, 1, 1)
     B.ll_sink_window_attn(c.h, 0, None, 26, C, None)
+
+
+def test_cross_attention_argument_checks():
+    c = B.Cache(1, 2, 64, 4, 1, 1, 2, dry_run=True)
+    B.ll_cross_attn(c.h, None, None, None, None, n_q=10, n_k=3)
+    for n_q, n_k in [(0, 3), (10, 0), (-1, 3), (1 << 31, 3)]:
+        with pytest.raises(B.LLError):
+            B.ll_cross_attn(c.h, None, None, None, None, n_q=n_q, n_k=n_k)
+    with pytest.raises(B.LLError):
+        B.ll_cross_attn(None, None, None, None, None, n_q=1, n_k=1)
+    real = B.ll_cache_create(1, 2, 64, 4, 1, 1, 2)           # no storage bound: must refuse, not compute
+    with pytest.raises(B.LLError) as e:
+        B.ll_cross_attn(real, None, None, None, None, n_q=1, n_k=1)
+    assert e.value.code in (B.LL_ERR_INVALID_ARG, B.LL_ERR_NO_STORAGE)
+    B.ll_cache_destroy(real)
+    assert c.state()["attn_calls"] == 0

@@ -306,6 +306,9 @@ int ll_debug_wait_timeout(ll_cache *cache, int limit_ms, ll_stream stream);
  * shares: CTA i takes shared steps [share_begin[k], share_begin[k + 1]) with
  * k = share_of_cta[i], or none when that is -1.  Shares are sized so that
  * whole columns plus share come to the same number of steps on every CTA.
+ * When the columns are short (merging the parts of a split column would cost
+ * more than splitting saves) nothing is shared: the last wave is partial,
+ * columns numbered all_cols and up do not exist, and n_shares is 0.
  * ll_debug_attn_plan_batched: the same for ll_sink_window_attn_batched of the
  * newest chunk of every item (only cache and layer of an item are read). */
 #define LL_MAX_GROUPS 24
@@ -316,7 +319,7 @@ typedef struct ll_attn_plan {
     int32_t heads;
     int32_t n_waves;
     int32_t n_shares;
-    int32_t reserved;
+    int32_t all_cols;
     int64_t shared_steps;
     int32_t tiles[LL_MAX_GROUPS];
     int32_t n_kt[LL_MAX_GROUPS];

@@ -51,7 +51,7 @@ class ll_attn_plan(C.Structure):
         ("heads", C.c_int32),
         ("n_waves", C.c_int32),
         ("n_shares", C.c_int32),
-        ("reserved", C.c_int32),
+        ("all_cols", C.c_int32),
         ("shared_steps", C.c_int64),
         ("tiles", C.c_int32 * LL_MAX_GROUPS),
         ("n_kt", C.c_int32 * LL_MAX_GROUPS),

@@ -154,11 +154,13 @@ struct WorkIter {
     {
         if (wave < p.n_waves) {
             const int col = wave * p.n_ctas + cta;                  // launch-wide column number
-            while (col >= p.g[g].col_begin + p.heads * p.g[g].tiles) ++g;
-            fill(s, g, col - p.g[g].col_begin, 0, p.g[g].n_kt);
-            s.col_begin = 0;
             ++wave;
-            return true;
+            if (col < p.all_cols) {
+                while (col >= p.g[g].col_begin + p.heads * p.g[g].tiles) ++g;
+                fill(s, g, col - p.g[g].col_begin, 0, p.g[g].n_kt);
+                s.col_begin = 0;
+                return true;
+            }
         }
         if (u >= end) return false;
         int gg = 0;

@@ -198,7 +198,27 @@ void plan_work(ll::AttnParams *p, int sms, long long all_cols, long long all_ste
     const bool waves = all_cols >= sms;
     p->n_ctas = waves ? sms : (int)std::min<long long>(sms, all_steps);
     p->n_waves = waves ? (int)(all_cols / sms) : 0;
-    const long long whole_cols = (long long)p->n_waves * p->n_ctas;
+    p->all_cols = (int)all_cols;
+    {
+        // Short columns: splitting the leftover columns saves at most their length minus an even
+        // share, and costs every part a trip through the scratch slots (about kMergeSteps steps'
+        // worth).  When that does not pay, the leftover goes out whole as one more, partial wave.
+        constexpr long long kMergeSteps = 3;
+        const long long first_left = (long long)p->n_waves * sms;
+        long long left_steps = 0, left_longest = 0;
+        for (int g = 0; g < p->n_groups; ++g) {
+            const ll::AttnGroup &G = p->g[g];
+            const long long cols = (long long)p->heads * G.tiles;
+            const long long left = std::min(cols, std::max<long long>(0, G.col_begin + cols - first_left));
+            left_steps += left * G.n_kt;
+            if (left > 0) left_longest = std::max<long long>(left_longest, G.n_kt);
+        }
+        if (left_steps > 0 && left_longest <= (left_steps + sms - 1) / sms + kMergeSteps) {
+            p->n_waves += 1;
+            p->n_ctas = (int)std::min<long long>(sms, all_cols);
+        }
+    }
+    const long long whole_cols = std::min<long long>((long long)p->n_waves * p->n_ctas, all_cols);
     long long steps = 0;
     for (int g = 0; g < p->n_groups; ++g) {
         ll::AttnGroup &G = p->g[g];
@@ -719,6 +739,7 @@ void copy_plan(const ll::AttnParams &p, ll_attn_plan *out)
     out->heads = p.heads;
     out->n_waves = p.n_waves;
     out->n_shares = p.n_shares;
+    out->all_cols = p.all_cols;
     out->shared_steps = p.total_steps;
     for (int k = 0; k <= p.n_shares; ++k) out->share_begin[k] = p.share_begin[k];
     for (int i = 0; i < p.n_ctas; ++i) out->share_of_cta[i] = p.share_of_cta[i];

@@ -42,7 +42,9 @@ struct LayerState {
 // i, i + n_ctas, ..., and the steps of the columns left over are laid end to
 // end and cut into one share per CTA, sized so that every CTA ends up with the
 // same number of steps (whole columns of groups with different key counts
-// weigh differently).
+// weigh differently).  When the columns are so short that merging the parts of a
+// split column would cost more than it saves, the last columns go out whole as
+// a partial wave instead and nothing is shared.
 struct AttnGroup {
     int item;                         // which (cache, layer, q, out) of the launch the group belongs to
     int q_begin;                      // first query row of the group in its item's q tensor
@@ -80,7 +82,8 @@ struct AttnParams {
     int nq_total;                     // rows of q / out of item 0 (the triage kernel serves one item)
     int n_ctas;                       // grid.x: persistent CTAs
     int kv_token_major;               // K/V maps are [token][head][dim] (dense attention) instead of [head][row][dim]
-    int n_waves;                      // whole-column waves
+    int n_waves;                      // whole-column waves (the last may be partial: columns >= all_cols do not exist)
+    int all_cols;                     // columns of all groups
     int n_shares;                     // non-empty shares of the shared steps
     long long total_steps;            // shared steps of all groups
     int64_t rows_per_head;            // (S+W)*P

@@ -26,6 +26,8 @@ def cta_work(plan, cta):
     g = 0
     for wave in range(plan.n_waves):
         col = wave * G + cta                                  # launch-wide column number
+        if col >= plan.all_cols:                              # a partial last wave
+            continue
         while col >= plan.col_begin[g] + plan.heads * plan.tiles[g]:
             g += 1
         out.append((g, col - plan.col_begin[g], 0, plan.n_kt[g]))
@@ -69,7 +71,7 @@ def check_plan(plan):
     for cta in range(G):
         work = cta_work(plan, cta)
         loads.append(sum(k1 - k0 for _, _, k0, k1 in work))
-        whole.append(sum(k1 - k0 for _, _, k0, k1 in work[:plan.n_waves]))
+        whole.append(sum(k1 - k0 for g, col, k0, k1 in work if col < plan.wave_cols[g]))
         for g, col, k0, k1 in work:
             assert 0 <= col < plan.heads * plan.tiles[g] and 0 <= k0 < k1 <= plan.n_kt[g]
             for k in range(k0, k1):
@@ -79,6 +81,13 @@ def check_plan(plan):
     assert len(done) == total, "steps left undone"
     # the shares level the CTAs: those that take one end within a step of each other, and a CTA
     # that takes none was at that level already
+    assert plan.all_cols == sum(plan.heads * plan.tiles[g] for g in range(plan.n_groups))
+    if plan.n_shares == 0:
+        # short columns: everything goes out whole; CTAs differ by their last column at most, and the
+        # choice was right: splitting could not have saved more than a merge costs
+        longest = max(plan.n_kt[g] for g in range(plan.n_groups))
+        assert plan.shared_steps == 0 and max(loads) - min(loads) <= longest
+        return
     level = max((loads[i] for i in range(G) if plan.share_of_cta[i] >= 0), default=min(loads))
     for i in range(G):
         if plan.share_of_cta[i] >= 0:
@@ -166,3 +175,24 @@ def test_plan_of_eight_ragged_streams():
     check_plan(plan)
     for h in handles:
         B.ll_cache_destroy(h)
+
+
+def test_short_columns_are_not_split():
+    """A prompt-sized key set (4 key tiles per column): 228 columns go out as one full and one
+    partial wave and nothing passes through the merge scratch."""
+    h = B.ll_cache_create(1, 12, 128, 1560, 3, 3, 3)
+    B.ll_cache_set_dry_run(h, True)
+    B.ll_rope_append_kv(h, 0, None, None, None, 0, 3, 1, 1560)
+    plan = B.ll_debug_attn_plan(h, sm_count=148)           # chunk 0 sees itself: 37 tiles per column, split
+    assert plan.n_waves == 1 and plan.n_shares == 148
+    small = B.ll_cache_create(1, 12, 128, 130, 3, 3, 3)     # 390 rows: 2 tiles x 12 heads = 24 columns of 4 key tiles
+    B.ll_cache_set_dry_run(small, True)
+    B.ll_rope_append_kv(small, 0, None, None, None, 0, 3, 1, 130)
+    plan = B.ll_debug_attn_plan(small, sm_count=148)
+    assert (plan.n_ctas, plan.n_waves, plan.n_shares, plan.shared_steps) == (24, 1, 0, 0)
+    check_plan(plan)
+    plan = B.ll_debug_attn_plan(small, sm_count=7)          # 24 columns on 7 CTAs: 3 full waves + 3 columns
+    assert (plan.n_ctas, plan.n_waves, plan.n_shares) == (7, 4, 0)
+    check_plan(plan)
+    B.ll_cache_destroy(h)
+    B.ll_cache_destroy(small)

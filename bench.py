@@ -376,6 +376,69 @@ def run_ours(args):
     recache_ms = rc[0].elapsed_time(rc[1]) / 3
     cache.check_device()
 
+    # The other entry points at the same layer shape, a few launches each, reported beside the
+    # headline: eight streams at ragged positions in one launch, a 21-frame clip in one call,
+    # cross-attention over a 512-token prompt.
+    def median_ms(fn, reps=10):
+        for _ in range(2):
+            fn()
+        torch.cuda.synchronize()
+        times = []
+        for _ in range(reps):
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record(stream)
+            fn()
+            b.record(stream)
+            torch.cuda.synchronize()
+            times.append(a.elapsed_time(b))
+        return sorted(times)[len(times) // 2]
+
+    others = {}
+    if rank == 0:
+        q, k, v = dev_sets[0]
+        positions = synth.SWEEP_POSITIONS
+        streams, items, flops8 = [], [], 0.0
+        for pos in positions:
+            c = B.Cache(1, H, D, P, C, wl.sink_frames, wl.window_frames, device="cuda:%d" % local_rank)
+            qr = torch.empty_like(q)
+            for chunk in range(pos + 1):
+                c.rope_append_kv(0, q, k, v, chunk * C, wl.grid_h, wl.grid_w, wl.rope_theta, qr)
+            streams.append(c)
+            items.append((c, 0, qr, pos * C, torch.empty_like(q), None))
+            ring = min(pos + 1, wl.window_frames // C) * C
+            sink = wl.sink_frames if pos + 1 > wl.window_frames // C else 0
+            flops8 += 4.0 * nq * (ring + sink) * P * D * H
+        ms = median_ms(lambda: B.Cache.sink_window_attn_batched(items))
+        others["batched_8_ragged_streams"] = {"ms": ms, "tflops": flops8 / ms / 1e9, "positions": list(positions)}
+        for c in streams:
+            c.check_device()
+            c.close()
+        del streams, items
+        clip_chunks = 7
+        T = clip_chunks * C
+        big = B.Cache(1, H, D, P, C, wl.sink_frames, wl.window_frames + T - C, device="cuda:%d" % local_rank)
+        for chunk in range(n_fill):
+            big.rope_append_kv(0, None, k, v, chunk * C, wl.grid_h, wl.grid_w, wl.rope_theta)
+        cq, ck, cv = (torch.cat([dev_sets[i % N_INPUT_SETS][j] for i in range(clip_chunks)]) for j in range(3))
+        cq_out, c_out = torch.empty_like(cq), torch.empty_like(cq)
+        pos = [n_fill * C]
+
+        def clip():
+            big.clip_append_attn(0, cq, ck, cv, pos[0], T, wl.window_frames, wl.grid_h, wl.grid_w, wl.rope_theta,
+                                 cq_out, c_out)
+            pos[0] += T
+        ms = median_ms(clip)
+        others["clip_21_frames"] = {"ms": ms, "tflops_attention_over_append_plus_attention":
+                                    clip_chunks * attn_flops(wl) / ms / 1e9}
+        big.check_device()
+        big.close()
+        n_prompt = 512
+        pk = torch.randn(n_prompt, H, D, device="cuda").bfloat16()
+        pv = torch.randn(n_prompt, H, D, device="cuda").bfloat16()
+        ms = median_ms(lambda: cache.cross_attn(q, pk, pv, out))
+        others["cross_attn_512_keys"] = {"us": ms * 1e3, "tflops": 4.0 * nq * n_prompt * D * H / ms / 1e9}
+        cache.check_device()
+
     total_ms, e2e_ms, attn_ms, append_ms = reduce_max([total_ms, e2e_ms, attn_ms, append_ms], dist, "cuda")
     if rank != 0:
         if dist is not None:
@@ -423,6 +486,7 @@ def run_ours(args):
                   "latent_frames_per_s_30_layers_4_passes": C / (120 * ms_per_step * 1e-3),
                   "recache_ms_per_layer": recache_ms,
                   "recache_tflops": 9 * attn_flops(wl) / 4 / (recache_ms * 1e-3) / 1e12,
+                  "other_entry_points": others,
                   "paper_context": "20.7 video FPS (about 5.2 latent frames/s) for the whole 1.3B model on one H100"},
     }
     print(json.dumps(line))

@@ -83,6 +83,8 @@ def lib():
             L.llo_clip.argtypes = [C.c_void_p, C.c_int] + [C.POINTER(C.c_double)] * 3 + \
                                   [C.c_int64, C.c_int, C.c_int, C.c_int, C.c_int, C.c_double,
                                    C.POINTER(C.c_int64), C.c_int64] + [C.POINTER(C.c_double)] * 3
+            L.llo_rms_norm.argtypes = [C.POINTER(C.c_double), C.POINTER(C.c_double), C.c_double, C.c_int64, C.c_int,
+                                       C.POINTER(C.c_double)]
             L.llo_dense_attn.argtypes = [C.POINTER(C.c_double)] * 3 + [C.c_int64, C.c_int64, C.c_int, C.c_int,
                                                                        C.POINTER(C.c_int64), C.c_int64,
                                                                        C.POINTER(C.c_double), C.POINTER(C.c_double)]
@@ -124,6 +126,20 @@ def rope(x, frame_start: int, gh: int, gw: int, theta: float = 10000.0, round_bf
     if st != OK:
         raise OracleError(st, "rope")
     return out
+
+
+def rms_norm(x, gain, eps: float):
+    """RMS norm of every token's whole row: x [tokens, H, D], gain [H, D] (or flat [H*D])."""
+    x = _f64(x)
+    g = _f64(gain).reshape(-1)
+    n = int(np.prod(x.shape[1:]))
+    if g.shape[0] != n:
+        raise OracleError(ERR_ARG, "rms_norm shape")
+    y = np.empty_like(x)
+    st = lib().llo_rms_norm(_dp(x), _dp(g), eps, x.shape[0], n, _dp(y))
+    if st != OK:
+        raise OracleError(st, "rms_norm")
+    return y
 
 
 def dense_attn(q, k, v, rows=None):

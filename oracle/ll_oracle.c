@@ -35,7 +35,10 @@
  *     pair j holds elements (2j, 2j+1); pair i of an axis with n_a pairs turns by
  *     pos_axis * theta^(-i/n_a).  Positions are absolute (t = frame index since
  *     the stream began).  K is cached after the rotation.
- *   - Softmax scale 1/sqrt(D); any q/k normalisation is upstream.
+ *   - Softmax scale 1/sqrt(D).  The paper does not define the q/k normalisation of
+ *     its base model; where a caller wants it fused into the append it is the RMS
+ *     norm over the token's whole row of H*D elements with a learned gain
+ *     (llo_rms_norm), applied before the rotation.
  *
  * Storage here is [layer][slot][token][head][dim] in double.  The slot rule
  * (frame f -> slot f if f < S, else S + (f - S) mod W) is the bit-exact
@@ -452,6 +455,24 @@ int llo_clip(llo *o, int layer, const double *q, const double *k, const double *
     int st = attn_in_window(o, layer, qr, frame_start, n_frames, 0, window, rows, n_rows, out, lse);
     if (!q_roped_out) free(qr);
     return st;
+}
+
+/* ---- step: RMS norm of q and k rows (upstream of the rotation) ---------------- */
+
+/* y[t][e] = x[t][e] / sqrt(mean_e(x[t][e]^2) + eps) * gain[e], e over the token's
+ * whole row of n_elems = H*D elements. */
+int llo_rms_norm(const double *x, const double *gain, double eps, int64_t n_tokens, int n_elems, double *y)
+{
+    if (!x || !gain || !y || n_tokens < 0 || n_elems <= 0) return LLO_ERR_ARG;
+    for (int64_t t = 0; t < n_tokens; ++t) {
+        const double *xr = x + (size_t)t * n_elems;
+        double ms = 0.0;
+        for (int e = 0; e < n_elems; ++e) ms += xr[e] * xr[e];
+        ms /= (double)n_elems;
+        double r = 1.0 / sqrt(ms + eps);
+        for (int e = 0; e < n_elems; ++e) y[(size_t)t * n_elems + e] = xr[e] * r * gain[e];
+    }
+    return LLO_OK;
 }
 
 /* ---- step: dense attention (cross-attention to the prompt, Sec. 3.1) -------- */

@@ -594,3 +594,41 @@ def test_dense_attention_special_cases(oracle_mod):
     c, _ = oracle_mod.dense_attn(q, k9b, v9)
     np.testing.assert_array_equal(a[:, 0], c[:, 0])
     assert np.abs(a[:, 1] - c[:, 1]).max() > 1e-6
+
+
+# ---------------------------------------------------------------------------
+# RMS norm of q/k rows (upstream of the rotation; not in the paper)
+# ---------------------------------------------------------------------------
+
+def test_rms_norm_closed_forms(oracle_mod):
+    # the 3-4-5 row: mean square 12.5
+    y = oracle_mod.rms_norm(np.array([[[3.0, 4.0]]]), np.ones(2), 0.0)
+    np.testing.assert_allclose(y, np.array([[[3.0, 4.0]]]) / np.sqrt(12.5), rtol=1e-15)
+    # a constant row c with eps: c / sqrt(c^2 + eps) * gain
+    g = np.array([0.5, -2.0, 1.0, 3.0])
+    y = oracle_mod.rms_norm(np.full((1, 2, 2), -1.5), g, 0.25)
+    np.testing.assert_allclose(y.reshape(-1), -1.5 / np.sqrt(2.5) * g, rtol=1e-15)
+    # a zero row stays zero (eps keeps the division finite)
+    assert np.all(oracle_mod.rms_norm(np.zeros((2, 1, 4)), np.ones(4), 1e-6) == 0.0)
+
+
+def test_rms_norm_invariants(oracle_mod):
+    x = rand((9, 3, 8), 77)
+    g = rand((3, 8), 78)
+    y = oracle_mod.rms_norm(x, g, 0.0)
+    # gain 1: every token's whole row has mean square 1, whatever its scale
+    y1 = oracle_mod.rms_norm(x, np.ones(24), 0.0)
+    np.testing.assert_allclose((y1.reshape(9, -1) ** 2).mean(axis=1), 1.0, rtol=1e-13)
+    np.testing.assert_allclose(oracle_mod.rms_norm(7.0 * x, g, 0.0), y, rtol=1e-13)
+    # the gain multiplies element-wise, the norm is over the row, not per head
+    np.testing.assert_allclose(y, y1 * g[None], rtol=1e-14)
+    per_head = x / np.sqrt((x ** 2).mean(axis=2, keepdims=True))
+    assert np.abs(per_head - y1).max() > 1e-3
+    # tokens are independent
+    x2 = x.copy(); x2[4] *= 3.0
+    y2 = oracle_mod.rms_norm(x2, g, 1e-6)
+    ye = oracle_mod.rms_norm(x, g, 1e-6)
+    np.testing.assert_array_equal(np.delete(y2, 4, axis=0), np.delete(ye, 4, axis=0))
+    # eps matters for small rows: with eps the output shrinks
+    small = 1e-3 * x
+    assert np.abs(oracle_mod.rms_norm(small, g, 1e-6)).max() < np.abs(oracle_mod.rms_norm(small, g, 0.0)).max()

@@ -432,6 +432,19 @@ def run_ours(args):
                                     clip_chunks * attn_flops(wl) / ms / 1e9}
         big.check_device()
         big.close()
+        gains = torch.ones(H * D, device="cuda")
+        layer_i = [0]
+
+        def norm_append(n=20):
+            for _ in range(n):
+                layer_i[0] = (layer_i[0] + 1) % N_LAYERS
+                fs = cache.state(layer_i[0])["end"] - C                  # overwrite the newest chunk in place
+                qq, kk, vv = dev_sets[layer_i[0] % N_INPUT_SETS]
+                cache.norm_rope_append_kv(layer_i[0], qq, kk, vv, gains, gains, 1e-6, fs, wl.grid_h, wl.grid_w,
+                                          wl.rope_theta, q_roped)
+        ms = median_ms(norm_append) / 20
+        others["norm_rope_append"] = {"us": ms * 1e3, "gbs": append_bytes(wl) / ms / 1e6,
+                                      "frac_of_copy_peak": append_bytes(wl) / ms / 1e6 / load_peaks()[0]["hbm_gbs"]}
         n_prompt = 512
         pk = torch.randn(n_prompt, H, D, device="cuda").bfloat16()
         pv = torch.randn(n_prompt, H, D, device="cuda").bfloat16()

@@ -125,6 +125,22 @@ int ll_rope_append_kv(ll_cache *cache, int layer, const ll_bf16 *q, const ll_bf1
                       int grid_h, int grid_w, float rope_theta, ll_bf16 *q_out,
                       ll_stream stream);
 
+/* The same with the base model's q/k normalisation in front (the paper does not
+ * define it; this is the RMS norm over a token's whole row of heads*head_dim
+ * elements with a learned gain, applied before the rotation):
+ *   x_hat[e] = x[e] / sqrt(mean_e(x[e]^2) + eps) * gain[e]
+ * for q (gain_q) and k (gain_k), in fp32, then RoPE and append as above; v is
+ * stored as it comes.  One pass over q, k, v instead of a norm kernel followed
+ * by ll_rope_append_kv.
+ *   gain_q, gain_k  [heads*head_dim] fp32, device, 16-byte aligned; gain_q may
+ *                   be null when q_out is null
+ *   eps >= 0
+ * Everything else (positions, state, errors) as ll_rope_append_kv. */
+int ll_norm_rope_append_kv(ll_cache *cache, int layer, const ll_bf16 *q, const ll_bf16 *k,
+                           const ll_bf16 *v, const float *gain_q, const float *gain_k, float eps,
+                           int64_t frame_start, int n_frames, int grid_h, int grid_w,
+                           float rope_theta, ll_bf16 *q_out, ll_stream stream);
+
 /* Sink+window attention of the newest chunk's queries (Sec. 3.3): every query
  * attends to all sink rows and all resident window rows (the chunk itself
  * included; bidirectional inside the chunk), softmax scale 1/sqrt(head_dim).

@@ -95,6 +95,9 @@ SIGNATURES = {
     "ll_cache_kv_offset": (C.c_int, [C.c_void_p, C.c_int, C.c_int, C.c_int, C.POINTER(C.c_size_t)]),
     "ll_rope_append_kv": (C.c_int, [C.c_void_p, C.c_int, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int64,
                                     C.c_int, C.c_int, C.c_int, C.c_float, C.c_void_p, C.c_void_p]),
+    "ll_norm_rope_append_kv": (C.c_int, [C.c_void_p, C.c_int, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p,
+                                         C.c_void_p, C.c_float, C.c_int64, C.c_int, C.c_int, C.c_int, C.c_float,
+                                         C.c_void_p, C.c_void_p]),
     "ll_sink_window_attn": (C.c_int, [C.c_void_p, C.c_int, C.c_void_p, C.c_int64, C.c_int, C.c_void_p,
                                       C.c_void_p, C.c_void_p]),
     "ll_sink_window_attn_batched": (C.c_int, [C.POINTER(ll_attn_item), C.c_int, C.c_void_p]),
@@ -192,6 +195,13 @@ def ll_rope_append_kv(h, layer, q, k, v, frame_start, n_frames, grid_h, grid_w, 
                       q_out=None, stream=None):
     _check(lib().ll_rope_append_kv(h, layer, _ptr(q), _ptr(k), _ptr(v), frame_start, n_frames, grid_h, grid_w,
                                    rope_theta, _ptr(q_out), _stream(stream)))
+
+
+def ll_norm_rope_append_kv(h, layer, q, k, v, gain_q, gain_k, eps, frame_start, n_frames, grid_h, grid_w,
+                           rope_theta=10000.0, q_out=None, stream=None):
+    _check(lib().ll_norm_rope_append_kv(h, layer, _ptr(q), _ptr(k), _ptr(v), _ptr(gain_q), _ptr(gain_k), eps,
+                                        frame_start, n_frames, grid_h, grid_w, rope_theta, _ptr(q_out),
+                                        _stream(stream)))
 
 
 def ll_sink_window_attn(h, layer, q_roped, q_frame_start, n_q_frames, out, lse_out=None, stream=None):
@@ -350,6 +360,11 @@ class Cache:
 
     def rope_append_kv(self, layer, q, k, v, frame_start, grid_h, grid_w, theta=10000.0, q_out=None, stream=None):
         ll_rope_append_kv(self.h, layer, q, k, v, frame_start, self.C, grid_h, grid_w, theta, q_out, stream)
+
+    def norm_rope_append_kv(self, layer, q, k, v, gain_q, gain_k, eps, frame_start, grid_h, grid_w, theta=10000.0,
+                            q_out=None, stream=None):
+        ll_norm_rope_append_kv(self.h, layer, q, k, v, gain_q, gain_k, eps, frame_start, self.C, grid_h, grid_w,
+                               theta, q_out, stream)
 
     def sink_window_attn(self, layer, q_roped, q_frame_start, out, lse_out=None, stream=None):
         ll_sink_window_attn(self.h, layer, q_roped, q_frame_start, self.C, out, lse_out, stream)

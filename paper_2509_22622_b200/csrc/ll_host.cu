@@ -510,9 +510,12 @@ int ll_cache_kv_offset(const ll_cache *c, int layer, int which, int head, size_t
     return LL_OK;
 }
 
-int ll_rope_append_kv(ll_cache *c, int layer, const ll_bf16 *q, const ll_bf16 *k, const ll_bf16 *v,
-                      int64_t frame_start, int n_frames, int grid_h, int grid_w, float rope_theta,
-                      ll_bf16 *q_out, ll_stream stream)
+namespace {
+// ll_rope_append_kv, and with gains given ll_norm_rope_append_kv.
+int append_entry(ll_cache *c, int layer, const ll_bf16 *q, const ll_bf16 *k, const ll_bf16 *v,
+                 const float *gain_q, const float *gain_k, float eps, bool with_norm,
+                 int64_t frame_start, int n_frames, int grid_h, int grid_w, float rope_theta,
+                 ll_bf16 *q_out, ll_stream stream)
 {
     if (!layer_ok(c, layer)) return fail(LL_ERR_INVALID_ARG, "bad cache handle or layer %d", layer);
     if (grid_h <= 0 || grid_w <= 0 || (int64_t)grid_h * grid_w != c->P)
@@ -531,13 +534,17 @@ int ll_rope_append_kv(ll_cache *c, int layer, const ll_bf16 *q, const ll_bf16 *k
         if (q_out && !q) return fail(LL_ERR_INVALID_ARG, "q_out given without q");
         if (!aligned16(k) || !aligned16(v) || !aligned16(q) || !aligned16(q_out))
             return fail(LL_ERR_INVALID_ARG, "q/k/v/q_out must be 16-byte aligned");
+        if (with_norm && (!gain_k || (q_out && !gain_q))) return fail(LL_ERR_INVALID_ARG, "null gain");
+        if (with_norm && (!aligned16(gain_q) || !aligned16(gain_k)))
+            return fail(LL_ERR_INVALID_ARG, "gains must be 16-byte aligned");
         int s = need_storage(c);
         if (s != LL_OK) return s;
         s = ensure_tables(c, frame_start, frame_start + n_frames, grid_h, grid_w, rope_theta, (cudaStream_t)stream);
         if (s != LL_OK) return s;
         ll::RopeAppendParams p;
         fill_rope_params(c, layer, q_out ? q : nullptr, k, v, q_out, frame_start, n_frames, grid_w, &p);
-        cudaError_t e = ll::launch_rope_append(p, c->D, (cudaStream_t)stream);
+        cudaError_t e = with_norm ? ll::launch_norm_rope_append(p, c->D, gain_q, gain_k, eps, (cudaStream_t)stream)
+                                  : ll::launch_rope_append(p, c->D, (cudaStream_t)stream);
         if (e != cudaSuccess) return cuda_fail(e, "rope+append kernel");
     }
     if (is_new) {
@@ -553,6 +560,24 @@ int ll_rope_append_kv(ll_cache *c, int layer, const ll_bf16 *q, const ll_bf16 *k
         st.n_overwrites += 1;
     }
     return LL_OK;
+}
+}  // namespace
+
+int ll_rope_append_kv(ll_cache *c, int layer, const ll_bf16 *q, const ll_bf16 *k, const ll_bf16 *v,
+                      int64_t frame_start, int n_frames, int grid_h, int grid_w, float rope_theta,
+                      ll_bf16 *q_out, ll_stream stream)
+{
+    return append_entry(c, layer, q, k, v, nullptr, nullptr, 0.f, false, frame_start, n_frames, grid_h, grid_w,
+                        rope_theta, q_out, stream);
+}
+
+int ll_norm_rope_append_kv(ll_cache *c, int layer, const ll_bf16 *q, const ll_bf16 *k, const ll_bf16 *v,
+                           const float *gain_q, const float *gain_k, float eps, int64_t frame_start, int n_frames,
+                           int grid_h, int grid_w, float rope_theta, ll_bf16 *q_out, ll_stream stream)
+{
+    if (!(eps >= 0.f)) return fail(LL_ERR_INVALID_ARG, "eps must be non-negative");
+    return append_entry(c, layer, q, k, v, gain_q, gain_k, eps, true, frame_start, n_frames, grid_h, grid_w,
+                        rope_theta, q_out, stream);
 }
 
 int ll_sink_window_attn(ll_cache *c, int layer, const ll_bf16 *q_roped, int64_t q_frame_start,

@@ -120,6 +120,8 @@ cudaError_t launch_rope_tables(float2 *t_tab, int64_t t_base, int n_t_frames, in
                                float2 *h_tab, int grid_h, float2 *w_tab, int grid_w, int n_hw,
                                float theta, bool do_t, bool do_hw, cudaStream_t stream);
 cudaError_t launch_rope_append(const RopeAppendParams &p, int head_dim, cudaStream_t stream);
+cudaError_t launch_norm_rope_append(const RopeAppendParams &p, int head_dim, const float *gain_q, const float *gain_k,
+                                    float eps, cudaStream_t stream);
 cudaError_t launch_attn_sm100(const AttnParams &p, int head_dim, const AttnMaps &maps, cudaStream_t stream);
 cudaError_t launch_attn_simt(const AttnParams &p, int head_dim, cudaStream_t stream);
 // what the probe of the bounded-wait machinery records as barrier and iteration

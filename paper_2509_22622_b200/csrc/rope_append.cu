@@ -119,7 +119,157 @@ rope_append_kernel(const __grid_constant__ RopeAppendParams p)
     }
 }
 
+// ---- the same with the RMS norm of q and k in front -----------------------------------
+//
+// One warp owns one token.  Its lanes take the row's 16-byte vectors round-robin; a first
+// pass over q and k sums the squares (fp32, then a butterfly over the warp), a second pass
+// scales by the row's factor and the gain, rotates and stores.  Rows of up to 192 vectors
+// (1536 elements at head_dim 128) stay in registers between the passes; longer ones are
+// read again (from L1/L2).  The row stride in vectors (32) is a multiple of the vectors per head (8 or
+// 16), so a lane meets the same four rotation pairs in every vector it owns and fetches
+// their (cos, sin) once.
+__device__ __forceinline__ float sum_squares(uint4 x)
+{
+    float s = 0.f;
+    const uint32_t w[4] = {x.x, x.y, x.z, x.w};
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+        const float a = __uint_as_float(w[u] << 16), b = __uint_as_float(w[u] & 0xffff0000u);
+        s = fmaf(a, a, s);
+        s = fmaf(b, b, s);
+    }
+    return s;
+}
+
+__device__ __forceinline__ uint32_t norm_rotate_pair(uint32_t packed, float r, float2 gain, float2 cs)
+{
+    const float a = __uint_as_float(packed << 16) * r * gain.x;
+    const float b = __uint_as_float(packed & 0xffff0000u) * r * gain.y;
+    const float r0 = fmaf(a, cs.x, -(b * cs.y));
+    const float r1 = fmaf(a, cs.y, b * cs.x);
+    __nv_bfloat162 o = __floats2bfloat162_rn(r0, r1);
+    return *reinterpret_cast<uint32_t *>(&o);
+}
+
+__device__ __forceinline__ uint4 norm_rotate_vec(uint4 x, float r, const float *gain, const float2 (&cs)[4])
+{
+    const float4 g0 = *reinterpret_cast<const float4 *>(gain), g1 = *reinterpret_cast<const float4 *>(gain + 4);
+    return make_uint4(norm_rotate_pair(x.x, r, make_float2(g0.x, g0.y), cs[0]),
+                      norm_rotate_pair(x.y, r, make_float2(g0.z, g0.w), cs[1]),
+                      norm_rotate_pair(x.z, r, make_float2(g1.x, g1.y), cs[2]),
+                      norm_rotate_pair(x.w, r, make_float2(g1.z, g1.w), cs[3]));
+}
+
+// kIters > 0: the row's vectors fit kIters per lane and stay in registers between the two
+// passes (one read of q, k, v from memory); kIters == 0: any row length, second pass re-reads.
+template <int D, int kIters>
+__global__ void __launch_bounds__(kThreads)
+norm_rope_append_kernel(const __grid_constant__ RopeAppendParams p, const float *__restrict__ gain_q,
+                        const float *__restrict__ gain_k, float eps)
+{
+    constexpr int kVecs = D / 8;                       // 16-byte vectors per head row
+    static_assert(32 % kVecs == 0, "a lane must meet the same rotation pairs in all its vectors");
+    constexpr int kHeld = kIters > 0 ? kIters : 1;
+    const int lane = threadIdx.x & 31;
+    const long long token = (long long)blockIdx.x * (kThreads / 32) + (threadIdx.x >> 5);
+    if (token >= p.n_tokens) return;
+    const int row_vecs = p.heads * kVecs;
+    const int frame = (int)(token / p.P);
+    const int cell = (int)(token % p.P);
+    const int y = cell / p.grid_w, x = cell % p.grid_w;
+    const size_t in_base = (size_t)token * row_vecs * 8;
+    const bool with_q = p.q_out != nullptr;
+
+    uint4 hq[kHeld], hk[kHeld], hv[kHeld];
+    float sq = 0.f, sk = 0.f;
+    if (kIters > 0) {
+#pragma unroll
+        for (int i = 0; i < kHeld; ++i) {
+            const int v = lane + 32 * i;
+            if (v < row_vecs) {
+                hk[i] = ld16(p.k + in_base + (size_t)v * 8);
+                hv[i] = ld16(p.v + in_base + (size_t)v * 8);
+                if (with_q) hq[i] = ld16(p.q + in_base + (size_t)v * 8);
+            }
+        }
+#pragma unroll
+        for (int i = 0; i < kHeld; ++i) {
+            if (lane + 32 * i < row_vecs) {
+                sk += sum_squares(hk[i]);
+                if (with_q) sq += sum_squares(hq[i]);
+            }
+        }
+    } else {
+        for (int v = lane; v < row_vecs; v += 32) {
+            sk += sum_squares(ld16(p.k + in_base + (size_t)v * 8));
+            if (with_q) sq += sum_squares(ld16(p.q + in_base + (size_t)v * 8));
+        }
+    }
+#pragma unroll
+    for (int m = 16; m > 0; m >>= 1) {
+        sq += __shfl_xor_sync(0xffffffffu, sq, m);
+        sk += __shfl_xor_sync(0xffffffffu, sk, m);
+    }
+    const float inv_n = 1.f / (float)(row_vecs * 8);
+    const float rq = 1.f / sqrtf(fmaf(sq, inv_n, eps)), rk = 1.f / sqrtf(fmaf(sk, inv_n, eps));
+
+    const int vec = lane % kVecs;                      // the lane's vector inside every head row it meets
+    float2 cs[4];
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+        const int j = vec * 4 + u;
+        const float2 *src;
+        if (j < p.n_t)             src = p.t_tab + (size_t)frame * p.n_t + j;
+        else if (j < p.n_t + p.n_h) src = p.h_tab + (size_t)y * p.n_h + (j - p.n_t);
+        else                        src = p.w_tab + (size_t)x * p.n_h + (j - p.n_t - p.n_h);
+        cs[u] = __ldg(src);
+    }
+    const size_t cache_row = (size_t)p.slot[frame] * p.P + cell;
+    auto emit = [&](int v, uint4 xq, uint4 xk, uint4 xv) {
+        const int head = v / kVecs;
+        const size_t src = in_base + (size_t)v * 8;
+        const size_t dst = ((size_t)head * p.rows_per_head + cache_row) * D + (size_t)vec * 8;
+        st16(p.kcache + dst, norm_rotate_vec(xk, rk, gain_k + (size_t)v * 8, cs));
+        st16(p.vcache + dst, xv);
+        if (with_q) st16(p.q_out + src, norm_rotate_vec(xq, rq, gain_q + (size_t)v * 8, cs));
+    };
+    if (kIters > 0) {
+#pragma unroll
+        for (int i = 0; i < kHeld; ++i) {
+            const int v = lane + 32 * i;
+            if (v < row_vecs) emit(v, hq[i], hk[i], hv[i]);
+        }
+    } else {
+        for (int v = lane; v < row_vecs; v += 32) {
+            const size_t src = in_base + (size_t)v * 8;
+            emit(v, with_q ? ld16(p.q + src) : make_uint4(0, 0, 0, 0), ld16(p.k + src), ld16(p.v + src));
+        }
+    }
+}
+
+template <int D>
+void launch_norm_variant(const RopeAppendParams &p, const float *gain_q, const float *gain_k, float eps,
+                         unsigned blocks, cudaStream_t stream)
+{
+    const int iters = (p.heads * (D / 8) + 31) / 32;
+    if (iters <= 2)      norm_rope_append_kernel<D, 2><<<blocks, kThreads, 0, stream>>>(p, gain_q, gain_k, eps);
+    else if (iters <= 4) norm_rope_append_kernel<D, 4><<<blocks, kThreads, 0, stream>>>(p, gain_q, gain_k, eps);
+    else if (iters <= 6) norm_rope_append_kernel<D, 6><<<blocks, kThreads, 0, stream>>>(p, gain_q, gain_k, eps);
+    else                 norm_rope_append_kernel<D, 0><<<blocks, kThreads, 0, stream>>>(p, gain_q, gain_k, eps);
+}
+
 }  // namespace
+
+cudaError_t launch_norm_rope_append(const RopeAppendParams &p, int head_dim, const float *gain_q, const float *gain_k,
+                                    float eps, cudaStream_t stream)
+{
+    const unsigned blocks = (unsigned)((p.n_tokens + kThreads / 32 - 1) / (kThreads / 32));
+    if (blocks == 0) return cudaSuccess;
+    if (head_dim == 128) launch_norm_variant<128>(p, gain_q, gain_k, eps, blocks, stream);
+    else                 launch_norm_variant<64>(p, gain_q, gain_k, eps, blocks, stream);
+    count_launch();
+    return cudaGetLastError();
+}
 
 cudaError_t launch_rope_tables(float2 *t_tab, int64_t t_base, int n_t_frames, int n_t, float2 *h_tab,
                                int grid_h, float2 *w_tab, int grid_w, int n_hw, float theta, bool do_t,

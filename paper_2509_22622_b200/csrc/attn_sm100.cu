@@ -42,6 +42,8 @@
 // common exit where TMEM is released.
 #include <cuda_bf16.h>
 
+#include <atomic>
+
 #include "bounded_wait.cuh"
 #include "ll_internal.h"
 #include "ptx.cuh"
@@ -799,20 +801,26 @@ cudaError_t launch_attn_sm100(const AttnParams &p, int head_dim, const AttnMaps 
     if (p.n_ctas <= 0) return cudaSuccess;
     dim3 grid((unsigned)p.n_ctas);
     cudaError_t e;
-    // the in-kernel register reallocation assumes the launch allocation it was sized for
-    cudaFuncAttributes fa;
-    e = head_dim == 128 ? cudaFuncGetAttributes(&fa, attn_sm100_kernel<128>) : cudaFuncGetAttributes(&fa, attn_sm100_kernel<64>);
+    // Once per device and head size: the in-kernel register reallocation assumes the launch
+    // allocation it was sized for, and the kernel needs its dynamic shared memory opted in.
+    constexpr int kMaxDevices = 64;
+    static std::atomic<unsigned char> prepared[kMaxDevices][2];
+    int dev = 0;
+    e = cudaGetDevice(&dev);
     if (e != cudaSuccess) return e;
-    if (fa.numRegs != kLaunchRegs) return cudaErrorLaunchOutOfResources;
-    if (head_dim == 128) {
-        e = cudaFuncSetAttribute(attn_sm100_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg<128>::kSmemBytes);
+    const int which = head_dim == 128 ? 1 : 0;
+    if (dev < 0 || dev >= kMaxDevices || !prepared[dev][which].load(std::memory_order_acquire)) {
+        cudaFuncAttributes fa;
+        e = which ? cudaFuncGetAttributes(&fa, attn_sm100_kernel<128>) : cudaFuncGetAttributes(&fa, attn_sm100_kernel<64>);
         if (e != cudaSuccess) return e;
-        attn_sm100_kernel<128><<<grid, kThreads, Cfg<128>::kSmemBytes, stream>>>(p, maps);
-    } else {
-        e = cudaFuncSetAttribute(attn_sm100_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg<64>::kSmemBytes);
+        if (fa.numRegs != kLaunchRegs) return cudaErrorLaunchOutOfResources;
+        e = which ? cudaFuncSetAttribute(attn_sm100_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg<128>::kSmemBytes)
+                  : cudaFuncSetAttribute(attn_sm100_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg<64>::kSmemBytes);
         if (e != cudaSuccess) return e;
-        attn_sm100_kernel<64><<<grid, kThreads, Cfg<64>::kSmemBytes, stream>>>(p, maps);
+        if (dev >= 0 && dev < kMaxDevices) prepared[dev][which].store(1, std::memory_order_release);
     }
+    if (which) attn_sm100_kernel<128><<<grid, kThreads, Cfg<128>::kSmemBytes, stream>>>(p, maps);
+    else       attn_sm100_kernel<64><<<grid, kThreads, Cfg<64>::kSmemBytes, stream>>>(p, maps);
     count_launch();
     return cudaGetLastError();
 }

@@ -230,12 +230,12 @@ void plan_work(ll::AttnParams *p, int sms, long long all_cols, long long all_ste
     p->total_steps = steps;
     // steps each CTA gets as whole columns
     long long load[ll::kMaxCtas] = {};
-    {
-        int g = 0;
-        for (long long col = 0; col < whole_cols; ++col) {
-            while (col >= p->g[g].col_begin + (long long)p->heads * p->g[g].tiles) ++g;
-            load[col % p->n_ctas] += p->g[g].n_kt;
-        }
+    for (int g = 0; g < p->n_groups && p->n_ctas > 0; ++g) {
+        // of the columns [0, x) CTA i takes those congruent to i: (x + n - 1 - i) / n of them
+        const ll::AttnGroup &G = p->g[g];
+        const long long lo = G.col_begin, hi = G.col_begin + G.wave_cols, n = p->n_ctas;
+        for (int i = 0; i < p->n_ctas; ++i)
+            load[i] += ((hi + n - 1 - i) / n - (lo + n - 1 - i) / n) * G.n_kt;
     }
     // the highest level T that the shared steps can fill: sum over CTAs of max(0, T - load) <= steps
     auto fill = [&](long long T) {

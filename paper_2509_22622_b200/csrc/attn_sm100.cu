@@ -2,13 +2,16 @@
 //
 // Work decomposition.  A *column* is up to 256 query rows of one head (two
 // 128-row MMA tiles, "lanes" 0 and 1) and a *step* is one 128-key tile of that
-// column's visible cache rows.  One persistent CTA runs per SM.  As long as there
-// is a column for every CTA, columns are handed out whole: the CTAs of a head
-// then walk the keys in step and each K/V tile is fetched from HBM once and
-// shared through L2.  The steps of the columns left over are laid end to end and
-// cut into equal shares, so every SM does the same amount of work whatever the
-// number of columns.  A column whose steps fall into several CTAs is finished by
-// whichever of them arrives last:
+// column's visible cache rows.  One persistent CTA runs per SM.  The columns of
+// all query groups of a launch (one per chunk of queries, of one or several
+// streams) are numbered through.  As long as there is a column for every CTA,
+// columns are handed out whole: the CTAs of a head then walk the keys in step and
+// each K/V tile is fetched from HBM once and shared through L2.  The steps of the
+// columns left over are laid end to end and cut into one share per CTA, sized on
+// the host so that every SM ends up with the same number of steps whatever the
+// number and length of the columns (very short columns go out whole instead).
+// A column whose steps fall into several CTAs is finished by whichever of them
+// arrives last:
 // every part leaves its unnormalised O rows, reference maxima and sums in a
 // scratch slot, bumps the column's arrival counter, and the last one merges the
 // parts and writes the output.  Nothing waits on another CTA.

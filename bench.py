@@ -16,8 +16,13 @@ e2e        : the same with pinned host Q/K/V copied in and the output copied out
 roofline   : the attention kernel alone against the measured dense bf16 peak.
 cpu_baseline / --impl reference: the fp64 CPU oracle on a bounded sample of the
              same workload's query rows.
+extra.in_loop: the same step repeated for at least two seconds, whatever --steps
+             is: the GPU then sits at its power limit and the figure is the one a long
+             stream sees; the --steps region of a short run is a burst.
 With N > 1 every rank runs an independent replica (the path has no exchange
-step); value is the sum over ranks divided by the slowest rank's time.
+step); value is the sum over ranks divided by the slowest rank's time.  Started
+without a launcher (no WORLD_SIZE in the environment), --gpus N > 1 starts the N
+ranks itself.
 """
 from __future__ import annotations
 
@@ -152,13 +157,13 @@ def oracle_sample(target_seconds: float, steps: int = 1, warmup: int = 0):
     q, _, _ = synth.chunk_qkv(wl, n_fill - 1)
     qr = orc.rope_q(synth.bf16_bits_to_f64(q), (n_fill - 1) * C, wl.grid_h, wl.grid_w)
     # calibrate: rows the oracle gets through in about target_seconds
-    probe = synth.sample_rows(C * P, 2 * cores, seed=1)
+    probe = synth.sample_rows(C * P, 2 * cores, seed=1, edges=False)
     t0 = time.perf_counter()
     orc.attn(0, qr, (n_fill - 1) * C, rows=probe)
     per_row = (time.perf_counter() - t0) / len(probe)
     n_rows = int(max(cores, min(C * P, target_seconds / per_row)))
     n_rows = max(cores, n_rows // cores * cores)
-    rows = synth.sample_rows(C * P, n_rows, seed=2)
+    rows = synth.sample_rows(C * P, n_rows, seed=2, edges=False)
     times = []
     for i in range(warmup + steps):
         t0 = time.perf_counter()
@@ -212,6 +217,37 @@ def reduce_max(values, dist, device="cpu"):
 def whole_job_tflops(world: int, steps: int, flops_per_step: float, slowest_ms: float) -> float:
     """Every rank ran `steps` independent steps; the job took as long as its slowest rank."""
     return world * steps * flops_per_step / (slowest_ms * 1e-3) / 1e12
+
+
+def spawn_ranks(args, argv):
+    """`bench.py --gpus N` started by hand: launch N ranks of this script (one per GPU) and
+    pass rank 0's JSON line through.  Returns the launcher's exit code."""
+    import socket
+    with socket.socket() as sock:
+        sock.bind(("127.0.0.1", 0))
+        port = sock.getsockname()[1]
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", "--nproc-per-node", str(args.gpus),
+           "--master-addr", "127.0.0.1", "--master-port", str(port), os.path.abspath(__file__)] + list(argv)
+    return subprocess.call(cmd)
+
+
+def run_dry(args):
+    """The multi-rank plumbing without a GPU (gloo): every rank contributes made-up device
+    times, the line is assembled as in the real run.  Measures nothing; for tests."""
+    import torch.distributed as dist
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    if world > 1:
+        dist.init_process_group("gloo")
+    total_ms = 10.0 + rank                      # the last rank is the slowest
+    red = reduce_max([total_ms], dist if world > 1 else None, "cpu")
+    if world > 1:
+        dist.barrier()
+        dist.destroy_process_group()
+    if rank == 0:
+        print(json.dumps({"dry_run": True, "metric": "sink_window_attn_tflops", "n_gpus": world, "steps": args.steps,
+                          "ms_per_step": red[0] / args.steps,
+                          "value": whole_job_tflops(world, args.steps, attn_flops(WL), red[0])}))
 
 
 # ---------------------------------------------------------------------------
@@ -361,6 +397,53 @@ def run_ours(args):
     clocks = sampler.stop() if sampler else None
     cache.check_device()
 
+    # The same step for a fixed length of time, whatever --steps was: after about a second the
+    # GPU sits at its power limit and the SM clock settles below its maximum, which is what a
+    # long stream sees.  Its own clock samples are reported with it.
+    in_loop = None
+    if args.in_loop_seconds > 0:
+        slowest_ms = reduce_max([total_ms], dist, "cuda")[0]            # every rank runs the same number of steps
+        n_loop = max(args.steps, int(args.in_loop_seconds * 1e3 / max(slowest_ms / args.steps, 1e-3)) + 1)
+        loop_sampler = ClockSampler(local_rank) if rank == 0 else None
+        lev = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(n_loop)]
+        l0, l1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        barrier()
+        l0.record(stream)
+        for i in range(n_loop):
+            step(ev=lev[i])
+        l1.record(stream)
+        barrier()
+        loop_ms = l0.elapsed_time(l1)
+        # the second half of the loop: the clock has settled by then
+        half = lev[n_loop // 2:]
+        loop_attn_ms = sum(e[1].elapsed_time(e[2]) for e in half) / len(half)
+        loop_clocks = loop_sampler.stop() if loop_sampler else None
+        cache.check_device()
+        in_loop = {"steps": n_loop, "ms_total": loop_ms, "ms_per_step": loop_ms / n_loop,
+                   "attn_ms_per_launch_second_half": loop_attn_ms, "clocks": loop_clocks}
+
+    # The append kernel alone: launches back to back on rotating layers and input sets (each
+    # overwrites its layer's newest chunk in place), one pair of events around all of them, so
+    # that no launch gap is counted.
+    n_app = 200
+    a0, a1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+
+    def appends(n):
+        for i in range(n):
+            layer = i % N_LAYERS
+            q, k, v = dev_sets[(i + i // N_LAYERS) % N_INPUT_SETS]
+            cache.rope_append_kv(layer, q, k, v, cache.state(layer)["end"] - C, wl.grid_h, wl.grid_w, wl.rope_theta,
+                                 q_roped)
+    appends(8)
+    barrier()
+    a0.record(stream)
+    appends(n_app)
+    a1.record(stream)
+    barrier()
+    append_b2b_ms = a0.elapsed_time(a1) / n_app
+    cache.check_device()
+
+
     # recache of the full window (one launch pair), reported beside the headline
     n_w = wl.window_frames
     rq, rk, rv = (dev(t) for t in synth.chunk_qkv(wl, 200, pass_id=synth.RECACHE_PASS, n_frames=n_w, stream=rank))
@@ -452,7 +535,9 @@ def run_ours(args):
         others["cross_attn_512_keys"] = {"us": ms * 1e3, "tflops": 4.0 * nq * n_prompt * D * H / ms / 1e9}
         cache.check_device()
 
-    total_ms, e2e_ms, attn_ms, append_ms = reduce_max([total_ms, e2e_ms, attn_ms, append_ms], dist, "cuda")
+    loop_vals = [in_loop["ms_total"], in_loop["attn_ms_per_launch_second_half"]] if in_loop else [0.0, 0.0]
+    total_ms, e2e_ms, attn_ms, append_ms, append_b2b_ms, loop_total_ms, loop_attn_ms = reduce_max(
+        [total_ms, e2e_ms, attn_ms, append_ms, append_b2b_ms] + loop_vals, dist, "cuda")
     if rank != 0:
         if dist is not None:
             dist.destroy_process_group()
@@ -464,7 +549,18 @@ def run_ours(args):
     value = whole_job_tflops(world, args.steps, flops_step, total_ms)
     e2e_value = whole_job_tflops(world, args.steps, flops_step, e2e_ms)
     attn_tflops = flops_step / (attn_ms * 1e-3) / 1e12
-    append_gbs = append_bytes(wl) / (append_ms * 1e-3) / 1e9
+    append_gbs = append_bytes(wl) / (append_b2b_ms * 1e-3) / 1e9
+    if in_loop:
+        n_loop = in_loop["steps"]
+        in_loop.update({
+            "ms_total": loop_total_ms, "ms_per_step": loop_total_ms / n_loop,
+            "value_tflops": whole_job_tflops(world, n_loop, flops_step, loop_total_ms),
+            "attn_ms_per_launch_second_half": loop_attn_ms,
+            "attn_tflops": flops_step / (loop_attn_ms * 1e-3) / 1e12,
+            "attn_frac_of_burst_peak": flops_step / (loop_attn_ms * 1e-3) / 1e12 / peaks["bf16_tflops"],
+            "attn_frac_of_sustained_peak": flops_step / (loop_attn_ms * 1e-3) / 1e12 / peaks["bf16_tflops_sustained"],
+            "note": "at least %.1f s of back-to-back steps; sw_power_cap in its clock record is expected and kept; "
+                    "the --steps region above is a burst when it is short" % args.in_loop_seconds})
     ms_per_step = total_ms / args.steps
     in_bytes = 3 * nq * H * D * 2
     cpu = None
@@ -492,10 +588,15 @@ def run_ours(args):
                      "traffic": traffic.get("attn_sm100_kernel")},
         "roofline_append": {"bound": "hbm", "kernel": "rope_append_kernel<128>", "achieved": append_gbs,
                             "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": append_gbs / peaks["hbm_gbs"],
-                            "peak_kind": "of %s (copy)" % peak_kind, "ms_per_launch": append_ms,
-                            "traffic": traffic.get("rope_append_kernel")},
+                            "peak_kind": "of %s (copy)" % peak_kind, "ms_per_launch": append_b2b_ms,
+                            "how": "%d launches back to back on rotating layers between two events" % n_app,
+                            "ms_between_events_inside_a_step": append_ms,
+                            "traffic": traffic.get("rope_append_kernel"),
+                            "traffic_note": "DRAM bytes under the profiler are below the 86.3 MB the kernel moves: "
+                                            "the cache rows it wrote are still in L2 when it ends"},
         "cpu_baseline": cpu,
-        "extra": {"latent_frames_per_s_30_layers_5_passes": C / (150 * ms_per_step * 1e-3),
+        "extra": {"in_loop": in_loop,
+                  "latent_frames_per_s_30_layers_5_passes": C / (150 * ms_per_step * 1e-3),
                   "latent_frames_per_s_30_layers_4_passes": C / (120 * ms_per_step * 1e-3),
                   "recache_ms_per_layer": recache_ms,
                   "recache_tflops": 9 * attn_flops(wl) / 4 / (recache_ms * 1e-3) / 1e12,
@@ -514,9 +615,16 @@ def main():
     ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--in-loop-seconds", type=float, default=2.0,
+                    help="length of the extra power-limited leg reported as extra.in_loop (0 = skip)")
+    ap.add_argument("--dry-run", action="store_true", help="multi-rank plumbing only, on CPU (gloo); measures nothing")
     args = ap.parse_args()
+    if args.impl == "ours" and args.gpus > 1 and "WORLD_SIZE" not in os.environ:
+        sys.exit(spawn_ranks(args, sys.argv[1:]))
     if args.impl == "reference":
         run_reference(args)
+    elif args.dry_run:
+        run_dry(args)
     else:
         run_ours(args)
 

@@ -119,7 +119,12 @@ int ll_cache_kv_offset(const ll_cache *cache, int layer, int which, int head, si
  * n_t = D/2 - 2*n_h pairs; pair j is elements (2j, 2j+1); pair i of an axis with
  * n_a pairs turns by pos * rope_theta^(-i/n_a); t is the absolute frame index.
  * K rows are stored rotated, V rows verbatim.  The arithmetic is fp32 on
- * fp64-accurate sine/cosine tables kept in the aux block. */
+ * fp64-accurate sine/cosine tables kept in the aux block.  The tables are
+ * rebuilt only when the grid, rope_theta or the resident range of frames
+ * changes - until a call on the handle is recorded into a CUDA graph: from then
+ * on every append of the handle, recorded or not, enqueues the small table
+ * kernel in front of itself, so a replayed graph never reads tables that a
+ * later call has moved. */
 int ll_rope_append_kv(ll_cache *cache, int layer, const ll_bf16 *q, const ll_bf16 *k,
                       const ll_bf16 *v, int64_t frame_start, int n_frames,
                       int grid_h, int grid_w, float rope_theta, ll_bf16 *q_out,
@@ -229,7 +234,12 @@ int ll_recache(ll_cache *cache, int layer, const ll_bf16 *q, const ll_bf16 *k,
                ll_bf16 *q_out, ll_bf16 *out, float *lse_out, ll_stream stream);
 
 /* Forget everything in every layer (Algorithm 2 "C <- []"): end = 0, all slots
- * empty, counters kept.  Stored bytes are not cleared. */
+ * empty, counters kept.  Stored bytes are not cleared: the next stream writes
+ * over them slot by slot, and until a slot is rewritten its stale rows may
+ * still be fetched by the ragged last tile of a neighbouring slot's keys (they
+ * are masked out of the softmax but pass through the PV product with weight
+ * zero), so they must hold finite numbers.  Rows written by this library from
+ * finite inputs always do. */
 int ll_cache_reset(ll_cache *cache);
 
 /* 3-D RoPE of a query tensor without any device allocation.  (The paper has no
@@ -291,62 +301,10 @@ int ll_cache_set_dry_run(ll_cache *cache, int on);
 
 /* Synchronise `stream`, read the aux status words and clear them.  LL_OK, or
  * LL_ERR_DEVICE_TIMEOUT if a kernel abandoned a bounded wait (its outputs are
- * then invalid); ll_last_error() names the role and barrier. */
+ * then invalid); ll_last_error() names the role and barrier.  On a time-out
+ * the call also zeroes the arrival counters of the split-column merge, which
+ * the abandoned launch left mid-count, so the handle can be used again. */
 int ll_cache_device_status(ll_cache *cache, ll_stream stream);
-
-/* Test-only triage kernel: the same computation as ll_sink_window_attn with one
- * thread block per (query row, head) and plain fp32 FMAs.  Never used by the
- * calls above. */
-int ll_debug_attn_simt(ll_cache *cache, int layer, const ll_bf16 *q_roped,
-                       int64_t q_frame_start, int n_q_frames, ll_bf16 *out,
-                       float *lse_out, ll_stream stream);
-
-/* Test-only: exercise the bounded-wait machinery the kernels share.  Enqueues a
- * one-warp kernel that waits on a barrier nobody completes, gives up after
- * limit_ms (1..1000), records the time-out in the status words and returns
- * normally; the next ll_cache_device_status then reports
- * LL_ERR_DEVICE_TIMEOUT (barrier 99, iteration 7) and clears the record.
- * Attention launches enqueued while the record stands skip their work. */
-int ll_debug_wait_timeout(ll_cache *cache, int limit_ms, ll_stream stream);
-
-/* How the attention kernel would divide the work of a call, given the current
- * state (host-only; for tests and tuning).  recache = 0: ll_sink_window_attn of
- * the newest chunk; recache = 1: ll_recache of the resident window.  sm_count > 0
- * overrides the SM count of the storage's device (148 when no storage is bound).
- * Per query group g: tiles[g] query tiles of 256 rows per head (so heads *
- * tiles[g] columns), n_kt[g] key tiles (steps) per column.  The columns of all
- * groups are numbered through (group g's first is col_begin[g]); the first
- * n_waves * n_ctas go out whole, CTA i taking columns i, i + n_ctas, ... (of
- * group g these are its first wave_cols[g]).  The steps of the other columns
- * are laid end to end (group g's from step_begin[g]) and cut into n_shares
- * shares: CTA i takes shared steps [share_begin[k], share_begin[k + 1]) with
- * k = share_of_cta[i], or none when that is -1.  Shares are sized so that
- * whole columns plus share come to the same number of steps on every CTA.
- * When the columns are short (merging the parts of a split column would cost
- * more than splitting saves) nothing is shared: the last wave is partial,
- * columns numbered all_cols and up do not exist, and n_shares is 0.
- * ll_debug_attn_plan_batched: the same for ll_sink_window_attn_batched of the
- * newest chunk of every item (only cache and layer of an item are read). */
-#define LL_MAX_GROUPS 24
-#define LL_MAX_CTAS 160
-typedef struct ll_attn_plan {
-    int32_t n_ctas;
-    int32_t n_groups;
-    int32_t heads;
-    int32_t n_waves;
-    int32_t n_shares;
-    int32_t all_cols;
-    int64_t shared_steps;
-    int32_t tiles[LL_MAX_GROUPS];
-    int32_t n_kt[LL_MAX_GROUPS];
-    int32_t col_begin[LL_MAX_GROUPS];
-    int32_t wave_cols[LL_MAX_GROUPS];
-    int64_t step_begin[LL_MAX_GROUPS];
-    int32_t share_begin[LL_MAX_CTAS + 1];
-    int32_t share_of_cta[LL_MAX_CTAS];
-} ll_attn_plan;
-int ll_debug_attn_plan(ll_cache *cache, int layer, int recache, int sm_count, ll_attn_plan *out);
-int ll_debug_attn_plan_batched(const ll_attn_item *items, int n_items, int sm_count, ll_attn_plan *out);
 
 /* Kernel launches made by this process through the library so far. */
 int64_t ll_launch_count(void);

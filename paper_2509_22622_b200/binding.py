@@ -86,7 +86,7 @@ class LLError(RuntimeError):
 
 _lib = None
 
-# name -> (restype, argtypes); also the list of symbols include/llattn.h declares
+# name -> (restype, argtypes); also the list of symbols include/llattn.h and include/llattn_debug.h declare
 SIGNATURES = {
     "ll_cache_create": (C.c_int, [C.c_int] * 7 + [C.POINTER(C.c_void_p)]),
     "ll_cache_destroy": (None, [C.c_void_p]),
@@ -122,6 +122,7 @@ SIGNATURES = {
     "ll_debug_wait_timeout": (C.c_int, [C.c_void_p, C.c_int, C.c_void_p]),
     "ll_debug_attn_plan": (C.c_int, [C.c_void_p, C.c_int, C.c_int, C.c_int, C.POINTER(ll_attn_plan)]),
     "ll_debug_attn_plan_batched": (C.c_int, [C.POINTER(ll_attn_item), C.c_int, C.c_int, C.POINTER(ll_attn_plan)]),
+    "ll_debug_aux_layout": (C.c_int, [C.c_void_p] + [C.POINTER(C.c_size_t)] * 4),
     "ll_launch_count": (C.c_int64, []),
     "ll_last_error": (C.c_char_p, []),
     "ll_version": (C.c_char_p, []),
@@ -298,6 +299,13 @@ def ll_debug_attn_plan_batched(handles_and_layers, sm_count=0) -> ll_attn_plan:
     plan = ll_attn_plan()
     _check(lib().ll_debug_attn_plan_batched(arr, len(handles_and_layers), sm_count, C.byref(plan)))
     return plan
+
+
+def ll_debug_aux_layout(h):
+    """(status_offset, status_bytes, counters_offset, counters_bytes) inside the bound storage."""
+    v = [C.c_size_t() for _ in range(4)]
+    _check(lib().ll_debug_aux_layout(h, *[C.byref(x) for x in v]))
+    return tuple(x.value for x in v)
 
 
 def ll_launch_count() -> int:

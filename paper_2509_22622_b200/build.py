@@ -10,7 +10,8 @@ ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libllattn.so")
 SOURCES = ["ll_host.cu", "rope_append.cu", "attn_sm100.cu", "attn_simt.cu", "rope_static.cu"]
-HEADERS = ["ll_internal.h", "ptx.cuh", "bounded_wait.cuh", os.path.join(ROOT, "include", "llattn.h")]
+HEADERS = ["ll_internal.h", "ptx.cuh", "bounded_wait.cuh", "rope_math.cuh", os.path.join(ROOT, "include", "llattn.h"),
+           os.path.join(ROOT, "include", "llattn_debug.h")]
 
 NVCC_FLAGS = [
     "-std=c++17", "-O3", "-lineinfo",

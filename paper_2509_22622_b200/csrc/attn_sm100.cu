@@ -72,10 +72,7 @@ constexpr int kProducerRegs = 64;
 static_assert(kSoftmaxWarps * kSoftmaxRegs + (kThreads / 32 - kSoftmaxWarps) * kProducerRegs <= (kThreads / 32) * kLaunchRegs,
               "setmaxnreg targets exceed the CTA's register allocation");
 // 8-key groups (bit k of 16 per 128-key tile) whose exponentials use the cubic
-#ifndef LL_POLY_MASK
-#define LL_POLY_MASK 0x8888u
-#endif
-constexpr uint32_t kPolyMask = LL_POLY_MASK;
+constexpr uint32_t kPolyMask = 0x8888u;
 
 template <int D>
 struct Cfg {

@@ -125,18 +125,39 @@ int visible_ranges(const ll_cache *c, int layer, int64_t q_frame_start, int64_t 
 }
 
 // Make sure the RoPE tables cover frames [f0, f1) and this grid/theta.
+//
+// Normally the tables are rebuilt only when the grid, theta or the resident window of
+// kTTabFrames frames changes, and the host remembers what is resident.  A call recorded
+// into a CUDA graph cannot rely on that memory: the graph may be replayed after other calls
+// on the handle have moved the tables, and a replay moves them back without the host
+// seeing it.  So from the first captured call on, every append of the handle (recorded or
+// not) brings its own tables: the table kernel is enqueued in front of it, for exactly the
+// frames it needs.
 int ensure_tables(ll_cache *c, int64_t f0, int64_t f1, int gh, int gw, float theta, cudaStream_t stream)
 {
     int n_t, n_h;
     rope_split(c->D, &n_t, &n_h);
+    cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
+    if (cudaStreamIsCapturing(stream, &cap) != cudaSuccess) {
+        cap = cudaStreamCaptureStatusNone;
+        (void)cudaGetLastError();
+    }
+    if (cap == cudaStreamCaptureStatusActive) c->tables_per_call = true;
     bool do_hw = !(c->hw_valid && c->tab_gh == gh && c->tab_gw == gw && c->tab_theta == theta);
     bool do_t = do_hw || c->t_base < 0 || f0 < c->t_base || f1 > c->t_base + ll::kTTabFrames;
-    if (!do_t && !do_hw) return LL_OK;
     int64_t base = do_t ? f0 / ll::kTTabAlign * ll::kTTabAlign : c->t_base;
+    int n_frames = ll::kTTabFrames;
+    if (c->tables_per_call) {
+        do_t = do_hw = true;
+        base = f0;
+        n_frames = (int)(f1 - f0);
+        if (n_frames > ll::kTTabFrames) return fail(LL_ERR_UNSUPPORTED_SHAPE, "more than %d frames in one call", ll::kTTabFrames);
+    }
+    if (!do_t && !do_hw) return LL_OK;
     float2 *t_tab = reinterpret_cast<float2 *>(c->storage + c->off_ttab);
     float2 *h_tab = reinterpret_cast<float2 *>(c->storage + c->off_hwtab);
     float2 *w_tab = h_tab + (size_t)gh * n_h;
-    cudaError_t e = ll::launch_rope_tables(t_tab, base, ll::kTTabFrames, n_t, h_tab, gh, w_tab, gw, n_h,
+    cudaError_t e = ll::launch_rope_tables(t_tab, base, n_frames, n_t, h_tab, gh, w_tab, gw, n_h,
                                            theta, do_t, do_hw, stream);
     if (e != cudaSuccess) return cuda_fail(e, "rope table kernel");
     c->t_base = base;
@@ -453,7 +474,7 @@ int ll_cache_create(int layers, int heads, int head_dim, int tokens_per_frame, i
     c->off_hwtab = align_up(c->off_ttab + (size_t)ll::kTTabFrames * n_t * sizeof(float2), 256);
     // grid_h + grid_w <= tokens_per_frame + 1 for any grid with grid_h*grid_w == tokens_per_frame
     c->off_counters = align_up(c->off_hwtab + (size_t)(tokens_per_frame + 1) * n_h * sizeof(float2), 256);
-    c->off_partial = align_up(c->off_counters + (size_t)ll::kMaxCtas * ll::kSlabs * sizeof(uint32_t), 1024);
+    c->off_partial = align_up(c->off_counters + ll::counters_bytes(), 1024);
     c->aux_bytes = align_up(c->off_partial + 2 * (size_t)ll::kMaxCtas * ll::attn_slot_bytes(head_dim), 1024);
     c->kv_bytes = (size_t)heads * rows * head_dim * sizeof(ll_bf16);
     *out = c;
@@ -843,6 +864,17 @@ int ll_debug_wait_timeout(ll_cache *c, int limit_ms, ll_stream stream)
     return e == cudaSuccess ? LL_OK : cuda_fail(e, "wait probe kernel");
 }
 
+int ll_debug_aux_layout(const ll_cache *c, size_t *status_offset, size_t *status_bytes, size_t *counters_offset,
+                        size_t *counters_bytes)
+{
+    if (!c) return fail(LL_ERR_INVALID_ARG, "null handle");
+    if (status_offset) *status_offset = c->off_status;
+    if (status_bytes) *status_bytes = ll::kStatusWords * sizeof(uint32_t);
+    if (counters_offset) *counters_offset = c->off_counters;
+    if (counters_bytes) *counters_bytes = ll::counters_bytes();
+    return LL_OK;
+}
+
 int ll_cache_reset(ll_cache *c)
 {
     if (!c) return fail(LL_ERR_INVALID_ARG, "null handle");
@@ -917,8 +949,12 @@ int ll_cache_device_status(ll_cache *c, ll_stream stream)
     e = cudaMemcpy(w, c->storage + c->off_status, sizeof w, cudaMemcpyDeviceToHost);
     if (e != cudaSuccess) return cuda_fail(e, "cudaMemcpy(status)");
     if (w[0] == ll::kStatusOk) return LL_OK;
+    // A CTA that gave up, and every CTA that then skipped its work, never made its arrival on
+    // the split-column counters, so the counters of that launch are left mid-count: clear them
+    // together with the record, or the next launch that splits a column would merge too early.
     e = cudaMemset(c->storage + c->off_status, 0, sizeof w);
-    if (e != cudaSuccess) return cuda_fail(e, "cudaMemset(status)");
+    if (e == cudaSuccess) e = cudaMemset(c->storage + c->off_counters, 0, ll::counters_bytes());
+    if (e != cudaSuccess) return cuda_fail(e, "cudaMemset(status, counters)");
     return fail(LL_ERR_DEVICE_TIMEOUT,
                 "a kernel gave up on a bounded wait: code %u role %u barrier %u iteration %u block (%u,%u,%u)",
                 w[0], w[1], w[2], w[3], w[4], w[5], w[6]);

@@ -9,6 +9,7 @@
 #include <vector>
 
 #include "llattn.h"
+#include "llattn_debug.h"
 
 namespace ll {
 
@@ -58,6 +59,9 @@ struct AttnGroup {
     int k_start[LL_MAX_RANGES];       // visible cache-row runs
     int k_len[LL_MAX_RANGES];
 };
+
+// Bytes of the arrival counters of the split-column merge (one per share and 16-row slab).
+inline size_t counters_bytes() { return (size_t)kMaxCtas * kSlabs * sizeof(uint32_t); }
 
 // Bytes of one partial-result slot: both tiles' unnormalised O rows in fp32 plus
 // (reference max, sum) per row.
@@ -154,4 +158,5 @@ struct ll_cache {
     int tab_gh = 0, tab_gw = 0;
     float tab_theta = 0.f;
     int64_t t_base = -1;
+    bool tables_per_call = false;     // set by the first captured call: every append then rebuilds its tables
 };

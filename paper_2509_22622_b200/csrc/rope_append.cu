@@ -10,6 +10,7 @@
 #include <cuda_bf16.h>
 
 #include "ll_internal.h"
+#include "rope_math.cuh"
 
 namespace ll {
 
@@ -49,17 +50,6 @@ __global__ void rope_table_kernel(float2 *t_tab, long long t_base, int n_t_frame
 
 __device__ __forceinline__ uint4 ld16(const ll_bf16 *p) { return *reinterpret_cast<const uint4 *>(p); }
 __device__ __forceinline__ void st16(ll_bf16 *p, uint4 v) { *reinterpret_cast<uint4 *>(p) = v; }
-
-// Rotate one packed pair (lo = element 2j, hi = element 2j+1) in fp32.
-__device__ __forceinline__ uint32_t rotate_pair(uint32_t packed, float2 cs)
-{
-    float a = __uint_as_float(packed << 16);
-    float b = __uint_as_float(packed & 0xffff0000u);
-    float r0 = fmaf(a, cs.x, -(b * cs.y));
-    float r1 = fmaf(a, cs.y, b * cs.x);
-    __nv_bfloat162 o = __floats2bfloat162_rn(r0, r1);   // .x (low half) = r0
-    return *reinterpret_cast<uint32_t *>(&o);
-}
 
 __device__ __forceinline__ uint4 rotate_vec(uint4 x, const float2 (&cs)[4])
 {

@@ -21,6 +21,7 @@
 #include <mutex>
 
 #include "ll_internal.h"
+#include "rope_math.cuh"
 
 namespace {
 
@@ -40,20 +41,12 @@ static __device__ __align__(256) float2 g_rope_scratch[kTEntries + kHwEntries];
 std::mutex g_setup_mutex;
 float2 *g_scratch_addr[kMaxDevices];   // device address of g_rope_scratch, per device ordinal
 
-__device__ __forceinline__ uint32_t rotate_pair_q(uint32_t packed, float2 cs)
-{
-    float a = __uint_as_float(packed << 16);
-    float b = __uint_as_float(packed & 0xffff0000u);
-    float r0 = fmaf(a, cs.x, -(b * cs.y));
-    float r1 = fmaf(a, cs.y, b * cs.x);
-    __nv_bfloat162 o = __floats2bfloat162_rn(r0, r1);
-    return *reinterpret_cast<uint32_t *>(&o);
-}
-
-// One thread rotates one 16-byte vector (4 pairs) of one head row of one token.
+// One thread rotates one 16-byte vector (4 pairs) of one head row of one token.  q_out may be
+// q itself (each thread reads its vector before it writes it), so neither pointer is
+// declared free of aliases.
 template <int D>
 __global__ void __launch_bounds__(256)
-rope_q_static_kernel(const ll_bf16 *__restrict__ q, ll_bf16 *__restrict__ q_out, const float2 *t_tab,
+rope_q_static_kernel(const ll_bf16 *q, ll_bf16 *q_out, const float2 *t_tab,
                      const float2 *h_tab, const float2 *w_tab, long long n_tokens, int heads, int P, int grid_w,
                      int n_t, int n_h)
 {
@@ -78,10 +71,10 @@ rope_q_static_kernel(const ll_bf16 *__restrict__ q, ll_bf16 *__restrict__ q_out,
     }
     const size_t off = (size_t)row * D + (size_t)vec * 8;
     uint4 v = *reinterpret_cast<const uint4 *>(q + off);
-    v.x = rotate_pair_q(v.x, cs[0]);
-    v.y = rotate_pair_q(v.y, cs[1]);
-    v.z = rotate_pair_q(v.z, cs[2]);
-    v.w = rotate_pair_q(v.w, cs[3]);
+    v.x = ll::rotate_pair(v.x, cs[0]);
+    v.y = ll::rotate_pair(v.y, cs[1]);
+    v.z = ll::rotate_pair(v.z, cs[2]);
+    v.w = ll::rotate_pair(v.w, cs[3]);
     *reinterpret_cast<uint4 *>(q_out + off) = v;
 }
 

@@ -123,25 +123,24 @@ def chunk_qkv(wl: Workload, chunk: int, layer: int = 0, pass_id: int = 0,
     return q, k, v
 
 
-def sample_rows(n_rows: int, n_samples: int, tile: int = 128, seed: int = 0) -> np.ndarray:
+def sample_rows(n_rows: int, n_samples: int, tile: int = 128, seed: int = 0, edges: bool = True) -> np.ndarray:
     """Query rows to check at sizes where the oracle cannot do every row.
 
-    Always holds the first and last row of every ``tile``-row tile that the
-    sampling budget allows, the ragged last tile's ends, and random rows.
+    With ``edges`` (the default) the result always holds the first and the last
+    row of every ``tile``-row tile, the ragged last tile's ends included, however
+    small ``n_samples`` is; random rows then fill it up to ``n_samples``.  With
+    ``edges=False`` it is ``n_samples`` random rows plus the first and last one
+    (for timing samples, where the count matters and the placement does not).
     """
     must = {0, n_rows - 1}
-    edges = []
-    for t0 in range(0, n_rows, tile):
-        edges += [t0, min(t0 + tile, n_rows) - 1]
+    if edges:
+        for t0 in range(0, n_rows, tile):
+            must.update((t0, min(t0 + tile, n_rows) - 1))
     rng = np.random.default_rng([seed, n_rows, n_samples])
-    if len(edges) > n_samples // 2:
-        edges = list(rng.choice(np.asarray(edges), size=n_samples // 2, replace=False))
-    must.update(int(e) for e in edges)
-    last_tile0 = (n_rows - 1) // tile * tile
-    must.update((last_tile0, n_rows - 1))
     rest = n_samples - len(must)
-    if rest > 0:
+    while rest > 0:
         must.update(int(r) for r in rng.integers(0, n_rows, size=rest))
+        rest = min(n_samples, n_rows) - len(must)
     return np.asarray(sorted(must), dtype=np.int64)
 
 

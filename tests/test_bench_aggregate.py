@@ -1,8 +1,11 @@
 """The benchmark's multi-rank path on CPU: two gloo ranks, replicas only.  Each
 rank reports its own device time; the job's time is the slowest rank's and the
 work is the sum over ranks."""
+import json
 import os
 import socket
+import subprocess
+import sys
 
 import torch.distributed as dist
 import torch.multiprocessing as mp
@@ -46,3 +49,21 @@ def test_two_rank_max_over_ranks_and_whole_job_value():
 
 def test_single_rank_reduce_is_identity():
     assert bench.reduce_max([1.5, 2.5], None) == [1.5, 2.5]
+
+
+def test_gpus_flag_starts_the_ranks_itself():
+    """`bench.py --gpus 2` without a launcher around it starts two ranks (here on CPU, gloo,
+    with made-up device times) and prints one line for the whole job: the slowest rank's time,
+    the work of both."""
+    env = {k: v for k, v in os.environ.items()
+           if k not in ("WORLD_SIZE", "RANK", "LOCAL_RANK", "MASTER_ADDR", "MASTER_PORT")}
+    root = os.path.dirname(os.path.abspath(bench.__file__))
+    r = subprocess.run([sys.executable, os.path.join(root, "bench.py"), "--gpus", "2", "--steps", "5", "--dry-run"],
+                       env=env, capture_output=True, text=True, timeout=300)
+    assert r.returncode == 0, r.stderr[-2000:]
+    lines = [json.loads(l) for l in r.stdout.splitlines() if l.startswith("{")]
+    assert len(lines) == 1
+    line = lines[0]
+    assert line["n_gpus"] == 2 and line["dry_run"] is True
+    assert abs(line["ms_per_step"] - 11.0 / 5) < 1e-9                 # rank 1 reported 11 ms, rank 0 10 ms
+    assert abs(line["value"] - bench.whole_job_tflops(2, 5, bench.attn_flops(bench.WL), 11.0)) < 1e-9

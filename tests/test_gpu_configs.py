@@ -10,7 +10,7 @@ import torch
 from paper_2509_22622_b200 import binding as B
 from paper_2509_22622_b200 import synth
 
-from gpu_util import bits, check_attn, dev, f64, new_cache
+from gpu_util import bits, check_attn, check_attn_outliers, dev, f64, new_cache
 
 pytestmark = pytest.mark.gpu
 
@@ -42,13 +42,23 @@ class DevicePool:
         return self.sets[self.pool.index(*key)]
 
 
-def check_rows(orc, cache_out, q_bits, frame_start, wl, n_rows, seed, orc_abs=None):
+# Rows the oracle evaluates per checked call: the first and last row of every 128-row
+# query tile (74 of them at 4680 rows) plus random rows.
+N_ROWS = 256
+
+
+def check_rows(orc, cache_out, q_bits, frame_start, wl, seed, orc_abs=None, orc_truth=None, label=""):
     nq = wl.chunk_tokens
-    rows = synth.sample_rows(nq, n_rows, seed=seed)
+    rows = synth.sample_rows(nq, N_ROWS, seed=seed)
     qr = orc.rope_q(F64(q_bits), frame_start, wl.grid_h, wl.grid_w, wl.rope_theta)
     want, _ = orc.attn(0, qr, frame_start, rows=rows)
-    scale = orc_abs.attn(0, qr, frame_start, rows=rows)[0] if orc_abs else None
-    return check_attn(f64(cache_out)[rows], want, scale=scale)
+    got = f64(cache_out)[rows]
+    if orc_abs is None:
+        return check_attn(got, want)
+    scale = orc_abs.attn(0, qr, frame_start, rows=rows)[0]
+    q_true = orc_truth.rope_q(F64(q_bits), frame_start, wl.grid_h, wl.grid_w, wl.rope_theta)
+    truth = orc_truth.attn(0, q_true, frame_start, rows=rows)[0]
+    return check_attn_outliers(got, want, scale, truth, label=label)
 
 
 # ---------------------------------------------------------------------------
@@ -73,7 +83,7 @@ def test_config1_streamed_layer(oracle_mod):
         orc.append(0, F64(k), F64(v), chunk * C, wl.grid_h, wl.grid_w, wl.rope_theta)
         assert cache.state()["slot_frame"] == list(orc.state()["slot_frame"])
         if chunk in (0, 2, 3, 6):
-            e = check_rows(orc, out, q, chunk * C, wl, 96, chunk)
+            e = check_rows(orc, out, q, chunk * C, wl, chunk)
             worst = (max(worst[0], e[0]), max(worst[1], e[1]))
     print("parity config1: worst max-abs %.3e mean-abs %.3e" % worst)
     cache.close()
@@ -109,7 +119,7 @@ def run_full_stack(oracle_mod, wl, dpool, check_layers, check_chunks):
             q, k, v = dpool.pool.get(chunk, layer, passes - 1)
             orcs[layer].append(0, F64(k), F64(v), chunk * C, wl.grid_h, wl.grid_w, wl.rope_theta)
             if chunk in check_chunks:
-                check_rows(orcs[layer], kept[(layer, chunk)], q, chunk * C, wl, 48, chunk)
+                check_rows(orcs[layer], kept[(layer, chunk)], q, chunk * C, wl, chunk)
     assert cache.state(0)["overwrites"] == wl.n_chunks * (passes - 1)
     cache.close()
     return kept
@@ -198,19 +208,19 @@ def test_config3_long_stream(oracle_mod):
     for c in range(7, 11):
         q, k, v = pool.get(c, probe_layer, last)
         orc.append(0, F64(k), F64(v), c * C, wl.grid_h, wl.grid_w, wl.rope_theta)
-    check_rows(orc, kept[(probe_layer, 10)], q, 10 * C, wl, 48, 10)
+    check_rows(orc, kept[(probe_layer, 10)], q, 10 * C, wl, 10)
     # (b) the recache before chunk 40 rebuilds chunks 37..39, then chunk 40 attends over them
     orc.seek(0, 37 * C)
     for c in range(37, 40):
         q, k, v = pool.get(c, probe_layer, last)
         orc.append(0, F64(k), F64(v), c * C, wl.grid_h, wl.grid_w, wl.rope_theta)
     rq, rk, rv = rpool.get(40, probe_layer)
-    rows = synth.sample_rows(W * wl.tokens_per_frame, 72, tile=256, seed=40)
+    rows = synth.sample_rows(W * wl.tokens_per_frame, 384, seed=40)
     _, want, _ = orc.recache(0, F64(rq), F64(rk), F64(rv), W, wl.grid_h, wl.grid_w, wl.rope_theta, rows=rows)
     check_attn(f64(kept["recache"])[rows], want)
     q, k, v = pool.get(40, probe_layer, last)
     orc.append(0, F64(k), F64(v), 40 * C, wl.grid_h, wl.grid_w, wl.rope_theta)
-    check_rows(orc, kept[(probe_layer, 40)], q, 40 * C, wl, 48, 40)
+    check_rows(orc, kept[(probe_layer, 40)], q, 40 * C, wl, 40)
     orc.close()
     # (c) the last chunk of the 240 s stream, last layer
     orc = make_oracle(oracle_mod, wl)
@@ -220,7 +230,7 @@ def test_config3_long_stream(oracle_mod):
     for c in range(316, 320):
         q, k, v = pool.get(c, 29, last)
         orc.append(0, F64(k), F64(v), c * C, wl.grid_h, wl.grid_w, wl.rope_theta)
-    check_rows(orc, kept[(29, 319)], q, 319 * C, wl, 48, 319)
+    check_rows(orc, kept[(29, 319)], q, 319 * C, wl, 319)
     assert list(orc.state()["slot_frame"]) == cache.state(29)["slot_frame"]
     cache.close()
 
@@ -264,20 +274,24 @@ def test_config4_ragged_streams_window_sweep(oracle_mod, W, batched):
         # reference: storage-faithful oracle; a twin with |V| gives the error scale sum_j p_j |v_j|
         orc = make_oracle(oracle_mod, wl, faithful=True)
         orc_abs = make_oracle(oracle_mod, wl, faithful=True)
+        orc_truth = make_oracle(oracle_mod, wl, faithful=False)       # unrounded rotations: the raw figure
         first = max(1, pos + 1 - W // C)
         for chunk in [0] + list(range(first, pos + 1)):
             if chunk == first and pos > 0:
-                orc.seek(0, first * C)
-                orc_abs.seek(0, first * C)
+                for o in (orc, orc_abs, orc_truth):
+                    o.seek(0, first * C)
             _, k, v = pool.get(chunk, 0, 0, stream)
             orc.append(0, F64(k), F64(v), chunk * C, wl.grid_h, wl.grid_w, wl.rope_theta)
             orc_abs.append(0, F64(k), np.abs(F64(v)), chunk * C, wl.grid_h, wl.grid_w, wl.rope_theta)
+            orc_truth.append(0, F64(k), F64(v), chunk * C, wl.grid_h, wl.grid_w, wl.rope_theta)
         assert cache.state()["slot_frame"] == list(orc.state()["slot_frame"]), (W, pos)
         q, _, _ = pool.get(pos, 0, 0, stream)
-        e = check_rows(orc, out, q, pos * C, wl, 32, pos, orc_abs=orc_abs)
+        e = check_rows(orc, out, q, pos * C, wl, pos, orc_abs=orc_abs, orc_truth=orc_truth,
+                       label="config4 W=%d stream %d (chunk %d)" % (W, stream, pos))
         worst = (max(worst[0], e[0]), max(worst[1], e[1]))
         orc.close()
         orc_abs.close()
+        orc_truth.close()
         cache.close()
     print("parity config4 W=%d %s: worst scaled max %.3e mean %.3e"
           % (W, "one launch" if batched else "per stream", worst[0], worst[1]))

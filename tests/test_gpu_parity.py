@@ -11,7 +11,7 @@ import torch
 from paper_2509_22622_b200 import binding as B
 from paper_2509_22622_b200 import synth
 
-from gpu_util import bits, check_attn, dev, f64, new_cache, ulp_distance
+from gpu_util import bits, check_attn, check_attn_outliers, dev, f64, guarded, new_cache, ulp_distance
 
 pytestmark = pytest.mark.gpu
 
@@ -125,6 +125,7 @@ def stream_and_check(oracle_mod, wl, attn, n_chunks=None, rows_per_chunk=None, r
     cache = new_cache(wl)
     orc = oracle_for(oracle_mod, wl, faithful=faithful)
     orc_abs = oracle_for(oracle_mod, wl, faithful=faithful) if relative else None   # same K, |V|
+    orc_truth = oracle_for(oracle_mod, wl, faithful=False) if relative else None    # unrounded rotations
     C, P = wl.chunk_frames, wl.tokens_per_frame
     nq = C * P
     worst = (0.0, 0.0)
@@ -132,25 +133,34 @@ def stream_and_check(oracle_mod, wl, attn, n_chunks=None, rows_per_chunk=None, r
         for pass_id in range(passes):
             q, k, v = synth.chunk_qkv(wl, chunk, pass_id=pass_id)
             dq, dk, dv = dev(q), dev(k), dev(v)
-            q_out = torch.empty_like(dq)
-            out = torch.full_like(dq, float("nan"))
+            q_out, q_guard = guarded(dq.shape)
+            out, out_guard = guarded(dq.shape, fill=float("nan"))
             lse = torch.full((wl.heads, nq), float("nan"), device="cuda", dtype=torch.float32)
             cache.rope_append_kv(0, dq, dk, dv, chunk * C, wl.grid_h, wl.grid_w, wl.rope_theta, q_out)
             attn(cache.h, 0, q_out, chunk * C, C, out, lse)
             cache.check_device()
+            q_guard()
+            out_guard()
             orc.append(0, synth.bf16_bits_to_f64(k), synth.bf16_bits_to_f64(v), chunk * C, wl.grid_h, wl.grid_w,
                        wl.rope_theta)
             if orc_abs:
                 orc_abs.append(0, synth.bf16_bits_to_f64(k), np.abs(synth.bf16_bits_to_f64(v)), chunk * C,
                                wl.grid_h, wl.grid_w, wl.rope_theta)
+                orc_truth.append(0, synth.bf16_bits_to_f64(k), synth.bf16_bits_to_f64(v), chunk * C,
+                                 wl.grid_h, wl.grid_w, wl.rope_theta)
         qr = orc.rope_q(synth.bf16_bits_to_f64(q), chunk * C, wl.grid_h, wl.grid_w, wl.rope_theta)
         rows = None if rows_per_chunk is None else synth.sample_rows(nq, rows_per_chunk, seed=chunk)
         want, want_lse = orc.attn(0, qr, chunk * C, rows=rows)
         got = f64(out) if rows is None else f64(out)[rows]
         got_lse = lse.cpu().numpy().T.astype(np.float64)
         got_lse = got_lse if rows is None else got_lse[rows]
-        scale = orc_abs.attn(0, qr, chunk * C, rows=rows)[0] if orc_abs else None
-        e = check_attn(got, want, scale=scale)
+        if orc_abs:
+            scale = orc_abs.attn(0, qr, chunk * C, rows=rows)[0]
+            q_true = orc_truth.rope_q(synth.bf16_bits_to_f64(q), chunk * C, wl.grid_h, wl.grid_w, wl.rope_theta)
+            truth = orc_truth.attn(0, q_true, chunk * C, rows=rows)[0]
+            e = check_attn_outliers(got, want, scale, truth, label="%s chunk %d" % (wl.name, chunk))
+        else:
+            e = check_attn(got, want)
         worst = (max(worst[0], e[0]), max(worst[1], e[1]))
         assert np.abs(got_lse - want_lse).max() <= 2e-2, np.abs(got_lse - want_lse).max()
         st, ost = cache.state(), orc.state()
@@ -179,8 +189,10 @@ def test_sink_window_attn_outliers(oracle_mod):
     """1% of the entries x20.  The stated bar is for unit-variance inputs; here a
     single bf16 rounding of a rotated outlier (|x| ~ 60, half-ulp 0.12) moves a
     score by ~0.5, so the reference is the oracle in storage-faithful mode (rotated
-    Q/K rounded to bf16, which is what the cache format holds) and the error is
-    measured in units of max(1, sum_j p_j |v_j|)."""
+    Q/K rounded to bf16, which is what the cache format holds).  Three figures are
+    printed and bounded: the raw error against the unrounded oracle, the error
+    relative to max(1, |reference|), and the error in units of
+    max(1, sum_j p_j |v_j|) (gpu_util.check_attn_outliers)."""
     wl = dataclasses.replace(MEDIUM, name="medium_outliers", outlier_frac=0.01, seed=14)
     stream_and_check(oracle_mod, wl, B.ll_sink_window_attn, relative=True, faithful=True)
 
@@ -195,6 +207,7 @@ def test_sink_window_attn_with_growing_scores(oracle_mod):
     cache = new_cache(wl)
     orc = oracle_for(oracle_mod, wl, faithful=True)
     orc_abs = oracle_for(oracle_mod, wl, faithful=True)
+    orc_truth = oracle_for(oracle_mod, wl, faithful=False)
     C, P = wl.chunk_frames, wl.tokens_per_frame
     nq = C * P
     for chunk in range(wl.n_chunks):
@@ -211,10 +224,13 @@ def test_sink_window_attn_with_growing_scores(oracle_mod):
         kf, vf = synth.bf16_bits_to_f64(k), synth.bf16_bits_to_f64(v)
         orc.append(0, kf, vf, chunk * C, wl.grid_h, wl.grid_w, wl.rope_theta)
         orc_abs.append(0, kf, np.abs(vf), chunk * C, wl.grid_h, wl.grid_w, wl.rope_theta)
+        orc_truth.append(0, kf, vf, chunk * C, wl.grid_h, wl.grid_w, wl.rope_theta)
         qr = orc.rope_q(synth.bf16_bits_to_f64(q), chunk * C, wl.grid_h, wl.grid_w, wl.rope_theta)
         want, want_lse = orc.attn(0, qr, chunk * C)
         scale = orc_abs.attn(0, qr, chunk * C)[0]
-        check_attn(f64(out), want, scale=scale)
+        truth = orc_truth.attn(0, orc_truth.rope_q(synth.bf16_bits_to_f64(q), chunk * C, wl.grid_h, wl.grid_w,
+                                                   wl.rope_theta), chunk * C)[0]
+        check_attn_outliers(f64(out), want, scale, truth, label="%s chunk %d" % (wl.name, chunk))
         got_lse = lse.cpu().numpy().T.astype(np.float64)
         assert np.abs(got_lse - want_lse).max() <= 2e-2 * max(1.0, np.abs(want_lse).max() / 16)
     cache.close()

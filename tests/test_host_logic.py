@@ -21,7 +21,8 @@ def built():
 
 
 def test_library_exports_every_declared_symbol():
-    text = open(os.path.join(ROOT, "include", "llattn.h")).read()
+    text = "".join(open(os.path.join(ROOT, "include", name)).read()
+                   for name in sorted(os.listdir(os.path.join(ROOT, "include"))) if name.endswith(".h"))
     declared = set(re.findall(r"\b(ll_[a-z_0-9]+)\s*\(", text))
     assert declared == set(B.SIGNATURES), declared ^ set(B.SIGNATURES)
     L = ctypes.CDLL(B.LIB_PATH)

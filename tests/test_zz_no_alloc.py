@@ -6,7 +6,8 @@ allocating at call time is forbidden).  Its tables sit in a fixed array inside
 the library, shared by every call, so the interesting failure is a call that
 reads what an earlier call left behind.  The test therefore makes two calls in a
 row with different frame positions and grids and compares each with the
-rotated queries that ``ll_rope_append_kv`` produces for the same inputs.
+rotated queries that ``ll_rope_append_kv`` produces for the same inputs, and
+with the CPU oracle's rotation, under the bar every other RoPE test uses.
 
 This file sorts last on purpose: a run that stops at the first failure has
 already been through every other test when it gets here.
@@ -44,8 +45,11 @@ def regular_q_out(wl, upto_chunk):
     return bits(q_out)
 
 
-def test_static_rope_matches_regular_entry_point_twice_in_a_row():
+def test_static_rope_matches_regular_entry_point_twice_in_a_row(oracle_mod):
     want = [regular_q_out(wl, chunk) for wl, chunk in CASES]
+    want_oracle = [synth.f32_to_bf16_bits(
+        oracle_mod.rope(synth.bf16_bits_to_f64(synth.chunk_qkv(wl, chunk)[0]), chunk * wl.chunk_frames,
+                        wl.grid_h, wl.grid_w, wl.rope_theta).astype(np.float32)) for wl, chunk in CASES]
     launches0 = B.ll_launch_count()
     got = []
     for wl, chunk in CASES:                      # back to back: the second call finds the first one's tables
@@ -57,9 +61,11 @@ def test_static_rope_matches_regular_entry_point_twice_in_a_row():
         got.append(out)
     torch.cuda.synchronize()
     assert B.ll_launch_count() - launches0 == 2 * len(CASES)     # table kernel + rotation kernel per call
-    for g, w in zip(got, want):
+    for g, w, wo in zip(got, want, want_oracle):
         d = ulp_distance(bits(g), w)
         # the same fp32 arithmetic on the same fp64-built tables: the parity tests allow one bf16 ulp
+        assert d.max() <= 1 and (d == 0).mean() >= 0.99
+        d = ulp_distance(bits(g), wo)                # and the fp64 definition, rounded once
         assert d.max() <= 1 and (d == 0).mean() >= 0.99
     # and once more in the opposite order, in place
     for (wl, chunk), w in reversed(list(zip(CASES, want))):

@@ -61,8 +61,11 @@ constexpr int kThreads = 640;
 constexpr int kSoftmaxWarps = 16;
 constexpr int kTmaWarp = 16;
 constexpr int kMmaWarp = 17;
-// a piece's 16 weights per thread and row were safe to compute if they sum to at most this
-constexpr float kSafeSum = 256.f;
+// A piece's 16 weights per thread and row were safe to compute if they sum to less than this:
+// no weight can exceed the sum, and a score too far above the row's reference shows up as a
+// weight of at least 2^127 on the special-function unit and of just under 256 (the top of its
+// clamped range) on the polynomial path.
+constexpr float kSafeSum = 128.f;
 // Register reallocation draws on what the CTA was launched with: 640 threads x 96
 // registers = (16 softmax warps x 104 + 4 producer-group warps x 64) x 32.  A
 // request beyond that total would block forever.
@@ -190,31 +193,36 @@ __device__ __forceinline__ uint64_t exp2_sfu2(uint64_t x2)
     return pack2(ex2(x0), ex2(x1));
 }
 
-// 2^x for two values on the FMA pipe: x = n + f with n = floor(x) taken from the
-// low mantissa bits of x + 1.5 * 2^23 (rounded down), 2^f by a cubic with maximum
-// relative error 7.5e-5 on [0, 1), and n added to the result's exponent field.
-// Inputs are clamped to [-126, 127]: below, a weight of 2^-126 instead of less; above, a
-// huge finite weight that the caller's safety check on the sums catches (NaN stays NaN).
-__device__ __forceinline__ uint64_t exp2_poly2(uint64_t x2)
+// 2^x for two scores on the FMA pipe, x = s * c - m (c = log2(e)/sqrt(D), m the row's reference).
+// The scale-and-shift itself does the clamping: y = sat(s * c/128 + (kPolyLow - m)/128) is
+// (x + kPolyLow)/128 held to [0, 1], i.e. x held to [-kPolyLow, 128 - kPolyLow].  Then
+// 128 y = j + f with j = floor(128 y) read from the low mantissa bits of 128 y + 1.5 * 2^23
+// (rounded down), 2^f by a cubic with maximum relative error 7.5e-5 on [0, 1) whose
+// coefficients carry the factor 2^-kPolyLow, and j added to the result's exponent field.
+// A score below the range gives a weight of 2^-kPolyLow instead of less (irrelevant against a
+// row sum >= 1); one above it gives just under 2^(128 - kPolyLow) = 256, which the caller's
+// check on the sums (kSafeSum) catches.  NaN scores clamp to the bottom of the range.
+constexpr int kPolyLow = 120;
+struct PolyRow {
+    float cs, bias;                 // c / 128 and (kPolyLow - m) / 128
+};
+__device__ __forceinline__ uint64_t exp2_poly2(float s0, float s1, const PolyRow &r)
 {
     constexpr float kMagic = 12582912.f;
-    float x0, x1;
-    unpack2(x2, x0, x1);
-    x0 = fminf(fmaxf(x0, -126.f), 127.f);
-    x1 = fminf(fmaxf(x1, -126.f), 127.f);
-    x2 = pack2(x0, x1);
-    const uint64_t r2 = add2_rm(x2, pack2(kMagic, kMagic));
-    const uint64_t n2 = add2(r2, pack2(-kMagic, -kMagic));                  // floor(x), exact
-    const uint64_t f2 = fma2(n2, pack2(-1.f, -1.f), x2);                    // x - floor(x), exact
-    uint64_t y2 = fma2(f2, pack2(0.07802491635f, 0.07802491635f), pack2(0.22606660426f, 0.22606660426f));
-    y2 = fma2(y2, f2, pack2(0.69583368301f, 0.69583368301f));
-    y2 = fma2(y2, f2, pack2(0.99992519617f, 0.99992519617f));
-    float y0, y1, r0, r1;
-    unpack2(y2, y0, y1);
+    constexpr float kUnit = 0x1p-120f;
+    static_assert(kPolyLow == 120, "the cubic's coefficients carry 2^-kPolyLow");
+    const uint64_t y2 = pack2(fma_sat(s0, r.cs, r.bias), fma_sat(s1, r.cs, r.bias));
+    const uint64_t r2 = fma2_rm(y2, pack2(128.f, 128.f), pack2(kMagic, kMagic));
+    const uint64_t nj2 = fma2(r2, pack2(-1.f, -1.f), pack2(kMagic, kMagic));          // -floor(128 y), exact
+    const uint64_t f2 = fma2(y2, pack2(128.f, 128.f), nj2);                           // 128 y - j, exact
+    uint64_t p2 = fma2(f2, pack2(0.07802491635f * kUnit, 0.07802491635f * kUnit),
+                       pack2(0.22606660426f * kUnit, 0.22606660426f * kUnit));
+    p2 = fma2(p2, f2, pack2(0.69583368301f * kUnit, 0.69583368301f * kUnit));
+    p2 = fma2(p2, f2, pack2(0.99992519617f * kUnit, 0.99992519617f * kUnit));
+    float p0, p1, r0, r1;
+    unpack2(p2, p0, p1);
     unpack2(r2, r0, r1);
-    y0 = as_f(as_u(y0) + (as_u(r0) << 23));
-    y1 = as_f(as_u(y1) + (as_u(r1) << 23));
-    return pack2(y0, y1);
+    return pack2(as_f(mad_lo(as_u(r0), 1u << 23, as_u(p0))), as_f(mad_lo(as_u(r1), 1u << 23, as_u(p1))));
 }
 
 // -inf into the registers of one 64-column piece (first column col0) whose key is not valid.
@@ -490,17 +498,17 @@ attn_sm100_kernel(const __grid_constant__ AttnParams p, const __grid_constant__ 
                         uint64_t ts_a = 0ull, ts_b = 0ull;         // the piece's sums, two partials per row
                         {
                             const uint64_t na2 = pack2(-m_a, -m_a), nb2 = pack2(-m_b, -m_b);
+                            const PolyRow ra{c * (1.f / 128.f), ((float)kPolyLow - m_a) * (1.f / 128.f)};
+                            const PolyRow rb{c * (1.f / 128.f), ((float)kPolyLow - m_b) * (1.f / 128.f)};
 #pragma unroll
                             for (int k = 0; k < 8; ++k) {
-                                const uint64_t xa = fma2(pack2(as_f(v[4 * k]), as_f(v[4 * k + 1])), c2, na2);
-                                const uint64_t xb = fma2(pack2(as_f(v[4 * k + 2]), as_f(v[4 * k + 3])), c2, nb2);
                                 uint64_t pa, pb;
                                 if ((kPolyMask >> (8 * piece + k)) & 1u) {
-                                    pa = exp2_poly2(xa);
-                                    pb = exp2_poly2(xb);
+                                    pa = exp2_poly2(as_f(v[4 * k]), as_f(v[4 * k + 1]), ra);
+                                    pb = exp2_poly2(as_f(v[4 * k + 2]), as_f(v[4 * k + 3]), rb);
                                 } else {
-                                    pa = exp2_sfu2(xa);
-                                    pb = exp2_sfu2(xb);
+                                    pa = exp2_sfu2(fma2(pack2(as_f(v[4 * k]), as_f(v[4 * k + 1])), c2, na2));
+                                    pb = exp2_sfu2(fma2(pack2(as_f(v[4 * k + 2]), as_f(v[4 * k + 3])), c2, nb2));
                                 }
                                 ts_a = add2(ts_a, pa);
                                 ts_b = add2(ts_b, pb);
@@ -519,7 +527,7 @@ attn_sm100_kernel(const __grid_constant__ AttnParams p, const __grid_constant__ 
                             unpack2(ts_b, x0, x1);
                             sb = x0 + x1;
                         }
-                        if (__any_sync(0xffffffffu, !(sa <= kSafeSum) || !(sb <= kSafeSum))) {
+                        if (__any_sync(0xffffffffu, !(sa < kSafeSum) || !(sb < kSafeSum))) {
                             // exact maxima of the piece's rows: 16 columns per thread, then across the quad
                             float ta = fmaxf(as_f(v[0]), as_f(v[1])), tb = fmaxf(as_f(v[2]), as_f(v[3]));
 #pragma unroll

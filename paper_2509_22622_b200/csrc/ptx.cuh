@@ -245,6 +245,30 @@ __device__ __forceinline__ uint64_t add2_rm(uint64_t a, uint64_t b)
     return d;
 }
 
+// a * b + c with both halves rounded toward minus infinity
+__device__ __forceinline__ uint64_t fma2_rm(uint64_t a, uint64_t b, uint64_t c)
+{
+    uint64_t d;
+    asm("fma.rm.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+    return d;
+}
+
+// a * b + c clamped to [0, 1] (NaN gives 0)
+__device__ __forceinline__ float fma_sat(float a, float b, float c)
+{
+    float d;
+    asm("fma.rn.sat.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+    return d;
+}
+
+// a * b + c on 32-bit integers (low half of the product)
+__device__ __forceinline__ uint32_t mad_lo(uint32_t a, uint32_t b, uint32_t c)
+{
+    uint32_t d;
+    asm("mad.lo.u32 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(b), "r"(c));
+    return d;
+}
+
 // Two fp32 -> packed bf16x2, round to nearest even; `lo` lands in the low half.
 __device__ __forceinline__ uint32_t cvt_bf16x2(float lo, float hi)
 {

@@ -25,10 +25,11 @@
 //   warps 0-15          softmax: warp (w, q, h) owns the 16 rows 32q + 16h .. of
 //                       lane w; its threads read S with the 16x256b TMEM shape, so
 //                       a row lives in the four threads of a quad.  P (bf16) goes to
-//                       a swizzled shared-memory tile, 64 keys at a time.  The rows'
-//                       reference maxima move, and O is rescaled in TMEM, only when
-//                       a weight computed against the old reference would have been
-//                       large.
+//                       a swizzled shared-memory tile, 64 keys at a time and as soon as
+//                       a 64-key piece is computed (its registers are then free for
+//                       the next piece).  The rows' reference maxima move, and O is
+//                       rescaled in TMEM, only when a weight computed against the old
+//                       reference would have been large.
 //   P does not go back over S: a lane's S buffer is free as soon as its softmax
 //   warps hold the tile in registers, so the MMA warp issues QK of step j+1 while
 //   the softmax of step j is still running, and the softmax warps find the next S
@@ -481,10 +482,10 @@ attn_sm100_kernel(const __grid_constant__ AttnParams p, const __grid_constant__ 
                     // the warp is large or not finite - always on a column's first piece, where the
                     // references are -inf - are the exact row maxima taken, the references moved,
                     // what has been accumulated rescaled, and the piece redone.
-                    uint32_t pk[32];                               // P of both pieces, handed over together
 #pragma unroll
                     for (int piece = 0; piece < 2; ++piece) {
                         uint32_t v[32];
+                        uint32_t pp[16];                           // the piece's P: 16 rows x 64 keys per warp
                         tmem_ld_16x256b_x8(t_s + 64 * piece, v);
                         tmem_wait_ld();
                         if (piece == 1) {
@@ -494,29 +495,46 @@ attn_sm100_kernel(const __grid_constant__ AttnParams p, const __grid_constant__ 
                             if (lane == 0) mbar_arrive(bar(kSEmpty + w));
                         }
                         if (nvalid < kKeyTile) mask_piece(v, 64 * piece, cq, nvalid);
-                        uint32_t *pp = pk + 16 * piece;
                         uint64_t ts_a = 0ull, ts_b = 0ull;         // the piece's sums, two partials per row
                         {
                             const uint64_t na2 = pack2(-m_a, -m_a), nb2 = pack2(-m_b, -m_b);
                             const PolyRow ra{c * (1.f / 128.f), ((float)kPolyLow - m_a) * (1.f / 128.f)};
                             const PolyRow rb{c * (1.f / 128.f), ((float)kPolyLow - m_b) * (1.f / 128.f)};
+                            // Four 8-key groups at a time, stage by stage, so that the exponentials of a
+                            // batch are all in flight before the first result is needed.
 #pragma unroll
-                            for (int k = 0; k < 8; ++k) {
-                                uint64_t pa, pb;
-                                if ((kPolyMask >> (8 * piece + k)) & 1u) {
-                                    pa = exp2_poly2(as_f(v[4 * k]), as_f(v[4 * k + 1]), ra);
-                                    pb = exp2_poly2(as_f(v[4 * k + 2]), as_f(v[4 * k + 3]), rb);
-                                } else {
-                                    pa = exp2_sfu2(fma2(pack2(as_f(v[4 * k]), as_f(v[4 * k + 1])), c2, na2));
-                                    pb = exp2_sfu2(fma2(pack2(as_f(v[4 * k + 2]), as_f(v[4 * k + 3])), c2, nb2));
+                            for (int g = 0; g < 2; ++g) {
+                                uint64_t xa[4], xb[4];
+#pragma unroll
+                                for (int kk = 0; kk < 4; ++kk) {
+                                    const int k = 4 * g + kk;
+                                    if (!((kPolyMask >> (8 * piece + k)) & 1u)) {
+                                        xa[kk] = fma2(pack2(as_f(v[4 * k]), as_f(v[4 * k + 1])), c2, na2);
+                                        xb[kk] = fma2(pack2(as_f(v[4 * k + 2]), as_f(v[4 * k + 3])), c2, nb2);
+                                    }
                                 }
-                                ts_a = add2(ts_a, pa);
-                                ts_b = add2(ts_b, pb);
-                                float a0, a1, b0, b1;
-                                unpack2(pa, a0, a1);
-                                unpack2(pb, b0, b1);
-                                pp[2 * k] = cvt_bf16x2(a0, a1);        // key 8k + cq in the low half
-                                pp[2 * k + 1] = cvt_bf16x2(b0, b1);
+#pragma unroll
+                                for (int kk = 0; kk < 4; ++kk) {
+                                    const int k = 4 * g + kk;
+                                    if ((kPolyMask >> (8 * piece + k)) & 1u) {
+                                        xa[kk] = exp2_poly2(as_f(v[4 * k]), as_f(v[4 * k + 1]), ra);
+                                        xb[kk] = exp2_poly2(as_f(v[4 * k + 2]), as_f(v[4 * k + 3]), rb);
+                                    } else {
+                                        xa[kk] = exp2_sfu2(xa[kk]);
+                                        xb[kk] = exp2_sfu2(xb[kk]);
+                                    }
+                                }
+#pragma unroll
+                                for (int kk = 0; kk < 4; ++kk) {
+                                    const int k = 4 * g + kk;
+                                    ts_a = add2(ts_a, xa[kk]);
+                                    ts_b = add2(ts_b, xb[kk]);
+                                    float a0, a1, b0, b1;
+                                    unpack2(xa[kk], a0, a1);
+                                    unpack2(xb[kk], b0, b1);
+                                    pp[2 * k] = cvt_bf16x2(a0, a1);        // key 8k + cq in the low half
+                                    pp[2 * k + 1] = cvt_bf16x2(b0, b1);
+                                }
                             }
                         }
                         float sa, sb;
@@ -547,11 +565,22 @@ attn_sm100_kernel(const __grid_constant__ AttnParams p, const __grid_constant__ 
                             acc_a = fma2(acc_a, pack2(al_a, al_a), 0ull);
                             acc_b = fma2(acc_b, pack2(al_b, al_b), 0ull);
                             if (piece == 1) {
-                                // the first piece's P, still in registers
+                                // the first piece's P already sits in shared memory, against the old
+                                // references: take it back, rescale, store again (nobody else reads it
+                                // before this step's hand-over)
+                                __syncwarp();
 #pragma unroll
-                                for (int k = 0; k < 8; ++k) {
-                                    pk[2 * k] = cvt_bf16x2(as_f(pk[2 * k] << 16) * al_a, as_f(pk[2 * k] & 0xffff0000u) * al_a);
-                                    pk[2 * k + 1] = cvt_bf16x2(as_f(pk[2 * k + 1] << 16) * al_b, as_f(pk[2 * k + 1] & 0xffff0000u) * al_b);
+                                for (int half = 0; half < 2; ++half) {
+                                    const uint32_t at = half ? (p_at ^ 64u) : p_at;
+                                    uint32_t ra0, ra1, ra2, ra3, rb0, rb1, rb2, rb3;
+                                    ldmatrix_x4(at, ra0, ra1, ra2, ra3);
+                                    ldmatrix_x4(at + 8 * 128, rb0, rb1, rb2, rb3);
+                                    auto scale = [](uint32_t x, float al) {
+                                        return cvt_bf16x2(as_f(x << 16) * al, as_f(x & 0xffff0000u) * al);
+                                    };
+                                    __syncwarp();
+                                    stmatrix_x4(at, scale(ra0, al_a), scale(ra1, al_a), scale(ra2, al_a), scale(ra3, al_a));
+                                    stmatrix_x4(at + 8 * 128, scale(rb0, al_b), scale(rb1, al_b), scale(rb2, al_b), scale(rb3, al_b));
                                 }
                             }
                             if (j != s.kt0) {
@@ -595,20 +624,19 @@ attn_sm100_kernel(const __grid_constant__ AttnParams p, const __grid_constant__ 
                         }
                         acc_a = add2(acc_a, ts_a);
                         acc_b = add2(acc_b, ts_b);
-                    }
-                    // P (bf16) into the lane's shared-memory tile, once the PV that read the previous
-                    // step's P from it has completed.  The tile is the K-major, 128-byte-swizzled A
-                    // operand of PV: one 64-key atom per piece, row r at r * 128 bytes, its 16-byte
-                    // chunk k (8 keys) at chunk position k ^ (r % 8).
-                    if (sc > 0 && !__all_sync(0xffffffffu, wait(kPEmpty + w, sc - 1, (int)sc))) return;
-#pragma unroll
-                    for (int piece = 0; piece < 2; ++piece) {
-                        const uint32_t *pp = pk + 16 * piece;
-                        const uint32_t at = p_at + piece * C::kAtomBytes;
-                        stmatrix_x4(at, pp[0], pp[2], pp[4], pp[6]);                       // rows a, chunks 0..3
-                        stmatrix_x4(at ^ 64u, pp[8], pp[10], pp[12], pp[14]);               // rows a, chunks 4..7
-                        stmatrix_x4(at + 8 * 128, pp[1], pp[3], pp[5], pp[7]);              // rows a + 8
-                        stmatrix_x4((at ^ 64u) + 8 * 128, pp[9], pp[11], pp[13], pp[15]);
+                        // The piece's P (bf16) goes into the lane's shared-memory tile straight away (the
+                        // first piece's once the PV that read the previous step's P has completed), so
+                        // its registers are free while the second piece is computed.  The tile is the
+                        // K-major, 128-byte-swizzled A operand of PV: one 64-key atom per piece, row r at
+                        // r * 128 bytes, its 16-byte chunk k (8 keys) at chunk position k ^ (r % 8).
+                        if (piece == 0 && sc > 0 && !__all_sync(0xffffffffu, wait(kPEmpty + w, sc - 1, (int)sc))) return;
+                        {
+                            const uint32_t at = p_at + piece * C::kAtomBytes;
+                            stmatrix_x4(at, pp[0], pp[2], pp[4], pp[6]);                       // rows a, chunks 0..3
+                            stmatrix_x4(at ^ 64u, pp[8], pp[10], pp[12], pp[14]);               // rows a, chunks 4..7
+                            stmatrix_x4(at + 8 * 128, pp[1], pp[3], pp[5], pp[7]);              // rows a + 8
+                            stmatrix_x4((at ^ 64u) + 8 * 128, pp[9], pp[11], pp[13], pp[15]);
+                        }
                     }
                     fence_proxy_async_smem();                      // the stores above are read by the tensor pipe
                     __syncwarp();

@@ -47,6 +47,13 @@ __device__ __forceinline__ void stmatrix_x4(uint32_t row_addr, uint32_t r0, uint
                  ::"r"(row_addr), "r"(r0), "r"(r1), "r"(r2), "r"(r3) : "memory");
 }
 
+// The inverse of stmatrix_x4: four 8x8 matrices of 16-bit elements back into the same registers.
+__device__ __forceinline__ void ldmatrix_x4(uint32_t row_addr, uint32_t &r0, uint32_t &r1, uint32_t &r2, uint32_t &r3)
+{
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0, %1, %2, %3}, [%4];"
+                 : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3) : "r"(row_addr) : "memory");
+}
+
 __device__ __forceinline__ void mbar_arrive(uint32_t bar)
 {
     asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");

@@ -65,6 +65,9 @@ def lib():
             L.llo_rope_split.restype = None
             L.llo_round_bf16.restype = C.c_double
             L.llo_round_bf16.argtypes = [C.c_double]
+            L.llo_round_e4m3.restype = C.c_double
+            L.llo_round_e4m3.argtypes = [C.c_double]
+            L.llo_set_kv_e4m3.argtypes = [C.c_void_p, C.POINTER(C.c_float), C.POINTER(C.c_float)]
             L.llo_rope.argtypes = [C.POINTER(C.c_double), C.POINTER(C.c_double), C.c_int64,
                                    C.c_int, C.c_int, C.c_int64, C.c_int, C.c_int, C.c_double, C.c_int]
             L.llo_append.argtypes = [C.c_void_p, C.c_int, C.POINTER(C.c_double), C.POINTER(C.c_double),
@@ -114,6 +117,12 @@ def rope_split(D: int):
 def round_bf16(x):
     """Nearest-bf16 (ties to even) of float64 values, returned as float64."""
     f = np.vectorize(lambda t: lib().llo_round_bf16(float(t)), otypes=[np.float64])
+    return f(np.asarray(x, dtype=np.float64))
+
+
+def round_e4m3(x):
+    """Nearest E4M3 value (ties to even, saturating at 448) of float64 values, as float64."""
+    f = np.vectorize(lambda t: lib().llo_round_e4m3(float(t)), otypes=[np.float64])
     return f(np.asarray(x, dtype=np.float64))
 
 
@@ -198,6 +207,17 @@ class Oracle:
 
     def visible(self, fq: int, fk: int, lo_floor: int = 0) -> bool:
         return bool(lib().llo_visible(self._h, fq, fk, lo_floor))
+
+    def set_kv_e4m3(self, k_scale, v_scale):
+        """8-bit storage from now on: rows hold scale * E4M3(x / scale), scales [L, H] fp32."""
+        ks = np.ascontiguousarray(k_scale, dtype=np.float32).reshape(-1)
+        vs = np.ascontiguousarray(v_scale, dtype=np.float32).reshape(-1)
+        if ks.shape[0] != self.L * self.H or vs.shape[0] != self.L * self.H:
+            raise OracleError(ERR_ARG, "set_kv_e4m3 shape")
+        fp = C.POINTER(C.c_float)
+        st = lib().llo_set_kv_e4m3(self._h, ks.ctypes.data_as(fp), vs.ctypes.data_as(fp))
+        if st != OK:
+            raise OracleError(st, "set_kv_e4m3")
 
     def reset(self):
         st = lib().llo_reset(self._h)

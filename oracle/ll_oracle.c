@@ -40,6 +40,10 @@
  *     norm over the token's whole row of H*D elements with a learned gain
  *     (llo_rms_norm), applied before the rotation.
  *
+ *   - 8-bit cache storage (the paper's appendix "Quantization" only motivates a
+ *     low-precision variant; the format is this library's): rotated K and V are
+ *     kept as E4M3 codes times one scale per (layer, head), see llo_set_kv_e4m3.
+ *
  * Storage here is [layer][slot][token][head][dim] in double.  The slot rule
  * (frame f -> slot f if f < S, else S + (f - S) mod W) is the bit-exact
  * contract for the cache state.
@@ -64,6 +68,8 @@ typedef struct llo {
     int32_t *slot_frame;   /* [L][S+W] absolute frame in each slot, -1 = empty */
     int64_t *evictions;    /* [L] frames overwritten by a newer frame */
     double *K, *V;         /* [L][S+W][P][H][D] */
+    int kv_e4m3;           /* 1: rows are stored as scale * E4M3(x / scale) */
+    float *k_scale, *v_scale;   /* [L][H], fp32 as the storage format defines them */
 } llo;
 
 /* ---- helpers that are not part of the method ---------------------------- */
@@ -81,6 +87,68 @@ double llo_round_bf16(double x)
     double m = frexp(x, &e);              /* x = m * 2^e, 0.5 <= |m| < 1 */
     double q = nearbyint(m * 256.0);      /* default rounding mode: ties to even */
     return ldexp(q, e - 8);
+}
+
+/* ---- 8-bit storage format -------------------------------------------------- */
+
+/* Nearest value of the 8-bit float format E4M3: 1 sign bit, 4 exponent bits with
+ * bias 7, 3 mantissa bits; no infinities; the largest finite magnitude is 448
+ * (exponent field 15, mantissa 110); below 2^-6 the values are subnormal with
+ * spacing 2^-9.  Ties go to the even mantissa; magnitudes beyond 448 clamp to
+ * 448 (saturating conversion); NaN stays NaN. */
+double llo_round_e4m3(double x)
+{
+    if (isnan(x) || x == 0.0) return x;
+    double a = fabs(x), sgn = x < 0 ? -1.0 : 1.0;
+    if (a >= 448.0) return sgn * 448.0;
+    int e;
+    frexp(a, &e);                         /* a = m * 2^e, 0.5 <= m < 1: binade [2^(e-1), 2^e) */
+    int lsb = e - 1 - 3;                  /* exponent of the last of 3 mantissa bits in that binade */
+    if (lsb < -9) lsb = -9;               /* subnormal range: fixed spacing 2^-9 */
+    double q = nearbyint(ldexp(a, -lsb)); /* ties to even */
+    double r = ldexp(q, lsb);
+    if (r > 448.0) r = 448.0;
+    return sgn * r;
+}
+
+/* The stored value of x under scale s: the division is done in fp32 (the format's
+ * definition: code = E4M3(fl32(fl32(x) / s))), the product back is exact in double. */
+static double store_e4m3(double x, float s)
+{
+    float t = (float)x / s;
+    return llo_round_e4m3((double)t) * (double)s;
+}
+
+/* Switch the cache to 8-bit storage: from now on every row written by append,
+ * recache or clip holds, per head h of layer l, k_scale[l*H+h] * E4M3(K / k_scale)
+ * for the rotated keys and v_scale[l*H+h] * E4M3(V / v_scale) for the values.
+ * Scales are positive fp32 numbers.  Rows already stored are not touched. */
+int llo_set_kv_e4m3(llo *o, const float *k_scale, const float *v_scale)
+{
+    if (!o || !k_scale || !v_scale) return LLO_ERR_ARG;
+    size_t n = (size_t)o->L * o->H;
+    for (size_t i = 0; i < n; ++i)
+        if (!(k_scale[i] > 0.f) || !(v_scale[i] > 0.f)) return LLO_ERR_ARG;
+    if (!o->k_scale) o->k_scale = (float *)malloc(n * sizeof(float));
+    if (!o->v_scale) o->v_scale = (float *)malloc(n * sizeof(float));
+    if (!o->k_scale || !o->v_scale) return LLO_ERR_ARG;
+    memcpy(o->k_scale, k_scale, n * sizeof(float));
+    memcpy(o->v_scale, v_scale, n * sizeof(float));
+    o->kv_e4m3 = 1;
+    return LLO_OK;
+}
+
+/* One token's K (already rotated, in place at K) and V rows under the storage format. */
+static void store_format(const llo *o, int layer, double *K, double *V)
+{
+    if (!o->kv_e4m3) return;
+    for (int h = 0; h < o->H; ++h) {
+        float ks = o->k_scale[(size_t)layer * o->H + h], vs = o->v_scale[(size_t)layer * o->H + h];
+        for (int d = 0; d < o->D; ++d) {
+            K[(size_t)h * o->D + d] = store_e4m3(K[(size_t)h * o->D + d], ks);
+            V[(size_t)h * o->D + d] = store_e4m3(V[(size_t)h * o->D + d], vs);
+        }
+    }
 }
 
 /* ---- lifetime ------------------------------------------------------------ */
@@ -107,6 +175,7 @@ void llo_destroy(llo *o)
 {
     if (!o) return;
     free(o->end); free(o->evictions); free(o->slot_frame); free(o->K); free(o->V);
+    free(o->k_scale); free(o->v_scale);
     free(o);
 }
 
@@ -234,6 +303,7 @@ int llo_append(llo *o, int layer, const double *k, const double *v,
                 rope_row(k + src + (size_t)h * o->D, K + dst + (size_t)h * o->D,
                          o->D, theta, f, y, x, o->faithful);
             memcpy(V + dst, v + src, re * sizeof(double));
+            store_format(o, layer, K + dst, V + dst);
         }
     }
     if (is_new) o->end[layer] = end + o->C;
@@ -416,6 +486,7 @@ int llo_recache(llo *o, int layer, const double *q, const double *k, const doubl
                 rope_row(k + src + (size_t)h * o->D, K + dst + (size_t)h * o->D,
                          o->D, theta, f, y, x, o->faithful);
             memcpy(V + dst, v + src, re * sizeof(double));
+            store_format(o, layer, K + dst, V + dst);
         }
     }
     int64_t nq = (int64_t)n_frames * o->P;

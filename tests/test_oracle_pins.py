@@ -632,3 +632,122 @@ def test_rms_norm_invariants(oracle_mod):
     # eps matters for small rows: with eps the output shrinks
     small = 1e-3 * x
     assert np.abs(oracle_mod.rms_norm(small, g, 1e-6)).max() < np.abs(oracle_mod.rms_norm(small, g, 0.0)).max()
+
+
+# ---------------------------------------------------------------------------
+# 8-bit (E4M3) cache storage
+# ---------------------------------------------------------------------------
+
+def e4m3_table():
+    """Every finite E4M3 value decoded from its bit pattern: sign(1) exponent(4, bias 7)
+    mantissa(3); exponent field 0 is subnormal; S.1111.111 is NaN (no infinities)."""
+    vals = {}
+    for code in range(256):
+        sgn, e, m = code >> 7, (code >> 3) & 15, code & 7
+        if e == 15 and m == 7:
+            continue
+        mag = (m / 8.0) * 2.0 ** -6 if e == 0 else (1.0 + m / 8.0) * 2.0 ** (e - 7)
+        vals[code] = -mag if sgn else mag
+    return vals
+
+
+def brute_force_e4m3(x):
+    """Nearest table value, ties to the code with an even mantissa, clamped to +-448."""
+    table = e4m3_table()
+    pos = sorted((v, c) for c, v in table.items() if c < 128)
+    a = min(abs(float(x)), 448.0)
+    best = min(pos, key=lambda vc: (abs(vc[0] - a), vc[1] & 1))
+    return best[0] if x >= 0 else -best[0]
+
+
+def test_e4m3_rounding_equals_brute_force_over_the_code_table(oracle_mod):
+    table = e4m3_table()
+    assert len(table) == 254 and max(table.values()) == 448.0 and table[1] == 2.0 ** -9
+    # every representable value is a fixed point
+    for v in table.values():
+        assert oracle_mod.round_e4m3(v) == v
+    # every midpoint between neighbours (the ties), points just off them, random values, the ends
+    pos = sorted(v for c, v in table.items() if c < 128)
+    xs = []
+    for lo, hi in zip(pos[:-1], pos[1:]):
+        mid = 0.5 * (lo + hi)
+        xs += [mid, np.nextafter(mid, 0.0), np.nextafter(mid, 1e9), 0.75 * lo + 0.25 * hi]
+    rng = np.random.default_rng(0)
+    xs += list(rng.standard_normal(2000) * np.exp(rng.uniform(-8, 7, 2000)))
+    xs += [448.0, 449.0, 464.0, 1e6, 2.0 ** -10, 2.0 ** -11, 1e-30]
+    for x in xs:
+        for s in (x, -x):
+            assert oracle_mod.round_e4m3(s) == brute_force_e4m3(s), s
+    assert np.isnan(oracle_mod.round_e4m3(float("nan")))
+
+
+def test_e4m3_cache_rows_and_attention_equal_a_flat_reference(oracle_mod):
+    """The rows an 8-bit cache holds are scale * E4M3(fl32(x) / scale) of the rotated keys and
+    the raw values (brute force over the code table), old rows stay as they were, and attention
+    over such a cache is library softmax over exactly those numbers."""
+    L, H, D, gh, gw, C, S, W = 2, 3, 64, 2, 3, 1, 1, 3
+    P = gh * gw
+    orc = oracle_mod.Oracle(L, H, D, P, C, S, W)
+    ks = np.array([[0.02, 0.5, 1.0], [0.013, 0.25, 3.0]], dtype=np.float32)
+    vs = np.array([[0.01, 0.125, 2.0], [0.7, 0.031, 1.5]], dtype=np.float32)
+    k0, v0 = rand((P, H, D), 1), rand((P, H, D), 2)
+    orc.append(1, k0, v0, 0, gh, gw)                       # written before the switch: stays exact
+    orc.set_kv_e4m3(ks, vs)
+    quant = np.vectorize(brute_force_e4m3)
+
+    def stored(x, scale):                                  # x [P, H, D], scale [H]
+        t = (x.astype(np.float32) / scale[None, :, None].astype(np.float32)).astype(np.float64)
+        return quant(t) * scale[None, :, None].astype(np.float64)
+
+    hist_k, hist_v = [oracle_mod.rope(k0, 0, gh, gw)], [v0]
+    for f in range(1, 6):
+        k, v = rand((P, H, D), 10 + f) * (1 + f), rand((P, H, D), 20 + f)
+        orc.append(1, k, v, f, gh, gw)
+        hist_k.append(stored(oracle_mod.rope(k, f, gh, gw), ks[1]))
+        hist_v.append(stored(v, vs[1]))
+    K, V = orc.read_layer(1)
+    for f in (0, 3, 4, 5):                                 # resident: sink 0 and window 3..5
+        slot = orc.slot_of(f)
+        assert np.array_equal(K[slot], hist_k[f]) and np.array_equal(V[slot], hist_v[f]), f
+    assert not np.array_equal(K[orc.slot_of(5)], oracle_mod.rope(k, 5, gh, gw))      # it did quantise
+    q = oracle_mod.rope(rand((P, H, D), 99), 5, gh, gw)
+    got, lse = orc.attn(1, q, 5)
+    keys = np.concatenate([hist_k[f] for f in (0, 3, 4, 5)])
+    vals = np.concatenate([hist_v[f] for f in (0, 3, 4, 5)])
+    s = np.einsum("qhd,khd->hqk", q, keys) / np.sqrt(D)
+    want = np.einsum("hqk,khd->qhd", softmax(s, axis=-1), vals)
+    assert np.abs(got - want).max() < 1e-12
+    assert np.abs(lse - logsumexp(s, axis=-1).T).max() < 1e-12
+    # a recache writes quantised rows too and leaves the sink alone
+    rq, rk, rv = rand((3 * P, H, D), 31), rand((3 * P, H, D), 32), rand((3 * P, H, D), 33)
+    orc.recache(1, rq, rk, rv, 3, gh, gw)
+    K2, V2 = orc.read_layer(1)
+    assert np.array_equal(K2[0], hist_k[0]) and np.array_equal(V2[0], hist_v[0])
+    for i, f in enumerate((3, 4, 5)):
+        slot = orc.slot_of(f)
+        assert np.array_equal(V2[slot], stored(rv[i * P:(i + 1) * P], vs[1]))
+        assert np.array_equal(K2[slot], stored(oracle_mod.rope(rk[i * P:(i + 1) * P], f, gh, gw), ks[1]))
+    # layer 0 uses its own scales
+    orc.append(0, k0, v0, 0, gh, gw)
+    K0, V0 = orc.read_layer(0)
+    assert np.array_equal(V0[0], stored(v0, vs[0]))
+
+
+def test_e4m3_storage_scales_by_powers_of_two_and_saturates(oracle_mod):
+    """Doubling the scale and the data doubles the stored value exactly; values beyond
+    448 scales clamp; the relative error inside the normal range is at most 2^-4."""
+    H, D = 1, 8
+    x = rand((1, H, D), 5) * 3.0
+    outs = []
+    for mult in (1.0, 2.0, 0.25):
+        orc = oracle_mod.Oracle(1, H, D, 1, 1, 1, 1)
+        orc.set_kv_e4m3(np.array([0.05 * mult], dtype=np.float32), np.array([0.05 * mult], dtype=np.float32))
+        orc.append(0, x * 0.0, x * mult, 0, 1, 1)
+        outs.append(orc.read_layer(0)[1][0] / mult)
+    assert np.array_equal(outs[0], outs[1]) and np.array_equal(outs[0], outs[2])
+    assert np.abs(outs[0] - x).max() <= 2.0 ** -4 * np.abs(x).max()
+    orc = oracle_mod.Oracle(1, H, D, 1, 1, 1, 1)
+    orc.set_kv_e4m3(np.array([0.001], dtype=np.float32), np.array([0.001], dtype=np.float32))
+    big = np.full((1, H, D), 7.0)
+    orc.append(0, big * 0.0, -big, 0, 1, 1)
+    assert np.array_equal(orc.read_layer(0)[1][0], np.full((1, H, D), -448.0 * float(np.float32(0.001))))

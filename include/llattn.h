@@ -98,9 +98,40 @@ size_t ll_cache_storage_bytes(const ll_cache *cache);
  * descriptors.  The memory must outlive every later call on the handle. */
 int ll_cache_bind_storage(ll_cache *cache, void *dev, size_t bytes, ll_stream stream);
 
+/* 8-bit cache storage.  (The paper's appendix "Quantization" reports an INT8 variant of
+ * the whole model; it defines no cache format.  This one is the library's: the rotated
+ * keys and the values are kept as E4M3 codes - 1 sign, 4 exponent bits with bias 7, 3
+ * mantissa bits, largest magnitude 448, no infinities - times one fp32 scale per layer
+ * and head: code = E4M3(fl32(x) / scale), round to nearest even, saturating.)
+ *
+ * ll_cache_set_kv_format must come before ll_cache_bind_storage and changes
+ * ll_cache_storage_bytes: per layer K and V take heads*(S+W)*tokens_per_frame*head_dim
+ * bytes each (half of bf16), and the aux block grows by ONE bf16 K/V pair of a layer's
+ * size, shared by all layers: an attention call first expands the visible rows' codes
+ * into it (exactly: every E4M3 value is a bf16 value) and then runs the same kernel as
+ * the bf16 path, with the scales folded into the softmax scale (keys) and into the
+ * final normalisation (values).  Net effect at 30 layers of the benchmark shape: 1.84 GB
+ * instead of 3.45 GB resident.  Queries stay bf16.
+ *
+ * ll_cache_set_kv_scales: k_scale, v_scale are HOST arrays of `heads` positive floats
+ * for one layer (default 1.0 everywhere); they apply to rows written afterwards, and an
+ * attention call uses the scales in force when it is made, so set them before the
+ * layer's first append and leave them alone while rows written under them are resident.
+ * Copied to the device on `stream`.
+ *
+ * With LL_KV_E4M3: ll_rope_append_kv, ll_sink_window_attn (also batched, and mixed with
+ * bf16 caches in one launch), ll_recache and ll_clip_append_attn work as documented;
+ * ll_norm_rope_append_kv returns LL_ERR_UNSUPPORTED_SHAPE. */
+#define LL_KV_BF16 0
+#define LL_KV_E4M3 1
+int ll_cache_set_kv_format(ll_cache *cache, int format);
+int ll_cache_set_kv_scales(ll_cache *cache, int layer, const float *k_scale, const float *v_scale,
+                           ll_stream stream);
+
 /* Byte offset, inside the bound storage, of head `head` of layer `layer`'s K
  * (which = 0) or V (which = 1) matrix: (S+W)*tokens_per_frame rows of head_dim
- * bf16, row = slot * tokens_per_frame + token.  For tests and checkpointing. */
+ * bf16 (or E4M3 bytes), row = slot * tokens_per_frame + token.  For tests and
+ * checkpointing. */
 int ll_cache_kv_offset(const ll_cache *cache, int layer, int which, int head, size_t *offset);
 
 /* ---- the hot path --------------------------------------------------------- */

@@ -21,6 +21,7 @@ LL_ERR_NO_STORAGE = -4
 LL_ERR_CUDA = -5
 LL_ERR_DEVICE_TIMEOUT = -6
 LL_MAX_SLOTS = 64
+LL_KV_BF16, LL_KV_E4M3 = 0, 1
 LL_MAX_RANGES = 4
 LL_STATIC_MAX_FRAMES = 64
 LL_STATIC_MAX_GRID_SUM = 1024
@@ -92,6 +93,8 @@ SIGNATURES = {
     "ll_cache_destroy": (None, [C.c_void_p]),
     "ll_cache_storage_bytes": (C.c_size_t, [C.c_void_p]),
     "ll_cache_bind_storage": (C.c_int, [C.c_void_p, C.c_void_p, C.c_size_t, C.c_void_p]),
+    "ll_cache_set_kv_format": (C.c_int, [C.c_void_p, C.c_int]),
+    "ll_cache_set_kv_scales": (C.c_int, [C.c_void_p, C.c_int, C.POINTER(C.c_float), C.POINTER(C.c_float), C.c_void_p]),
     "ll_cache_kv_offset": (C.c_int, [C.c_void_p, C.c_int, C.c_int, C.c_int, C.POINTER(C.c_size_t)]),
     "ll_rope_append_kv": (C.c_int, [C.c_void_p, C.c_int, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int64,
                                     C.c_int, C.c_int, C.c_int, C.c_float, C.c_void_p, C.c_void_p]),
@@ -184,6 +187,18 @@ def ll_cache_storage_bytes(h) -> int:
 
 def ll_cache_bind_storage(h, storage, stream=None):
     _check(lib().ll_cache_bind_storage(h, _ptr(storage), storage.numel() * storage.element_size(), _stream(stream)))
+
+
+def ll_cache_set_kv_format(h, fmt: int):
+    _check(lib().ll_cache_set_kv_format(h, fmt))
+
+
+def ll_cache_set_kv_scales(h, layer, k_scale, v_scale, stream=None):
+    """k_scale, v_scale: sequences of `heads` floats (host)."""
+    n = len(k_scale)
+    ks = (C.c_float * n)(*[float(x) for x in k_scale])
+    vs = (C.c_float * n)(*[float(x) for x in v_scale])
+    _check(lib().ll_cache_set_kv_scales(h, layer, ks, vs, _stream(stream)))
 
 
 def ll_cache_kv_offset(h, layer, which, head) -> int:
@@ -322,12 +337,15 @@ class Cache:
     """Owns a handle plus the torch tensor that backs it.  Marshalling only."""
 
     def __init__(self, layers, heads, head_dim, tokens_per_frame, chunk_frames, sink_frames, window_frames,
-                 device="cuda:0", dry_run=False):
+                 device="cuda:0", dry_run=False, kv_format=0):
         self.L, self.H, self.D, self.P = layers, heads, head_dim, tokens_per_frame
         self.C, self.S, self.W = chunk_frames, sink_frames, window_frames
         self.h = ll_cache_create(layers, heads, head_dim, tokens_per_frame, chunk_frames, sink_frames,
                                  window_frames)
         self.storage = None
+        self.kv_format = kv_format
+        if kv_format:
+            ll_cache_set_kv_format(self.h, kv_format)
         if dry_run:
             ll_cache_set_dry_run(self.h, True)
         else:
@@ -359,12 +377,19 @@ class Cache:
                 "recaches": st.n_recaches, "attn_calls": st.n_attn_calls}
 
     def kv_view(self, layer, which):
-        """bf16 view [H, rows, D] of a layer's K (which=0) or V (which=1) matrix."""
+        """View [H, rows, D] of a layer's K (which=0) or V (which=1) matrix: bf16, or the
+        E4M3 codes as uint8 for an 8-bit cache."""
         import torch
         rows = (self.S + self.W) * self.P
         off = ll_cache_kv_offset(self.h, layer, which, 0)
+        if self.kv_format == LL_KV_E4M3:
+            n = self.H * rows * self.D
+            return self.storage[off:off + n].view(self.H, rows, self.D)
         n = self.H * rows * self.D * 2
         return self.storage[off:off + n].view(torch.bfloat16).view(self.H, rows, self.D)
+
+    def set_kv_scales(self, layer, k_scale, v_scale, stream=None):
+        ll_cache_set_kv_scales(self.h, layer, k_scale, v_scale, stream)
 
     def rope_append_kv(self, layer, q, k, v, frame_start, grid_h, grid_w, theta=10000.0, q_out=None, stream=None):
         ll_rope_append_kv(self.h, layer, q, k, v, frame_start, self.C, grid_h, grid_w, theta, q_out, stream)

@@ -462,14 +462,16 @@ attn_sm100_kernel(const __grid_constant__ AttnParams p, const __grid_constant__ 
             // Chunks 4..7 are at the same address ^ 64, the second eight rows 1024 bytes on.
             const uint32_t p_at = p_smem + w * C::kPBytes + (uint32_t)(32 * q + 16 * h + (lane & 7)) * 128 +
                                   ((uint32_t)((lane >> 3) ^ (lane & 7)) << 4);
-            const float c = p.scale_log2;
-            const uint64_t c2 = pack2(c, c);
             uint32_t sc = 0, oc = 0;
             Segment s;
             for (WorkIter it(p, cta); it.next(s);) {
                 if (w >= s.n_sub) continue;
                 const AttnGroup &G = p.g[s.g];
                 KeyIter kit(&G, s.kt0);
+                // log2(e)/sqrt(D), times the head's key scale when the cache holds 8-bit codes
+                const float *k_scale = p.item[G.item].k_scale;
+                const float c = k_scale ? p.scale_log2 * __ldg(k_scale + s.head) : p.scale_log2;
+                const uint64_t c2 = pack2(c, c);
                 float m_a = -INFINITY, m_b = -INFINITY;
                 uint64_t acc_a = 0ull, acc_b = 0ull;       // two partial sums per row
                 for (int j = s.kt0; j < s.kt1; ++j, kit.next(), ++sc) {
@@ -734,7 +736,8 @@ attn_sm100_kernel(const __grid_constant__ AttnParams p, const __grid_constant__ 
                             ll_b = fmaf(pb.y, ex2(pb.x - mm_b), ll_b);
                         }
                     }
-                    const float inv_a = 1.f / ll_a, inv_b = 1.f / ll_b;
+                    const float v_scale = item.v_scale ? __ldg(item.v_scale + s.head) : 1.f;   // 8-bit caches: value codes x scale
+                    const float inv_a = v_scale / ll_a, inv_b = v_scale / ll_b;
 #pragma unroll 1
                     for (int ch = 0; ch < C::kOChunks; ++ch) {
                         uint32_t o[32];

@@ -85,8 +85,36 @@ int encode_map(CUtensorMap *m, const void *base, uint64_t d0, uint64_t d1, uint6
     return LL_OK;
 }
 
-char *layer_k(const ll_cache *c, int layer) { return c->storage + c->aux_bytes + (size_t)layer * 2 * c->kv_bytes; }
-char *layer_v(const ll_cache *c, int layer) { return layer_k(c, layer) + c->kv_bytes; }
+char *layer_k(const ll_cache *c, int layer) { return c->storage + c->aux_bytes + (size_t)layer * 2 * c->kv_store_bytes; }
+char *layer_v(const ll_cache *c, int layer) { return layer_k(c, layer) + c->kv_store_bytes; }
+const float *layer_scales(const ll_cache *c, int layer, int which)
+{
+    return reinterpret_cast<const float *>(c->storage + c->off_scales) + ((size_t)layer * 2 + which) * c->H;
+}
+
+// Offsets of the aux block's parts and the size of a stored K (or V) matrix set.
+void compute_layout(ll_cache *c)
+{
+    int n_t, n_h;
+    rope_split(c->D, &n_t, &n_h);
+    c->off_status = 0;
+    c->off_ttab = align_up(ll::kStatusWords * sizeof(uint32_t), 256);
+    c->off_hwtab = align_up(c->off_ttab + (size_t)ll::kTTabFrames * n_t * sizeof(float2), 256);
+    // grid_h + grid_w <= tokens_per_frame + 1 for any grid with grid_h*grid_w == tokens_per_frame
+    c->off_counters = align_up(c->off_hwtab + (size_t)(c->P + 1) * n_h * sizeof(float2), 256);
+    c->off_partial = align_up(c->off_counters + ll::counters_bytes(), 1024);
+    size_t end = align_up(c->off_partial + 2 * (size_t)ll::kMaxCtas * ll::attn_slot_bytes(c->D), 1024);
+    c->kv_bytes = (size_t)c->H * c->rows * c->D * sizeof(ll_bf16);
+    c->kv_store_bytes = c->kv_bytes;
+    c->off_scales = c->off_stage = 0;
+    if (c->kv_format == LL_KV_E4M3) {
+        c->kv_store_bytes = c->kv_bytes / 2;
+        c->off_scales = end;
+        c->off_stage = align_up(c->off_scales + (size_t)c->L * 2 * c->H * sizeof(float), 1024);
+        end = align_up(c->off_stage + 2 * c->kv_bytes, 1024);
+    }
+    c->aux_bytes = end;
+}
 
 // Visible cache-row runs for queries of the chunk holding q_frame_start.
 int visible_ranges(const ll_cache *c, int layer, int64_t q_frame_start, int64_t lo_floor,
@@ -177,8 +205,10 @@ int fill_rope_params(ll_cache *c, int layer, const ll_bf16 *q, const ll_bf16 *k,
     int n_t, n_h;
     rope_split(c->D, &n_t, &n_h);
     p->q = q; p->k = k; p->v = v; p->q_out = q_out;
-    p->kcache = reinterpret_cast<ll_bf16 *>(layer_k(c, layer));
-    p->vcache = reinterpret_cast<ll_bf16 *>(layer_v(c, layer));
+    p->kcache = layer_k(c, layer);
+    p->vcache = layer_v(c, layer);
+    p->k_scale = c->kv_format == LL_KV_E4M3 ? layer_scales(c, layer, 0) : nullptr;
+    p->v_scale = c->kv_format == LL_KV_E4M3 ? layer_scales(c, layer, 1) : nullptr;
     const float2 *t_tab = reinterpret_cast<const float2 *>(c->storage + c->off_ttab);
     p->t_tab = t_tab + (size_t)(frame_start - c->t_base) * n_t;
     p->h_tab = reinterpret_cast<const float2 *>(c->storage + c->off_hwtab);
@@ -189,6 +219,12 @@ int fill_rope_params(ll_cache *c, int layer, const ll_bf16 *q, const ll_bf16 *k,
     p->n_t = n_t; p->n_h = n_h;
     for (int i = 0; i < n_frames; ++i) p->slot[i] = slot_of(c, frame_start + i);
     return LL_OK;
+}
+
+cudaError_t launch_append(const ll_cache *c, const ll::RopeAppendParams &p, cudaStream_t stream)
+{
+    return c->kv_format == LL_KV_E4M3 ? ll::launch_rope_append_e4m3(p, c->D, stream)
+                                      : ll::launch_rope_append(p, c->D, stream);
 }
 
 // One (cache, layer, q, out) of an attention launch and the chunks of queries it brings.
@@ -321,6 +357,9 @@ int build_attn_params(const AttnCall *calls, int n_calls, ll::AttnParams *p)
         p->kv_token_major = dense ? 1 : 0;
         p->item[i].out = call.out;
         p->item[i].lse = call.lse;
+        const bool e4m3 = !dense && c->kv_format == LL_KV_E4M3 && c->storage;
+        p->item[i].k_scale = e4m3 ? layer_scales(c, call.layer, 0) : nullptr;
+        p->item[i].v_scale = e4m3 ? layer_scales(c, call.layer, 1) : nullptr;
         p->item[i].nq_total = call.n_groups * rows_per_group;
         for (int g = 0; g < call.n_groups; ++g, ++ng) {
             ll::AttnGroup &G = p->g[ng];
@@ -382,6 +421,39 @@ int launch_attention(const AttnCall *calls, int n_calls, const ll::AttnParams &p
             if (st != LL_OK) return st;
             continue;
         }
+        if (c->kv_format == LL_KV_E4M3) {
+            // expand the codes of every cache row some group of this call can see into the bf16
+            // staging pair the kernel reads (the union of the groups' runs, merged by slot)
+            bool seen[LL_MAX_SLOTS] = {false};
+            for (int g = 0; g < p.n_groups; ++g) {
+                if (p.g[g].item != i) continue;
+                for (int r = 0; r < p.g[g].n_ranges; ++r)
+                    for (int sl = p.g[g].k_start[r] / c->P; sl < (p.g[g].k_start[r] + p.g[g].k_len[r]) / c->P; ++sl)
+                        seen[sl] = true;
+            }
+            ll::StageParams sp;
+            memset(&sp, 0, sizeof sp);
+            sp.k8 = reinterpret_cast<const uint8_t *>(layer_k(c, calls[i].layer));
+            sp.v8 = reinterpret_cast<const uint8_t *>(layer_v(c, calls[i].layer));
+            sp.k16 = reinterpret_cast<ll_bf16 *>(c->storage + c->off_stage);
+            sp.v16 = reinterpret_cast<ll_bf16 *>(c->storage + c->off_stage + c->kv_bytes);
+            sp.rows_per_head = c->rows;
+            sp.heads = c->H;
+            for (int sl = 0; sl < c->n_slots;) {
+                if (!seen[sl]) { ++sl; continue; }
+                int e = sl;
+                while (e < c->n_slots && seen[e]) ++e;
+                sp.start[sp.n_runs] = sl * c->P;
+                sp.len[sp.n_runs] = (e - sl) * c->P;
+                ++sp.n_runs;                                   // at most n_slots / 2 + 1 <= kMaxStageRuns runs
+                sl = e;
+            }
+            cudaError_t es = ll::launch_stage_e4m3(sp, c->D, stream);
+            if (es != cudaSuccess) return cuda_fail(es, "staging kernel of the 8-bit cache");
+            maps.k[i] = c->stage_kmap;
+            maps.v[i] = c->stage_vmap;
+            continue;
+        }
         maps.k[i] = c->kmap[calls[i].layer];
         maps.v[i] = c->vmap[calls[i].layer];
     }
@@ -414,6 +486,7 @@ int attn_entry(ll_cache *c, int layer, const ll_bf16 *q_roped, int64_t q_frame_s
 {
     int s = check_decode_item(c, layer, q_roped, q_frame_start, n_q_frames, out, lse_out);
     if (s != LL_OK) return s;
+    if (simt && c->kv_format != LL_KV_BF16) return fail(LL_ERR_UNSUPPORTED_SHAPE, "the triage kernel reads bf16 caches only");
     AttnCall call{c, layer, q_roped, out, lse_out, 1, {q_frame_start}, 0};
     ll::AttnParams p;
     s = build_attn_params(&call, 1, &p);
@@ -467,16 +540,8 @@ int ll_cache_create(int layers, int heads, int head_dim, int tokens_per_frame, i
     c->layers.resize(layers);
     for (auto &l : c->layers)
         for (int s = 0; s < LL_MAX_SLOTS; ++s) l.slot_frame[s] = -1;
-    int n_t, n_h;
-    rope_split(head_dim, &n_t, &n_h);
-    c->off_status = 0;
-    c->off_ttab = align_up(ll::kStatusWords * sizeof(uint32_t), 256);
-    c->off_hwtab = align_up(c->off_ttab + (size_t)ll::kTTabFrames * n_t * sizeof(float2), 256);
-    // grid_h + grid_w <= tokens_per_frame + 1 for any grid with grid_h*grid_w == tokens_per_frame
-    c->off_counters = align_up(c->off_hwtab + (size_t)(tokens_per_frame + 1) * n_h * sizeof(float2), 256);
-    c->off_partial = align_up(c->off_counters + ll::counters_bytes(), 1024);
-    c->aux_bytes = align_up(c->off_partial + 2 * (size_t)ll::kMaxCtas * ll::attn_slot_bytes(head_dim), 1024);
-    c->kv_bytes = (size_t)heads * rows * head_dim * sizeof(ll_bf16);
+    c->scales.assign((size_t)layers * 2 * heads, 1.f);
+    compute_layout(c);
     *out = c;
     return LL_OK;
 }
@@ -486,7 +551,7 @@ void ll_cache_destroy(ll_cache *cache) { delete cache; }
 size_t ll_cache_storage_bytes(const ll_cache *c)
 {
     if (!c) return 0;
-    return c->aux_bytes + (size_t)c->L * 2 * c->kv_bytes;
+    return c->aux_bytes + (size_t)c->L * 2 * c->kv_store_bytes;
 }
 
 int ll_cache_bind_storage(ll_cache *c, void *dev, size_t bytes, ll_stream stream)
@@ -506,7 +571,20 @@ int ll_cache_bind_storage(ll_cache *c, void *dev, size_t bytes, ll_stream stream
     c->sm_count = sms;
     std::vector<CUtensorMap> km(c->L), vm(c->L);
     char *base = static_cast<char *>(dev) + c->aux_bytes;
-    for (int l = 0; l < c->L; ++l) {
+    if (c->kv_format == LL_KV_E4M3) {
+        // the attention kernel reads the bf16 staging pair, whichever layer was expanded into it
+        char *k = static_cast<char *>(dev) + c->off_stage;
+        int s = encode_map(&c->stage_kmap, k, c->D, (uint64_t)c->rows, c->H, (uint64_t)c->D * 2,
+                           (uint64_t)c->rows * c->D * 2, 128, 1);
+        if (s != LL_OK) return s;
+        s = encode_map(&c->stage_vmap, k + c->kv_bytes, c->D, (uint64_t)c->rows, c->H, (uint64_t)c->D * 2,
+                       (uint64_t)c->rows * c->D * 2, 128, 1);
+        if (s != LL_OK) return s;
+        e = cudaMemcpyAsync(static_cast<char *>(dev) + c->off_scales, c->scales.data(), c->scales.size() * sizeof(float),
+                            cudaMemcpyHostToDevice, (cudaStream_t)stream);
+        if (e != cudaSuccess) return cuda_fail(e, "cudaMemcpyAsync(scales)");
+    }
+    for (int l = 0; l < c->L && c->kv_format == LL_KV_BF16; ++l) {
         char *k = base + (size_t)l * 2 * c->kv_bytes;
         int s = encode_map(&km[l], k, c->D, (uint64_t)c->rows, c->H, (uint64_t)c->D * 2,
                            (uint64_t)c->rows * c->D * 2, 128, 1);
@@ -522,12 +600,41 @@ int ll_cache_bind_storage(ll_cache *c, void *dev, size_t bytes, ll_stream stream
     return LL_OK;
 }
 
+int ll_cache_set_kv_format(ll_cache *c, int format)
+{
+    if (!c) return fail(LL_ERR_INVALID_ARG, "null handle");
+    if (format != LL_KV_BF16 && format != LL_KV_E4M3) return fail(LL_ERR_INVALID_ARG, "unknown cache format %d", format);
+    if (c->storage) return fail(LL_ERR_INVALID_ARG, "the cache format is fixed once storage is bound");
+    static_assert(LL_MAX_SLOTS / 2 + 1 <= ll::kMaxStageRuns, "staging run list too short");
+    c->kv_format = format;
+    compute_layout(c);
+    return LL_OK;
+}
+
+int ll_cache_set_kv_scales(ll_cache *c, int layer, const float *k_scale, const float *v_scale, ll_stream stream)
+{
+    if (!layer_ok(c, layer) || !k_scale || !v_scale) return fail(LL_ERR_INVALID_ARG, "bad argument to ll_cache_set_kv_scales");
+    if (c->kv_format != LL_KV_E4M3) return fail(LL_ERR_INVALID_ARG, "scales belong to the 8-bit cache format");
+    for (int h = 0; h < c->H; ++h)
+        if (!(k_scale[h] > 0.f) || !(v_scale[h] > 0.f) || !std::isfinite(k_scale[h]) || !std::isfinite(v_scale[h]))
+            return fail(LL_ERR_INVALID_ARG, "scales must be positive and finite");
+    float *dst = c->scales.data() + (size_t)layer * 2 * c->H;
+    memcpy(dst, k_scale, c->H * sizeof(float));
+    memcpy(dst + c->H, v_scale, c->H * sizeof(float));
+    if (c->storage && !c->dry_run) {
+        cudaError_t e = cudaMemcpyAsync(c->storage + c->off_scales + (size_t)layer * 2 * c->H * sizeof(float), dst,
+                                        2 * c->H * sizeof(float), cudaMemcpyHostToDevice, (cudaStream_t)stream);
+        if (e != cudaSuccess) return cuda_fail(e, "cudaMemcpyAsync(scales)");
+    }
+    return LL_OK;
+}
+
 int ll_cache_kv_offset(const ll_cache *c, int layer, int which, int head, size_t *offset)
 {
     if (!layer_ok(c, layer) || !offset || which < 0 || which > 1 || head < 0 || head >= c->H)
         return fail(LL_ERR_INVALID_ARG, "bad argument to ll_cache_kv_offset");
-    *offset = c->aux_bytes + (size_t)layer * 2 * c->kv_bytes + (size_t)which * c->kv_bytes +
-              (size_t)head * c->rows * c->D * sizeof(ll_bf16);
+    *offset = c->aux_bytes + (size_t)layer * 2 * c->kv_store_bytes + (size_t)which * c->kv_store_bytes +
+              (size_t)head * (c->kv_store_bytes / c->H);
     return LL_OK;
 }
 
@@ -542,6 +649,8 @@ int append_entry(ll_cache *c, int layer, const ll_bf16 *q, const ll_bf16 *k, con
     if (grid_h <= 0 || grid_w <= 0 || (int64_t)grid_h * grid_w != c->P)
         return fail(LL_ERR_INVALID_ARG, "grid %dx%d does not give %d tokens per frame", grid_h, grid_w, c->P);
     if (!(rope_theta > 0.f)) return fail(LL_ERR_INVALID_ARG, "rope_theta must be positive");
+    if (with_norm && c->kv_format != LL_KV_BF16)
+        return fail(LL_ERR_UNSUPPORTED_SHAPE, "the fused norm is built for bf16 caches only");
     if (n_frames != c->C) return fail(LL_ERR_BAD_POSITION, "n_frames %d != chunk_frames %d", n_frames, c->C);
     ll::LayerState &st = c->layers[layer];
     const bool is_new = frame_start == st.end;
@@ -565,7 +674,7 @@ int append_entry(ll_cache *c, int layer, const ll_bf16 *q, const ll_bf16 *k, con
         ll::RopeAppendParams p;
         fill_rope_params(c, layer, q_out ? q : nullptr, k, v, q_out, frame_start, n_frames, grid_w, &p);
         cudaError_t e = with_norm ? ll::launch_norm_rope_append(p, c->D, gain_q, gain_k, eps, (cudaStream_t)stream)
-                                  : ll::launch_rope_append(p, c->D, (cudaStream_t)stream);
+                                  : launch_append(c, p, (cudaStream_t)stream);
         if (e != cudaSuccess) return cuda_fail(e, "rope+append kernel");
     }
     if (is_new) {
@@ -676,7 +785,7 @@ int ll_recache(ll_cache *c, int layer, const ll_bf16 *q, const ll_bf16 *k, const
         if (s != LL_OK) return s;
         ll::RopeAppendParams rp;
         fill_rope_params(c, layer, q, k, v, q_out, r0, n_frames, grid_w, &rp);
-        cudaError_t e = ll::launch_rope_append(rp, c->D, (cudaStream_t)stream);
+        cudaError_t e = launch_append(c, rp, (cudaStream_t)stream);
         if (e != cudaSuccess) return cuda_fail(e, "rope+append kernel (recache)");
         s = launch_attention(&call, 1, ap, (cudaStream_t)stream, false);
         if (s != LL_OK) return s;
@@ -763,7 +872,7 @@ int ll_clip_append_attn(ll_cache *c, int layer, const ll_bf16 *q, const ll_bf16 
         if (s == LL_OK) {
             ll::RopeAppendParams rp;
             fill_rope_params(c, layer, q, k, v, q_out, frame_start, n_frames, grid_w, &rp);
-            cudaError_t e = ll::launch_rope_append(rp, c->D, (cudaStream_t)stream);
+            cudaError_t e = launch_append(c, rp, (cudaStream_t)stream);
             if (e != cudaSuccess) s = cuda_fail(e, "rope+append kernel (clip)");
         }
         if (s == LL_OK) s = launch_attention(&call, 1, ap, (cudaStream_t)stream, false);

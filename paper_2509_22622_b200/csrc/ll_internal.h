@@ -71,6 +71,8 @@ inline size_t attn_slot_bytes(int head_dim) { return (size_t)kQTileRows * (head_
 struct AttnItem {
     ll_bf16 *out;                     // [nq_total, H, D]
     float *lse;                       // [H, nq_total] or null
+    const float *k_scale;             // [H] per-head factor on the keys (8-bit caches), or null
+    const float *v_scale;             // [H] per-head factor on the values, or null
     int nq_total;                     // rows of this item's q / out
     int pad;
 };
@@ -109,7 +111,8 @@ struct AttnParams {
 struct RopeAppendParams {
     const ll_bf16 *q, *k, *v;         // [n_tokens, H, D]; q may be null
     ll_bf16 *q_out;                   // nullable
-    ll_bf16 *kcache, *vcache;         // layer base, [H][rows][D]
+    void *kcache, *vcache;            // layer base, [H][rows][D] of bf16 or of E4M3 codes
+    const float *k_scale, *v_scale;   // [H], 8-bit caches only: codes hold value / scale
     const float2 *t_tab;              // entry of the call's first frame: [frame][n_t] (cos, sin)
     const float2 *h_tab;              // [grid_h][n_h]
     const float2 *w_tab;              // [grid_w][n_w]
@@ -124,6 +127,18 @@ cudaError_t launch_rope_tables(float2 *t_tab, int64_t t_base, int n_t_frames, in
                                float2 *h_tab, int grid_h, float2 *w_tab, int grid_w, int n_hw,
                                float theta, bool do_t, bool do_hw, cudaStream_t stream);
 cudaError_t launch_rope_append(const RopeAppendParams &p, int head_dim, cudaStream_t stream);
+cudaError_t launch_rope_append_e4m3(const RopeAppendParams &p, int head_dim, cudaStream_t stream);
+// E4M3 codes of the cache-row runs [start, start + len) of every head -> bf16 values (the codes
+// themselves, scales not applied) at the same rows of a bf16 matrix set of the same shape
+constexpr int kMaxStageRuns = LL_MAX_SLOTS / 2 + 1;
+struct StageParams {
+    const uint8_t *k8, *v8;           // [H][rows][D] codes
+    ll_bf16 *k16, *v16;               // [H][rows][D]
+    int64_t rows_per_head;
+    int heads, n_runs;
+    int start[kMaxStageRuns], len[kMaxStageRuns];
+};
+cudaError_t launch_stage_e4m3(const StageParams &p, int head_dim, cudaStream_t stream);
 cudaError_t launch_norm_rope_append(const RopeAppendParams &p, int head_dim, const float *gain_q, const float *gain_k,
                                     float eps, cudaStream_t stream);
 cudaError_t launch_attn_sm100(const AttnParams &p, int head_dim, const AttnMaps &maps, cudaStream_t stream);
@@ -150,8 +165,14 @@ struct ll_cache {
     // aux block layout (byte offsets from storage)
     size_t off_status = 0, off_ttab = 0, off_hwtab = 0, off_counters = 0, off_partial = 0, aux_bytes = 0;
     int sm_count = 0;                 // of the device the storage lives on
-    size_t kv_bytes = 0;              // one K (or V) matrix set of one layer: H*rows*D*2
+    size_t kv_bytes = 0;              // one K (or V) matrix set of one layer in bf16: H*rows*D*2
+    size_t kv_store_bytes = 0;        // the same as stored: kv_bytes, or half of it for E4M3 codes
     std::vector<CUtensorMap> kmap, vmap;
+    // 8-bit storage: codes per layer, one bf16 staging pair shared by all layers, scales [L][2][H]
+    int kv_format = LL_KV_BF16;
+    size_t off_scales = 0, off_stage = 0;
+    CUtensorMap stage_kmap, stage_vmap;
+    std::vector<float> scales;        // host copy, [L][2][H]
 
     // which RoPE tables are resident
     bool hw_valid = false;

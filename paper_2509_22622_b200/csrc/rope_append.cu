@@ -102,11 +102,112 @@ rope_append_kernel(const __grid_constant__ RopeAppendParams p)
     for (int u = 0; u < kHeadsPerThread; ++u) {
         if (h0 + u < p.heads) {
             const size_t dst = (((size_t)(h0 + u)) * p.rows_per_head + cache_row) * D + (size_t)vec * 8;
-            st16(p.kcache + dst, rotate_vec(kk[u], cs));
-            st16(p.vcache + dst, kv[u]);
+            st16(static_cast<ll_bf16 *>(p.kcache) + dst, rotate_vec(kk[u], cs));
+            st16(static_cast<ll_bf16 *>(p.vcache) + dst, kv[u]);
             if (p.q_out) st16(p.q_out + in_base + (size_t)u * D, rotate_vec(kq[u], cs));
         }
     }
+}
+
+// ---- the same into an 8-bit cache ---------------------------------------------------------
+//
+// K (rotated, fp32) and V are divided by their head's scale (IEEE division) and rounded to
+// E4M3, round to nearest even, saturating; a thread's eight elements make one 8-byte store, 16
+// consecutive threads cover a 128-byte cache row.  Q is rotated to bf16 as in the bf16 kernel.
+__device__ __forceinline__ uint2 quantise_vec(const float (&x)[8], float scale)
+{
+    uint32_t c[4];
+#pragma unroll
+    for (int u = 0; u < 4; ++u) c[u] = cvt_e4m3x2(__fdiv_rn(x[2 * u], scale), __fdiv_rn(x[2 * u + 1], scale));
+    return make_uint2(c[0] | (c[1] << 16), c[2] | (c[3] << 16));
+}
+
+template <int D>
+__global__ void __launch_bounds__(kThreads)
+rope_append_e4m3_kernel(const __grid_constant__ RopeAppendParams p)
+{
+    constexpr int kVecs = D / 8;
+    const int head_groups = (p.heads + kHeadsPerThread - 1) / kHeadsPerThread;
+    const long long gid = (long long)blockIdx.x * kThreads + threadIdx.x;
+    const int vec = (int)(gid % kVecs);
+    const long long rest = gid / kVecs;
+    const int hg = (int)(rest % head_groups);
+    const long long token = rest / head_groups;
+    if (token >= p.n_tokens) return;
+
+    const int frame = (int)(token / p.P);
+    const int cell = (int)(token % p.P);
+    const int y = cell / p.grid_w, x = cell % p.grid_w;
+    float2 cs[4];
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+        const int j = vec * 4 + u;
+        const float2 *src;
+        if (j < p.n_t)             src = p.t_tab + (size_t)frame * p.n_t + j;
+        else if (j < p.n_t + p.n_h) src = p.h_tab + (size_t)y * p.n_h + (j - p.n_t);
+        else                        src = p.w_tab + (size_t)x * p.n_h + (j - p.n_t - p.n_h);
+        cs[u] = __ldg(src);
+    }
+    const int h0 = hg * kHeadsPerThread;
+    const size_t in_base = ((size_t)token * p.heads + h0) * D + (size_t)vec * 8;
+    const size_t cache_row = (size_t)p.slot[frame] * p.P + cell;
+    uint8_t *kc = static_cast<uint8_t *>(p.kcache), *vc = static_cast<uint8_t *>(p.vcache);
+#pragma unroll
+    for (int u = 0; u < kHeadsPerThread; ++u) {
+        if (h0 + u >= p.heads) break;
+        const uint4 k = ld16(p.k + in_base + (size_t)u * D);
+        const uint4 v = ld16(p.v + in_base + (size_t)u * D);
+        const uint32_t kw[4] = {k.x, k.y, k.z, k.w}, vw[4] = {v.x, v.y, v.z, v.w};
+        float kr[8], vr[8];
+#pragma unroll
+        for (int t = 0; t < 4; ++t) {
+            rotate_pair_f32(kw[t], cs[t], kr[2 * t], kr[2 * t + 1]);
+            vr[2 * t] = __uint_as_float(vw[t] << 16);
+            vr[2 * t + 1] = __uint_as_float(vw[t] & 0xffff0000u);
+        }
+        const size_t dst = (((size_t)(h0 + u)) * p.rows_per_head + cache_row) * D + (size_t)vec * 8;
+        *reinterpret_cast<uint2 *>(kc + dst) = quantise_vec(kr, __ldg(p.k_scale + h0 + u));
+        *reinterpret_cast<uint2 *>(vc + dst) = quantise_vec(vr, __ldg(p.v_scale + h0 + u));
+        if (p.q_out) st16(p.q_out + in_base + (size_t)u * D, rotate_vec(ld16(p.q + in_base + (size_t)u * D), cs));
+    }
+}
+
+// Codes of the listed cache-row runs, all heads, K and V: to bf16 at the same rows of the
+// staging pair.  One thread converts 16 codes (one 16-byte load, two 16-byte stores).
+template <int D>
+__global__ void __launch_bounds__(kThreads)
+stage_e4m3_kernel(const __grid_constant__ StageParams p)
+{
+    constexpr int kVecs = D / 16;                      // 16-code vectors per row
+    long long gid = (long long)blockIdx.x * kThreads + threadIdx.x;
+    const int vec = (int)(gid % kVecs);
+    gid /= kVecs;
+    int run = 0;
+    long long rows_before = 0;
+    // threads are numbered run by run, within a run head-major over its rows
+    while (run < p.n_runs && gid >= rows_before + (long long)p.len[run] * p.heads) {
+        rows_before += (long long)p.len[run] * p.heads;
+        ++run;
+    }
+    if (run >= p.n_runs) return;
+    const long long r = gid - rows_before;
+    const int head = (int)(r / p.len[run]);
+    const long long row = p.start[run] + r % p.len[run];
+    const size_t off = ((size_t)head * p.rows_per_head + row) * D + (size_t)vec * 16;
+    auto expand = [&](const uint8_t *src, ll_bf16 *dst) {
+        const uint4 c = *reinterpret_cast<const uint4 *>(src + off);
+        const uint32_t w[4] = {c.x, c.y, c.z, c.w};
+        uint32_t o[8];
+#pragma unroll
+        for (int t = 0; t < 4; ++t) {
+            o[2 * t] = e4m3x2_to_bf16x2(w[t] & 0xffffu);
+            o[2 * t + 1] = e4m3x2_to_bf16x2(w[t] >> 16);
+        }
+        st16(dst + off, make_uint4(o[0], o[1], o[2], o[3]));
+        st16(dst + off + 8, make_uint4(o[4], o[5], o[6], o[7]));
+    };
+    expand(p.k8, p.k16);
+    expand(p.v8, p.v16);
 }
 
 // ---- the same with the RMS norm of q and k in front -----------------------------------
@@ -219,8 +320,8 @@ norm_rope_append_kernel(const __grid_constant__ RopeAppendParams p, const float 
         const int head = v / kVecs;
         const size_t src = in_base + (size_t)v * 8;
         const size_t dst = ((size_t)head * p.rows_per_head + cache_row) * D + (size_t)vec * 8;
-        st16(p.kcache + dst, norm_rotate_vec(xk, rk, gain_k + (size_t)v * 8, cs));
-        st16(p.vcache + dst, xv);
+        st16(static_cast<ll_bf16 *>(p.kcache) + dst, norm_rotate_vec(xk, rk, gain_k + (size_t)v * 8, cs));
+        st16(static_cast<ll_bf16 *>(p.vcache) + dst, xv);
         if (with_q) st16(p.q_out + src, norm_rotate_vec(xq, rq, gain_q + (size_t)v * 8, cs));
     };
     if (kIters > 0) {
@@ -270,6 +371,31 @@ cudaError_t launch_rope_tables(float2 *t_tab, int64_t t_base, int n_t_frames, in
     int blocks = (total + 127) / 128;
     rope_table_kernel<<<blocks, 128, 0, stream>>>(t_tab, (long long)t_base, n_t_frames, n_t, h_tab, grid_h,
                                                   w_tab, grid_w, n_hw, (double)theta, do_t, do_hw);
+    count_launch();
+    return cudaGetLastError();
+}
+
+cudaError_t launch_rope_append_e4m3(const RopeAppendParams &p, int head_dim, cudaStream_t stream)
+{
+    const int head_groups = (p.heads + kHeadsPerThread - 1) / kHeadsPerThread;
+    const long long threads = (long long)p.n_tokens * head_groups * (head_dim / 8);
+    const unsigned blocks = (unsigned)((threads + kThreads - 1) / kThreads);
+    if (blocks == 0) return cudaSuccess;
+    if (head_dim == 128) rope_append_e4m3_kernel<128><<<blocks, kThreads, 0, stream>>>(p);
+    else                 rope_append_e4m3_kernel<64><<<blocks, kThreads, 0, stream>>>(p);
+    count_launch();
+    return cudaGetLastError();
+}
+
+cudaError_t launch_stage_e4m3(const StageParams &p, int head_dim, cudaStream_t stream)
+{
+    long long rows = 0;
+    for (int i = 0; i < p.n_runs; ++i) rows += (long long)p.len[i] * p.heads;
+    const long long threads = rows * (head_dim / 16);
+    const unsigned blocks = (unsigned)((threads + kThreads - 1) / kThreads);
+    if (blocks == 0) return cudaSuccess;
+    if (head_dim == 128) stage_e4m3_kernel<128><<<blocks, kThreads, 0, stream>>>(p);
+    else                 stage_e4m3_kernel<64><<<blocks, kThreads, 0, stream>>>(p);
     count_launch();
     return cudaGetLastError();
 }

@@ -177,6 +177,36 @@ int ll_norm_rope_append_kv(ll_cache *cache, int layer, const ll_bf16 *q, const l
                            int64_t frame_start, int n_frames, int grid_h, int grid_w,
                            float rope_theta, ll_bf16 *q_out, ll_stream stream);
 
+/* The QKV projection of a DiT self-attention layer (Sec. 3.1: the block this path sits
+ * in; the projection itself is the base model's, the paper does not restate it) with the
+ * front end of the path in the GEMM's epilogue: one tcgen05 GEMM
+ *     y = x W^T + b,   q | k | v = y
+ * whose accumulators go through the optional q/k RMS norm (as in
+ * ll_norm_rope_append_kv), the 3-D rotation and the append without a round trip
+ * through memory: v rows and rotated k rows land in the cache, rotated q in q_out.
+ *   x        device, bf16 [n_frames*tokens_per_frame, d_model]; d_model a multiple of 8
+ *   w_qkv    device, bf16 [3*heads*head_dim, d_model]: q features, then k, then v
+ *   bias     device, fp32 [3*heads*head_dim], nullable
+ *   gain_q, gain_k  device, fp32 [heads*head_dim]; both NULL: no norm
+ *   q_out    device, bf16 [tokens, heads, head_dim]
+ * With the norm, a token's factor 1/sqrt(mean(q^2) + eps) is known only when all its
+ * heads are done, and they are computed by different thread blocks.  So q_out receives
+ * rotate(gain * q) WITHOUT that factor and q_row_scale[token] (device, fp32 [tokens])
+ * receives the factor: pass both to ll_sink_window_attn_scaled, which folds the factor
+ * into the row's softmax scale.  k rows are completed inside the call (a second small
+ * kernel), for which it needs `workspace`: device, 256-byte aligned, at least
+ * ll_qkv_proj_workspace_bytes (4 bytes per k element of a chunk plus a table of partial
+ * sums), caller-owned, free again when the call's kernels have run.  Without the norm
+ * q_row_scale and workspace may be NULL.
+ * heads*head_dim must be a multiple of 256; bf16 caches only; positions, state and errors
+ * as ll_rope_append_kv. */
+size_t ll_qkv_proj_workspace_bytes(const ll_cache *cache);
+int ll_qkv_proj_append(ll_cache *cache, int layer, const ll_bf16 *x, int d_model, const ll_bf16 *w_qkv,
+                       const float *bias, const float *gain_q, const float *gain_k, float eps,
+                       int64_t frame_start, int n_frames, int grid_h, int grid_w, float rope_theta,
+                       ll_bf16 *q_out, float *q_row_scale, void *workspace, size_t workspace_bytes,
+                       ll_stream stream);
+
 /* Sink+window attention of the newest chunk's queries (Sec. 3.3): every query
  * attends to all sink rows and all resident window rows (the chunk itself
  * included; bidirectional inside the chunk), softmax scale 1/sqrt(head_dim).
@@ -191,6 +221,14 @@ int ll_norm_rope_append_kv(ll_cache *cache, int layer, const ll_bf16 *q, const l
 int ll_sink_window_attn(ll_cache *cache, int layer, const ll_bf16 *q_roped,
                         int64_t q_frame_start, int n_q_frames, ll_bf16 *out,
                         float *lse_out, ll_stream stream);
+
+/* The same with one extra factor per query row on the scores (q_row_scale: device, fp32
+ * [n_q_frames*tokens_per_frame], 16-byte aligned; NULL = 1): row i attends with
+ * softmax scale q_row_scale[i]/sqrt(head_dim).  For queries whose normalisation factor
+ * was left out of q_roped (ll_qkv_proj_append). */
+int ll_sink_window_attn_scaled(ll_cache *cache, int layer, const ll_bf16 *q_roped, const float *q_row_scale,
+                               int64_t q_frame_start, int n_q_frames, ll_bf16 *out, float *lse_out,
+                               ll_stream stream);
 
 /* The same for several independent streams in ONE launch (serving: the streams
  * of a batch sit at different positions, with windows filled to different

@@ -151,6 +151,19 @@ def rms_norm(x, gain, eps: float):
     return y
 
 
+def qkv_proj(x, w, bias=None):
+    """The layer's QKV projection (upstream of the path; Sec. 3.1 names the block, the base
+    model defines the projection): y = x W^T + b in fp64 with the library matrix product.
+    x [tokens, d_model], w [3*H*D, d_model] (q features, then k, then v), bias [3*H*D] or None.
+    Returns (q, k, v), each [tokens, H*D]."""
+    x, w = _f64(x), _f64(w)
+    y = x @ w.T
+    if bias is not None:
+        y = y + _f64(bias)[None, :]
+    n = w.shape[0] // 3
+    return y[:, :n], y[:, n:2 * n], y[:, 2 * n:]
+
+
 def dense_attn(q, k, v, rows=None):
     """Plain softmax attention, every query over every key (cross-attention, Sec. 3.1).
     q [n_q, H, D], k and v [n_k, H, D].  Returns (out [n_rows, H, D], lse [n_rows, H])."""

@@ -103,6 +103,12 @@ SIGNATURES = {
                                          C.c_void_p, C.c_void_p]),
     "ll_sink_window_attn": (C.c_int, [C.c_void_p, C.c_int, C.c_void_p, C.c_int64, C.c_int, C.c_void_p,
                                       C.c_void_p, C.c_void_p]),
+    "ll_sink_window_attn_scaled": (C.c_int, [C.c_void_p, C.c_int, C.c_void_p, C.c_void_p, C.c_int64, C.c_int, C.c_void_p,
+                                             C.c_void_p, C.c_void_p]),
+    "ll_qkv_proj_workspace_bytes": (C.c_size_t, [C.c_void_p]),
+    "ll_qkv_proj_append": (C.c_int, [C.c_void_p, C.c_int, C.c_void_p, C.c_int, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p,
+                                     C.c_float, C.c_int64, C.c_int, C.c_int, C.c_int, C.c_float, C.c_void_p, C.c_void_p,
+                                     C.c_void_p, C.c_size_t, C.c_void_p]),
     "ll_sink_window_attn_batched": (C.c_int, [C.POINTER(ll_attn_item), C.c_int, C.c_void_p]),
     "ll_cross_attn": (C.c_int, [C.c_void_p, C.c_void_p, C.c_int64, C.c_void_p, C.c_void_p, C.c_int64, C.c_void_p,
                                 C.c_void_p, C.c_void_p]),
@@ -223,6 +229,24 @@ def ll_norm_rope_append_kv(h, layer, q, k, v, gain_q, gain_k, eps, frame_start, 
 def ll_sink_window_attn(h, layer, q_roped, q_frame_start, n_q_frames, out, lse_out=None, stream=None):
     _check(lib().ll_sink_window_attn(h, layer, _ptr(q_roped), q_frame_start, n_q_frames, _ptr(out),
                                      _ptr(lse_out), _stream(stream)))
+
+
+def ll_sink_window_attn_scaled(h, layer, q_roped, q_row_scale, q_frame_start, n_q_frames, out, lse_out=None,
+                               stream=None):
+    _check(lib().ll_sink_window_attn_scaled(h, layer, _ptr(q_roped), _ptr(q_row_scale), q_frame_start, n_q_frames,
+                                            _ptr(out), _ptr(lse_out), _stream(stream)))
+
+
+def ll_qkv_proj_workspace_bytes(h) -> int:
+    return lib().ll_qkv_proj_workspace_bytes(h)
+
+
+def ll_qkv_proj_append(h, layer, x, w_qkv, bias, gain_q, gain_k, eps, frame_start, n_frames, grid_h, grid_w,
+                       rope_theta, q_out, q_row_scale=None, workspace=None, stream=None):
+    nbytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
+    _check(lib().ll_qkv_proj_append(h, layer, _ptr(x), x.shape[-1], _ptr(w_qkv), _ptr(bias), _ptr(gain_q), _ptr(gain_k),
+                                    eps, frame_start, n_frames, grid_h, grid_w, rope_theta, _ptr(q_out),
+                                    _ptr(q_row_scale), _ptr(workspace), nbytes, _stream(stream)))
 
 
 def ll_sink_window_attn_batched(items, stream=None):

@@ -471,7 +471,15 @@ attn_sm100_kernel(const __grid_constant__ AttnParams p, const __grid_constant__ 
                 // log2(e)/sqrt(D), times the head's key scale when the cache holds 8-bit codes
                 const float *k_scale = p.item[G.item].k_scale;
                 const float c = k_scale ? p.scale_log2 * __ldg(k_scale + s.head) : p.scale_log2;
-                const uint64_t c2 = pack2(c, c);
+                // ... and times the query row's own factor when the caller brings one (a q/k norm whose
+                // per-token factor was left out of the stored q)
+                float c_a = c, c_b = c;
+                if (const float *q_scale = p.item[G.item].q_scale) {
+                    const int r = 128 * w + row_a;
+                    if (r < s.rows_valid) c_a *= __ldg(q_scale + s.q0 + r);
+                    if (r + 8 < s.rows_valid) c_b *= __ldg(q_scale + s.q0 + r + 8);
+                }
+                const uint64_t c2a = pack2(c_a, c_a), c2b = pack2(c_b, c_b);
                 float m_a = -INFINITY, m_b = -INFINITY;
                 uint64_t acc_a = 0ull, acc_b = 0ull;       // two partial sums per row
                 for (int j = s.kt0; j < s.kt1; ++j, kit.next(), ++sc) {
@@ -500,8 +508,8 @@ attn_sm100_kernel(const __grid_constant__ AttnParams p, const __grid_constant__ 
                         uint64_t ts_a = 0ull, ts_b = 0ull;         // the piece's sums, two partials per row
                         {
                             const uint64_t na2 = pack2(-m_a, -m_a), nb2 = pack2(-m_b, -m_b);
-                            const PolyRow ra{c * (1.f / 128.f), ((float)kPolyLow - m_a) * (1.f / 128.f)};
-                            const PolyRow rb{c * (1.f / 128.f), ((float)kPolyLow - m_b) * (1.f / 128.f)};
+                            const PolyRow ra{c_a * (1.f / 128.f), ((float)kPolyLow - m_a) * (1.f / 128.f)};
+                            const PolyRow rb{c_b * (1.f / 128.f), ((float)kPolyLow - m_b) * (1.f / 128.f)};
                             // Four 8-key groups at a time, stage by stage, so that the exponentials of a
                             // batch are all in flight before the first result is needed.
 #pragma unroll
@@ -511,8 +519,8 @@ attn_sm100_kernel(const __grid_constant__ AttnParams p, const __grid_constant__ 
                                 for (int kk = 0; kk < 4; ++kk) {
                                     const int k = 4 * g + kk;
                                     if (!((kPolyMask >> (8 * piece + k)) & 1u)) {
-                                        xa[kk] = fma2(pack2(as_f(v[4 * k]), as_f(v[4 * k + 1])), c2, na2);
-                                        xb[kk] = fma2(pack2(as_f(v[4 * k + 2]), as_f(v[4 * k + 3])), c2, nb2);
+                                        xa[kk] = fma2(pack2(as_f(v[4 * k]), as_f(v[4 * k + 1])), c2a, na2);
+                                        xb[kk] = fma2(pack2(as_f(v[4 * k + 2]), as_f(v[4 * k + 3])), c2b, nb2);
                                     }
                                 }
 #pragma unroll
@@ -557,8 +565,8 @@ attn_sm100_kernel(const __grid_constant__ AttnParams p, const __grid_constant__ 
                             }
                             ta = fmaxf(ta, __shfl_xor_sync(0xffffffffu, ta, 1));
                             tb = fmaxf(tb, __shfl_xor_sync(0xffffffffu, tb, 1));
-                            ta = fmaxf(ta, __shfl_xor_sync(0xffffffffu, ta, 2)) * c;
-                            tb = fmaxf(tb, __shfl_xor_sync(0xffffffffu, tb, 2)) * c;
+                            ta = fmaxf(ta, __shfl_xor_sync(0xffffffffu, ta, 2)) * c_a;
+                            tb = fmaxf(tb, __shfl_xor_sync(0xffffffffu, tb, 2)) * c_b;
                             const bool fresh = j == s.kt0 && piece == 0;     // nothing accumulated yet
                             const float new_a = fresh ? ta : fmaxf(m_a, ta), new_b = fresh ? tb : fmaxf(m_b, tb);
                             const float al_a = fresh ? 0.f : ex2(m_a - new_a), al_b = fresh ? 0.f : ex2(m_b - new_b);
@@ -613,8 +621,8 @@ attn_sm100_kernel(const __grid_constant__ AttnParams p, const __grid_constant__ 
                             ts_a = ts_b = 0ull;
 #pragma unroll
                             for (int k = 0; k < 8; ++k) {
-                                const uint64_t pa = exp2_sfu2(fma2(pack2(as_f(v[4 * k]), as_f(v[4 * k + 1])), c2, na2));
-                                const uint64_t pb = exp2_sfu2(fma2(pack2(as_f(v[4 * k + 2]), as_f(v[4 * k + 3])), c2, nb2));
+                                const uint64_t pa = exp2_sfu2(fma2(pack2(as_f(v[4 * k]), as_f(v[4 * k + 1])), c2a, na2));
+                                const uint64_t pb = exp2_sfu2(fma2(pack2(as_f(v[4 * k + 2]), as_f(v[4 * k + 3])), c2b, nb2));
                                 ts_a = add2(ts_a, pa);
                                 ts_b = add2(ts_b, pb);
                                 float a0, a1, b0, b1;

@@ -242,6 +242,7 @@ struct AttnCall {
     // token-major k/v tensors given here; the cache lends its shape and scratch only
     int64_t dense_rows, dense_keys;
     const ll_bf16 *dense_k, *dense_v;
+    const float *q_scale;                         // per-row factor on the queries, or null
 };
 
 // Divide the columns of all groups between the CTAs (one persistent CTA per SM).  The
@@ -358,6 +359,7 @@ int build_attn_params(const AttnCall *calls, int n_calls, ll::AttnParams *p)
         p->item[i].out = call.out;
         p->item[i].lse = call.lse;
         const bool e4m3 = !dense && c->kv_format == LL_KV_E4M3 && c->storage;
+        p->item[i].q_scale = call.q_scale;
         p->item[i].k_scale = e4m3 ? layer_scales(c, call.layer, 0) : nullptr;
         p->item[i].v_scale = e4m3 ? layer_scales(c, call.layer, 1) : nullptr;
         p->item[i].nq_total = call.n_groups * rows_per_group;
@@ -482,12 +484,13 @@ int check_decode_item(ll_cache *c, int layer, const ll_bf16 *q_roped, int64_t q_
 }
 
 int attn_entry(ll_cache *c, int layer, const ll_bf16 *q_roped, int64_t q_frame_start, int n_q_frames,
-               ll_bf16 *out, float *lse_out, ll_stream stream, bool simt)
+               ll_bf16 *out, float *lse_out, ll_stream stream, bool simt, const float *q_scale = nullptr)
 {
     int s = check_decode_item(c, layer, q_roped, q_frame_start, n_q_frames, out, lse_out);
     if (s != LL_OK) return s;
     if (simt && c->kv_format != LL_KV_BF16) return fail(LL_ERR_UNSUPPORTED_SHAPE, "the triage kernel reads bf16 caches only");
     AttnCall call{c, layer, q_roped, out, lse_out, 1, {q_frame_start}, 0};
+    call.q_scale = q_scale;
     ll::AttnParams p;
     s = build_attn_params(&call, 1, &p);
     if (s != LL_OK) return s;
@@ -714,6 +717,97 @@ int ll_sink_window_attn(ll_cache *c, int layer, const ll_bf16 *q_roped, int64_t 
                         int n_q_frames, ll_bf16 *out, float *lse_out, ll_stream stream)
 {
     return attn_entry(c, layer, q_roped, q_frame_start, n_q_frames, out, lse_out, stream, false);
+}
+
+int ll_sink_window_attn_scaled(ll_cache *c, int layer, const ll_bf16 *q_roped, const float *q_row_scale,
+                               int64_t q_frame_start, int n_q_frames, ll_bf16 *out, float *lse_out, ll_stream stream)
+{
+    if (q_row_scale && !aligned16(q_row_scale)) return fail(LL_ERR_INVALID_ARG, "q_row_scale must be 16-byte aligned");
+    return attn_entry(c, layer, q_roped, q_frame_start, n_q_frames, out, lse_out, stream, false, q_row_scale);
+}
+
+size_t ll_qkv_proj_workspace_bytes(const ll_cache *c)
+{
+    if (!c) return 0;
+    const size_t tokens = (size_t)c->C * c->P, hd = (size_t)c->H * c->D;
+    // parked fp32 k rows, then the per-tile sums of squares of q and k
+    return align_up(tokens * hd * sizeof(float), 256) + align_up(2 * tokens * ((hd + 255) / 256) * sizeof(float), 256);
+}
+
+int ll_qkv_proj_append(ll_cache *c, int layer, const ll_bf16 *x, int d_model, const ll_bf16 *w_qkv, const float *bias,
+                       const float *gain_q, const float *gain_k, float eps, int64_t frame_start, int n_frames,
+                       int grid_h, int grid_w, float rope_theta, ll_bf16 *q_out, float *q_row_scale,
+                       void *workspace, size_t workspace_bytes, ll_stream stream)
+{
+    if (!layer_ok(c, layer)) return fail(LL_ERR_INVALID_ARG, "bad cache handle or layer %d", layer);
+    if (grid_h <= 0 || grid_w <= 0 || (int64_t)grid_h * grid_w != c->P)
+        return fail(LL_ERR_INVALID_ARG, "grid %dx%d does not give %d tokens per frame", grid_h, grid_w, c->P);
+    if (!(rope_theta > 0.f)) return fail(LL_ERR_INVALID_ARG, "rope_theta must be positive");
+    if (d_model < 64 || d_model % 8) return fail(LL_ERR_UNSUPPORTED_SHAPE, "d_model must be a multiple of 8, at least 64");
+    if ((c->H * c->D) % 256) return fail(LL_ERR_UNSUPPORTED_SHAPE, "heads * head_dim must be a multiple of 256");
+    if (c->kv_format != LL_KV_BF16) return fail(LL_ERR_UNSUPPORTED_SHAPE, "the fused projection is built for bf16 caches only");
+    const bool with_norm = gain_q || gain_k;
+    if (with_norm && (!gain_q || !gain_k || !(eps >= 0.f))) return fail(LL_ERR_INVALID_ARG, "both gains and eps >= 0 are needed for the norm");
+    if (n_frames != c->C) return fail(LL_ERR_BAD_POSITION, "n_frames %d != chunk_frames %d", n_frames, c->C);
+    ll::LayerState &st = c->layers[layer];
+    const bool is_new = frame_start == st.end;
+    const bool is_over = st.end >= c->C && frame_start == st.end - c->C;
+    if (!is_new && !is_over)
+        return fail(LL_ERR_BAD_POSITION, "frame_start %lld is neither end (%lld) nor end - chunk_frames",
+                    (long long)frame_start, (long long)st.end);
+    if (frame_start + n_frames > INT32_MAX) return fail(LL_ERR_BAD_POSITION, "frame index exceeds int32");
+    if (!c->dry_run) {
+        if (!x || !w_qkv || !q_out) return fail(LL_ERR_INVALID_ARG, "null x, w_qkv or q_out");
+        if (!aligned16(x) || !aligned16(w_qkv) || !aligned16(q_out) || !aligned16(bias) || !aligned16(gain_q) ||
+            !aligned16(gain_k) || !aligned16(q_row_scale) || (reinterpret_cast<uintptr_t>(workspace) & 255u))
+            return fail(LL_ERR_INVALID_ARG, "pointers must be 16-byte aligned (workspace: 256)");
+        if (with_norm && (!q_row_scale || !workspace || workspace_bytes < ll_qkv_proj_workspace_bytes(c)))
+            return fail(LL_ERR_INVALID_ARG, "the norm needs q_row_scale and a workspace of ll_qkv_proj_workspace_bytes");
+        int s = need_storage(c);
+        if (s != LL_OK) return s;
+        s = ensure_tables(c, frame_start, frame_start + n_frames, grid_h, grid_w, rope_theta, (cudaStream_t)stream);
+        if (s != LL_OK) return s;
+        ll::RopeAppendParams rp;
+        fill_rope_params(c, layer, nullptr, nullptr, nullptr, nullptr, frame_start, n_frames, grid_w, &rp);
+        ll::QkvParams p;
+        memset(&p, 0, sizeof p);
+        p.n_tokens = n_frames * c->P; p.d_model = d_model; p.heads = c->H; p.head_dim = c->D;
+        p.m_tiles = (p.n_tokens + 127) / 128; p.n_tiles = 3 * c->H * c->D / 256;
+        p.P = c->P; p.grid_w = grid_w; p.n_t = rp.n_t; p.n_h = rp.n_h;
+        p.with_norm = with_norm ? 1 : 0; p.eps = eps;
+        p.bias = bias; p.gain_q = gain_q; p.gain_k = gain_k;
+        p.t_tab = rp.t_tab; p.h_tab = rp.h_tab; p.w_tab = rp.w_tab;
+        p.q_out = q_out; p.q_row_scale = q_row_scale;
+        p.kcache = static_cast<ll_bf16 *>(rp.kcache); p.vcache = static_cast<ll_bf16 *>(rp.vcache);
+        p.rows_per_head = c->rows;
+        p.k_park = static_cast<float *>(workspace);
+        p.ssq = reinterpret_cast<float *>(static_cast<char *>(workspace) +
+                                          align_up((size_t)p.n_tokens * c->H * c->D * sizeof(float), 256));
+        p.status = reinterpret_cast<uint32_t *>(c->storage + c->off_status);
+        for (int i = 0; i < n_frames; ++i) p.slot[i] = rp.slot[i];
+        CUtensorMap xmap, wmap;
+        s = encode_map(&xmap, x, (uint64_t)d_model, (uint64_t)p.n_tokens, 1, (uint64_t)d_model * 2,
+                       (uint64_t)p.n_tokens * d_model * 2, 128, 1);
+        if (s != LL_OK) return s;
+        s = encode_map(&wmap, w_qkv, (uint64_t)d_model, (uint64_t)3 * c->H * c->D, 1, (uint64_t)d_model * 2,
+                       (uint64_t)3 * c->H * c->D * d_model * 2, 256, 1);
+        if (s != LL_OK) return s;
+        cudaError_t e = ll::launch_qkv_gemm(p, xmap, wmap, c->sm_count > 0 ? c->sm_count : 148, (cudaStream_t)stream);
+        if (e != cudaSuccess) return cuda_fail(e, "qkv projection kernel");
+    }
+    if (is_new) {
+        for (int i = 0; i < n_frames; ++i) {
+            int64_t f = frame_start + i;
+            int sl = slot_of(c, f);
+            if (st.slot_frame[sl] >= 0 && st.slot_frame[sl] != (int32_t)f) st.n_evictions += 1;
+            st.slot_frame[sl] = (int32_t)f;
+        }
+        st.end += n_frames;
+        st.n_appends += 1;
+    } else {
+        st.n_overwrites += 1;
+    }
+    return LL_OK;
 }
 
 int ll_sink_window_attn_batched(const ll_attn_item *items, int n_items, ll_stream stream)

@@ -73,6 +73,7 @@ struct AttnItem {
     float *lse;                       // [H, nq_total] or null
     const float *k_scale;             // [H] per-head factor on the keys (8-bit caches), or null
     const float *v_scale;             // [H] per-head factor on the values, or null
+    const float *q_scale;             // [nq_total] per-row factor on the queries, or null
     int nq_total;                     // rows of this item's q / out
     int pad;
 };
@@ -121,6 +122,28 @@ struct RopeAppendParams {
     int n_t, n_h;                     // pairs of the t and h bands (w band takes the rest)
     int slot[LL_MAX_SLOTS];           // storage slot of the call's i-th frame
 };
+
+// QKV projection with norm, rotation and append in its epilogue (qkv_gemm.cu).
+struct QkvParams {
+    int n_tokens, d_model, heads, head_dim;
+    int m_tiles, n_tiles;             // tiles of 128 tokens x 256 output features
+    int P, grid_w, n_t, n_h;
+    int with_norm;
+    float eps;
+    const float *bias;                // [3*H*D] or null
+    const float *gain_q, *gain_k;     // [H*D] (with_norm)
+    const float2 *t_tab, *h_tab, *w_tab;   // as in RopeAppendParams
+    ll_bf16 *q_out;                   // [n_tokens, H, D]: rotated q (without the norm's row factor)
+    float *q_row_scale;               // [n_tokens] (with_norm): the norm's factor of every q row
+    ll_bf16 *kcache, *vcache;         // layer base, [H][rows][D]
+    int64_t rows_per_head;
+    float *k_park;                    // [n_tokens, H*D] fp32 (with_norm): rotated k without its row factor
+    float *ssq;                       // [2][n_tokens][H*D/256] (with_norm): sums of squares per tile, q then k
+    uint32_t *status;
+    int slot[LL_MAX_SLOTS];
+};
+cudaError_t launch_qkv_gemm(const QkvParams &p, const CUtensorMap &xmap, const CUtensorMap &wmap, int sm_count,
+                            cudaStream_t stream);
 
 // kernel launchers (each returns the cudaError of the launch)
 cudaError_t launch_rope_tables(float2 *t_tab, int64_t t_base, int n_t_frames, int n_t,

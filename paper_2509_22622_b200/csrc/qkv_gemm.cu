@@ -1,0 +1,287 @@
+// QKV projection with the path's front end in its epilogue (sm_100a):
+//
+//   y = x W^T + b          x [n_tokens, d_model] bf16, W [3*H*D, d_model] bf16, fp32 accumulation
+//   q | k | v = y          (the rows of W are the q features, then k, then v)
+//   q, k: optional RMS norm over the token's whole row of H*D elements with a learned gain,
+//         then the 3-D rotation;  rotated q -> q_out, rotated k and raw v -> the cache rows.
+//
+// The GEMM is a persistent tcgen05 kernel: CTA tile 128 tokens x 256 output features (two
+// heads of 128, or four of 64), K blocks of 64 through a 4-stage TMA ring, accumulators
+// double-buffered in TMEM (2 x 256 columns) so that the epilogue of a tile runs under the
+// main loop of the next.  Warp 0 (one lane): TMA producer.  Warp 1 (one elected lane): MMA
+// issuer.  Warps 4-7: epilogue, one thread per token row (the 32x32b TMEM shape).
+//
+// The norm needs the sum of squares of a token's whole q (or k) row, which is spread over
+// H*D/256 tiles that run on different SMs at different times.  The factor is one scalar per
+// token and everything after it is linear, so a tile stores rotate(gain * y) without it and
+// leaves its part of the sum of squares in a table (one slot per token and tile: no atomics,
+// the sum is taken in a fixed order).  For q the scalar then travels with q_out to the
+// attention call as a per-row softmax scale; for k a small second kernel applies it: the
+// epilogue parks the un-normalised rotated k rows in fp32 in the caller's workspace and the
+// second kernel scales, rounds once to bf16 and writes the cache rows.
+#include <cuda_bf16.h>
+
+#include "bounded_wait.cuh"
+#include "ll_internal.h"
+#include "ptx.cuh"
+
+namespace ll {
+
+namespace {
+
+using namespace ptx;
+
+constexpr int kGemmThreads = 256;
+constexpr int kTileM = 128, kTileN = 256, kBlockK = 64;
+constexpr int kGemmStages = 4;
+constexpr int kABytes = kTileM * kBlockK * 2;          // 16 KB
+constexpr int kBBytes = kTileN * kBlockK * 2;          // 32 KB
+constexpr int kStageBytes = kABytes + kBBytes;
+constexpr int kGemmSmem = kGemmStages * kStageBytes + 1024 /*barriers*/ + 1024 /*alignment*/;
+
+enum GBar { kFull = 0, kEmpty = kGemmStages, kAccFull = 2 * kGemmStages, kAccEmpty = 2 * kGemmStages + 2, kGemmBars = 2 * kGemmStages + 4 };
+
+__device__ __forceinline__ void tmem_ld_32x32b_x32(uint32_t taddr, uint32_t *r)
+{
+    asm volatile("tcgen05.ld.sync.aligned.32x32b.x32.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+                 : "r"(taddr)
+                 : "memory");
+}
+
+// One token row of a 128 x 256 accumulator tile: bias, sum of squares, gain, rotation, stores.
+__device__ __forceinline__ void epilogue_tile(const QkvParams &p, uint32_t taddr, int token, int n0)
+{
+    const int HD = p.heads * p.head_dim;
+    const int which = n0 / HD;                         // 0 q, 1 k, 2 v (a tile never straddles them)
+    const int cw0 = n0 - which * HD;                   // the tile's first feature inside q, k or v
+    const bool live = token < p.n_tokens;
+    const int tok = live ? token : 0;
+    const int frame = tok / p.P, cell = tok % p.P;
+    const int y = cell / p.grid_w, x = cell % p.grid_w;
+    const size_t cache_row = (size_t)p.slot[frame] * p.P + cell;
+    const bool park = which == 1 && p.with_norm;       // k under the norm: fp32, finished by the second kernel
+    const float *gain = which == 0 ? p.gain_q : p.gain_k;
+    float ssq = 0.f;
+#pragma unroll 1
+    for (int ch = 0; ch < kTileN / 32; ++ch) {
+        uint32_t r[32];
+        tmem_ld_32x32b_x32(taddr + 32 * ch, r);
+        tmem_wait_ld();
+        const int cw = cw0 + 32 * ch;                  // first feature of this 32-wide piece
+        const int head = cw / p.head_dim, d0 = cw % p.head_dim;
+        float v[32];
+#pragma unroll
+        for (int i = 0; i < 32; ++i) {
+            v[i] = __uint_as_float(r[i]);
+            if (p.bias) v[i] += __ldg(p.bias + n0 + 32 * ch + i);
+        }
+        if (which < 2) {
+#pragma unroll
+            for (int i = 0; i < 32; ++i) ssq = fmaf(v[i], v[i], ssq);
+            if (p.with_norm) {
+#pragma unroll
+                for (int i = 0; i < 32; ++i) v[i] *= __ldg(gain + cw + i);
+            }
+#pragma unroll
+            for (int i = 0; i < 16; ++i) {
+                const int j = d0 / 2 + i;              // rotation pair inside the head row
+                const float2 *src;
+                if (j < p.n_t)             src = p.t_tab + (size_t)frame * p.n_t + j;
+                else if (j < p.n_t + p.n_h) src = p.h_tab + (size_t)y * p.n_h + (j - p.n_t);
+                else                        src = p.w_tab + (size_t)x * p.n_h + (j - p.n_t - p.n_h);
+                const float2 cs = __ldg(src);
+                const float a = v[2 * i], b = v[2 * i + 1];
+                v[2 * i] = fmaf(a, cs.x, -(b * cs.y));
+                v[2 * i + 1] = fmaf(a, cs.y, b * cs.x);
+            }
+        }
+        if (!live) continue;
+        if (park) {
+            float4 *dst = reinterpret_cast<float4 *>(p.k_park + (size_t)token * HD + cw);
+#pragma unroll
+            for (int i = 0; i < 8; ++i) dst[i] = make_float4(v[4 * i], v[4 * i + 1], v[4 * i + 2], v[4 * i + 3]);
+        } else {
+            ll_bf16 *dst;
+            if (which == 0) dst = p.q_out + ((size_t)token * p.heads + head) * p.head_dim + d0;
+            else            dst = (which == 1 ? p.kcache : p.vcache) + ((size_t)head * p.rows_per_head + cache_row) * p.head_dim + d0;
+            uint32_t o[16];
+#pragma unroll
+            for (int i = 0; i < 16; ++i) o[i] = cvt_bf16x2(v[2 * i], v[2 * i + 1]);
+#pragma unroll
+            for (int i = 0; i < 4; ++i)
+                reinterpret_cast<uint4 *>(dst)[i] = make_uint4(o[4 * i], o[4 * i + 1], o[4 * i + 2], o[4 * i + 3]);
+        }
+    }
+    if (live && p.with_norm && which < 2)
+        p.ssq[((size_t)which * p.n_tokens + token) * (HD / kTileN) + cw0 / kTileN] = ssq;
+}
+
+__global__ void __launch_bounds__(kGemmThreads, 1)
+qkv_gemm_kernel(const __grid_constant__ QkvParams p, const __grid_constant__ CUtensorMap xmap,
+                const __grid_constant__ CUtensorMap wmap)
+{
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    uint8_t *smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));
+    const uint32_t bars = smem_base + kGemmStages * kStageBytes;
+    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(smem_gen + kGemmStages * kStageBytes + kGemmBars * 8);
+    volatile int *abort_flag = reinterpret_cast<volatile int *>(tmem_slot + 1);
+    auto bar = [&](int i) -> uint32_t { return bars + 8u * (uint32_t)i; };
+    const int warp = __shfl_sync(0xffffffffu, (int)(threadIdx.x >> 5), 0);
+    const int lane = threadIdx.x & 31;
+
+    if (threadIdx.x == 0) {
+        for (int i = 0; i < kGemmBars; ++i) mbar_init(bar(i), (i >= kAccEmpty) ? 4u : 1u);   // four epilogue warps free a buffer
+        *abort_flag = (*reinterpret_cast<volatile uint32_t *>(p.status) != kStatusOk) ? 2 : 0;
+        fence_mbar_init();
+    }
+    if (warp == 0) {
+        tmem_alloc(smem_u32(tmem_slot), 512);
+        tmem_relinquish();
+    }
+    tc_fence_before_sync();
+    __syncthreads();
+    tc_fence_after_sync();
+    const uint32_t tmem = *tmem_slot;
+    WaitCtx ctx{abort_flag, p.status, warp};
+    const bool skip = *abort_flag != 0;
+    auto wait = [&](int bar_id, uint32_t parity, int iter) -> bool {
+        return wait_bar(bar(bar_id), parity & 1u, ctx, bar_id, iter);
+    };
+    const int n_kb = (p.d_model + kBlockK - 1) / kBlockK;
+    const int n_tiles = p.m_tiles * p.n_tiles;
+
+    if (skip) {
+        // an earlier kernel gave up on a wait: nothing to do
+    } else if (warp == 0 && lane == 0) {
+        // ---- TMA producer: tiles in the order all roles walk them; n runs fastest so that the
+        // CTAs of a wave share x rows and stream the weights (which stay in L2 anyway) ----
+        prefetch_tensormap(&xmap);
+        prefetch_tensormap(&wmap);
+        uint32_t n = 0;
+        for (int tile = blockIdx.x; tile < n_tiles; tile += gridDim.x) {
+            const int m0 = (tile / p.n_tiles) * kTileM, n0 = (tile % p.n_tiles) * kTileN;
+            for (int kb = 0; kb < n_kb; ++kb, ++n) {
+                const int stage = n % kGemmStages;
+                if (!wait(kEmpty + stage, (n / kGemmStages) ^ 1u, (int)n)) goto done;
+                mbar_arrive_expect_tx(bar(kFull + stage), kStageBytes);
+                const uint32_t a = smem_base + stage * kStageBytes;
+                tma_load_3d(a, &xmap, bar(kFull + stage), kb * kBlockK, m0, 0);
+                tma_load_3d(a + kABytes, &wmap, bar(kFull + stage), kb * kBlockK, n0, 0);
+            }
+        }
+    } else if (warp == 1) {
+        // ---- MMA issuer ----
+        const bool elected = elect_one();
+        constexpr uint32_t idesc = idesc_bf16_f32(kTileM, kTileN, 0, 0);
+        constexpr uint32_t hi = smem_desc_hi_sw128(1024);
+        uint32_t n = 0, t = 0;
+        for (int tile = blockIdx.x; tile < n_tiles; tile += gridDim.x, ++t) {
+            const uint32_t buf = t & 1u;
+            // the epilogue has read this accumulator buffer out (two tiles ago)
+            if (t >= 2 && !wait(kAccEmpty + buf, (t >> 1) - 1, (int)t)) goto done;
+            tc_fence_after_sync();
+            for (int kb = 0; kb < n_kb; ++kb, ++n) {
+                const int stage = n % kGemmStages;
+                if (!wait(kFull + stage, n / kGemmStages, (int)n)) goto done;
+                tc_fence_after_sync();
+                if (elected) {
+                    const uint32_t a_lo = smem_desc_lo(smem_base + stage * kStageBytes, 16);
+                    const uint32_t b_lo = smem_desc_lo(smem_base + stage * kStageBytes + kABytes, 16);
+#pragma unroll
+                    for (int kk = 0; kk < kBlockK / 16; ++kk)
+                        mma_ss(tmem + buf * kTileN, smem_desc_join(a_lo + ((kk * 32) >> 4), hi),
+                               smem_desc_join(b_lo + ((kk * 32) >> 4), hi), idesc, (kb > 0 || kk > 0) ? 1u : 0u);
+                    tc_commit(bar(kEmpty + stage));
+                    if (kb == n_kb - 1) tc_commit(bar(kAccFull + buf));
+                }
+                __syncwarp();
+            }
+        }
+    } else if (warp >= 4) {
+        // ---- epilogue: thread = one token row of the tile ----
+        const int q4 = warp & 3;
+        uint32_t t = 0;
+        for (int tile = blockIdx.x; tile < n_tiles; tile += gridDim.x, ++t) {
+            const uint32_t buf = t & 1u;
+            const int m0 = (tile / p.n_tiles) * kTileM, n0 = (tile % p.n_tiles) * kTileN;
+            if (!__all_sync(0xffffffffu, wait(kAccFull + buf, t >> 1, (int)t))) goto done;
+            tc_fence_after_sync();
+            epilogue_tile(p, tmem + buf * kTileN + ((uint32_t)(32 * q4) << 16), m0 + 32 * q4 + lane, n0);
+            tc_fence_before_sync();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar(kAccEmpty + buf));
+        }
+    }
+done:
+    tc_fence_before_sync();
+    __syncthreads();
+    if (*abort_flag == 1) {
+        const uint64_t t0 = globaltimer_ns();
+        while (globaltimer_ns() - t0 < 200000ull) __nanosleep(1000);
+        __syncthreads();
+    }
+    if (warp == 0) {
+        __syncwarp();
+        tc_fence_after_sync();
+        tmem_dealloc(tmem, 512);
+    }
+}
+
+// The norm's second step: every token's row factors from the per-tile sums of squares (summed
+// in tile order), q's to q_row_scale, k's applied to the parked fp32 rows, which are rounded
+// once to bf16 into the cache rows.  One thread per 8 features of a token's k row.
+__global__ void __launch_bounds__(256)
+qkv_finish_kernel(const __grid_constant__ QkvParams p)
+{
+    const int HD = p.heads * p.head_dim;
+    const int vecs = HD / 8, tiles = HD / kTileN;
+    const long long gid = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    const int vec = (int)(gid % vecs);
+    const long long token = gid / vecs;
+    if (token >= p.n_tokens) return;
+    float sq = 0.f, sk = 0.f;
+    for (int t = 0; t < tiles; ++t) {
+        sq += p.ssq[(size_t)token * tiles + t];
+        sk += p.ssq[((size_t)p.n_tokens + token) * tiles + t];
+    }
+    const float inv_n = 1.f / (float)HD;
+    const float rq = 1.f / sqrtf(fmaf(sq, inv_n, p.eps)), rk = 1.f / sqrtf(fmaf(sk, inv_n, p.eps));
+    if (vec == 0) p.q_row_scale[token] = rq;
+    const int f0 = vec * 8, head = f0 / p.head_dim, d0 = f0 % p.head_dim;
+    const int frame = (int)(token / p.P), cell = (int)(token % p.P);
+    const size_t cache_row = (size_t)p.slot[frame] * p.P + cell;
+    const float4 *src = reinterpret_cast<const float4 *>(p.k_park + (size_t)token * HD + f0);
+    const float4 a = src[0], b = src[1];
+    *reinterpret_cast<uint4 *>(p.kcache + ((size_t)head * p.rows_per_head + cache_row) * p.head_dim + d0) =
+        make_uint4(cvt_bf16x2(a.x * rk, a.y * rk), cvt_bf16x2(a.z * rk, a.w * rk), cvt_bf16x2(b.x * rk, b.y * rk),
+                   cvt_bf16x2(b.z * rk, b.w * rk));
+}
+
+}  // namespace
+
+cudaError_t launch_qkv_gemm(const QkvParams &p, const CUtensorMap &xmap, const CUtensorMap &wmap, int sm_count,
+                            cudaStream_t stream)
+{
+    static bool prepared = false;                      // the attribute is per function, not per device state we track
+    cudaError_t e;
+    if (!prepared) {
+        e = cudaFuncSetAttribute(qkv_gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kGemmSmem);
+        if (e != cudaSuccess) return e;
+        prepared = true;
+    }
+    const int n_tiles = p.m_tiles * p.n_tiles;
+    if (n_tiles <= 0) return cudaSuccess;
+    const int grid = n_tiles < sm_count ? n_tiles : sm_count;
+    qkv_gemm_kernel<<<grid, kGemmThreads, kGemmSmem, stream>>>(p, xmap, wmap);
+    count_launch();
+    e = cudaGetLastError();
+    if (e != cudaSuccess || !p.with_norm) return e;
+    const long long threads = (long long)p.n_tokens * (p.heads * p.head_dim / 8);
+    qkv_finish_kernel<<<(unsigned)((threads + 255) / 256), 256, 0, stream>>>(p);
+    count_launch();
+    return cudaGetLastError();
+}
+
+}  // namespace ll

@@ -751,3 +751,23 @@ def test_e4m3_storage_scales_by_powers_of_two_and_saturates(oracle_mod):
     big = np.full((1, H, D), 7.0)
     orc.append(0, big * 0.0, -big, 0, 1, 1)
     assert np.array_equal(orc.read_layer(0)[1][0], np.full((1, H, D), -448.0 * float(np.float32(0.001))))
+
+
+# ---------------------------------------------------------------------------
+# QKV projection (the step in front of the path)
+# ---------------------------------------------------------------------------
+
+def test_qkv_projection_equals_the_written_out_sum_and_splits_q_k_v(oracle_mod):
+    rng = np.random.default_rng(3)
+    T, dm, n = 5, 7, 4
+    x, w, b = rng.standard_normal((T, dm)), rng.standard_normal((3 * n, dm)), rng.standard_normal(3 * n)
+    q, k, v = oracle_mod.qkv_proj(x, w, b)
+    for t in range(T):
+        for j in range(3 * n):
+            want = b[j] + sum(x[t, i] * w[j, i] for i in range(dm))
+            got = (q, k, v)[j // n][t, j % n]
+            assert abs(got - want) < 1e-12
+    # identity blocks: q = x, k = 2x, v = -x (catches a transposed weight or a wrong split)
+    eye = np.eye(dm)
+    q, k, v = oracle_mod.qkv_proj(x, np.concatenate([eye, 2 * eye, -eye]))
+    assert np.array_equal(q, x) and np.array_equal(k, 2 * x) and np.array_equal(v, -x)

@@ -399,6 +399,21 @@ int build_attn_params(const AttnCall *calls, int n_calls, ll::AttnParams *p)
     return LL_OK;
 }
 
+// Map of a token-major [tokens, H, D] tensor of the caller (box: 64 elements x 1 head x 128 tokens),
+// from the handle's small cache when this address and length were seen before.
+int token_major_map(ll_cache *c, CUtensorMap *out, const void *base, uint64_t tokens)
+{
+    for (const auto &e : c->map_cache)
+        if (e.base == base && e.d2 == tokens) { *out = e.map; return LL_OK; }
+    int st = encode_map(out, base, (uint64_t)c->D, (uint64_t)c->H, tokens, (uint64_t)c->D * 2, (uint64_t)c->H * c->D * 2, 1, 128);
+    if (st != LL_OK) return st;
+    constexpr size_t kEntries = 16;
+    ll_cache::CachedMap e{base, tokens, 1, 128, *out};
+    if (c->map_cache.size() < kEntries) c->map_cache.push_back(e);
+    else c->map_cache[c->map_cache_next++ % kEntries] = e;
+    return LL_OK;
+}
+
 int launch_attention(const AttnCall *calls, int n_calls, const ll::AttnParams &p, cudaStream_t stream, bool simt)
 {
     ll_cache *c0 = calls[0].c;
@@ -410,16 +425,13 @@ int launch_attention(const AttnCall *calls, int n_calls, const ll::AttnParams &p
     memset(&maps, 0, sizeof maps);
     for (int i = 0; i < n_calls; ++i) {
         ll_cache *c = calls[i].c;
-        int st = encode_map(&maps.q[i], calls[i].q, (uint64_t)c->D, (uint64_t)c->H, (uint64_t)p.item[i].nq_total,
-                            (uint64_t)c->D * 2, (uint64_t)c->H * c->D * 2, 1, 128);
+        int st = token_major_map(c, &maps.q[i], calls[i].q, (uint64_t)p.item[i].nq_total);
         if (st != LL_OK) return st;
         if (calls[i].dense_keys > 0) {
             // token-major K/V: coordinates (dim, head, token), a tile = 128 tokens of one head
-            st = encode_map(&maps.k[i], calls[i].dense_k, (uint64_t)c->D, (uint64_t)c->H, (uint64_t)calls[i].dense_keys,
-                            (uint64_t)c->D * 2, (uint64_t)c->H * c->D * 2, 1, 128);
+            st = token_major_map(c, &maps.k[i], calls[i].dense_k, (uint64_t)calls[i].dense_keys);
             if (st != LL_OK) return st;
-            st = encode_map(&maps.v[i], calls[i].dense_v, (uint64_t)c->D, (uint64_t)c->H, (uint64_t)calls[i].dense_keys,
-                            (uint64_t)c->D * 2, (uint64_t)c->H * c->D * 2, 1, 128);
+            st = token_major_map(c, &maps.v[i], calls[i].dense_v, (uint64_t)calls[i].dense_keys);
             if (st != LL_OK) return st;
             continue;
         }
@@ -731,7 +743,7 @@ size_t ll_qkv_proj_workspace_bytes(const ll_cache *c)
     if (!c) return 0;
     const size_t tokens = (size_t)c->C * c->P, hd = (size_t)c->H * c->D;
     // parked fp32 k rows, then the per-tile sums of squares of q and k
-    return align_up(tokens * hd * sizeof(float), 256) + align_up(2 * tokens * ((hd + 255) / 256) * sizeof(float), 256);
+    return align_up(tokens * hd * sizeof(float), 256) + align_up(2 * tokens * ((hd + 127) / 128) * sizeof(float), 256);
 }
 
 int ll_qkv_proj_append(ll_cache *c, int layer, const ll_bf16 *x, int d_model, const ll_bf16 *w_qkv, const float *bias,
@@ -744,7 +756,8 @@ int ll_qkv_proj_append(ll_cache *c, int layer, const ll_bf16 *x, int d_model, co
         return fail(LL_ERR_INVALID_ARG, "grid %dx%d does not give %d tokens per frame", grid_h, grid_w, c->P);
     if (!(rope_theta > 0.f)) return fail(LL_ERR_INVALID_ARG, "rope_theta must be positive");
     if (d_model < 64 || d_model % 8) return fail(LL_ERR_UNSUPPORTED_SHAPE, "d_model must be a multiple of 8, at least 64");
-    if ((c->H * c->D) % 256) return fail(LL_ERR_UNSUPPORTED_SHAPE, "heads * head_dim must be a multiple of 256");
+    if ((c->H * c->D) % 256 || c->H * c->D > 8192)
+        return fail(LL_ERR_UNSUPPORTED_SHAPE, "heads * head_dim must be a multiple of 256, at most 8192");
     if (c->kv_format != LL_KV_BF16) return fail(LL_ERR_UNSUPPORTED_SHAPE, "the fused projection is built for bf16 caches only");
     const bool with_norm = gain_q || gain_k;
     if (with_norm && (!gain_q || !gain_k || !(eps >= 0.f))) return fail(LL_ERR_INVALID_ARG, "both gains and eps >= 0 are needed for the norm");

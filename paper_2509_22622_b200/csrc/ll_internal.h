@@ -138,7 +138,7 @@ struct QkvParams {
     ll_bf16 *kcache, *vcache;         // layer base, [H][rows][D]
     int64_t rows_per_head;
     float *k_park;                    // [n_tokens, H*D] fp32 (with_norm): rotated k without its row factor
-    float *ssq;                       // [2][n_tokens][H*D/256] (with_norm): sums of squares per tile, q then k
+    float *ssq;                       // [2][n_tokens][H*D/128] (with_norm): sums of squares per 128 features, q then k
     uint32_t *status;
     int slot[LL_MAX_SLOTS];
 };
@@ -196,6 +196,12 @@ struct ll_cache {
     size_t off_scales = 0, off_stage = 0;
     CUtensorMap stage_kmap, stage_vmap;
     std::vector<float> scales;        // host copy, [L][2][H]
+
+    // Tensor maps of caller tensors met recently (q of the attention calls, k/v of the dense ones):
+    // a map depends on address and shape only, and encoding one costs more than a microsecond.
+    struct CachedMap { const void *base; uint64_t d2; uint32_t box1, box2; CUtensorMap map; };
+    std::vector<CachedMap> map_cache;
+    size_t map_cache_next = 0;
 
     // which RoPE tables are resident
     bool hw_valid = false;

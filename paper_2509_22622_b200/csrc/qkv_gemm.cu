@@ -14,7 +14,7 @@
 // The norm needs the sum of squares of a token's whole q (or k) row, which is spread over
 // H*D/256 tiles that run on different SMs at different times.  The factor is one scalar per
 // token and everything after it is linear, so a tile stores rotate(gain * y) without it and
-// leaves its part of the sum of squares in a table (one slot per token and tile: no atomics,
+// leaves its part of the sum of squares in a table (one slot per token and 128 features: no atomics,
 // the sum is taken in a fixed order).  For q the scalar then travels with q_out to the
 // attention call as a per-row softmax scale; for k a small second kernel applies it: the
 // epilogue parks the un-normalised rotated k rows in fp32 in the caller's workspace and the
@@ -31,7 +31,7 @@ namespace {
 
 using namespace ptx;
 
-constexpr int kGemmThreads = 256;
+constexpr int kGemmThreads = 384;                      // TMA, MMA, two idle warps, eight epilogue warps
 constexpr int kTileM = 128, kTileN = 256, kBlockK = 64;
 constexpr int kGemmStages = 4;
 constexpr int kABytes = kTileM * kBlockK * 2;          // 16 KB
@@ -49,12 +49,17 @@ __device__ __forceinline__ void tmem_ld_32x32b_x32(uint32_t taddr, uint32_t *r)
                  : "memory");
 }
 
-// One token row of a 128 x 256 accumulator tile: bias, sum of squares, gain, rotation, stores.
-__device__ __forceinline__ void epilogue_tile(const QkvParams &p, uint32_t taddr, int token, int n0)
+// One token row of half a 128 x 256 accumulator tile (128 features: `half` 0 or 1): bias, sum
+// of squares, gain, rotation, stores.  D is a template parameter and the 32-feature pieces are
+// unrolled, so which band (t, h or w) a rotation pair belongs to is known at compile time and
+// the piece's (cos, sin) pairs come from three row pointers at fixed offsets.
+template <int D>
+__device__ __forceinline__ float epilogue_half(const QkvParams &p, uint32_t taddr, int token, int n0, int half)
 {
-    const int HD = p.heads * p.head_dim;
+    constexpr int kNh = D / 6, kNt = D / 2 - 2 * kNh;  // pairs of the h (= w) and t bands
+    const int HD = p.heads * D;
     const int which = n0 / HD;                         // 0 q, 1 k, 2 v (a tile never straddles them)
-    const int cw0 = n0 - which * HD;                   // the tile's first feature inside q, k or v
+    const int cw0 = n0 - which * HD + 128 * half;      // this half's first feature inside q, k or v
     const bool live = token < p.n_tokens;
     const int tok = live ? token : 0;
     const int frame = tok / p.P, cell = tok % p.P;
@@ -62,35 +67,42 @@ __device__ __forceinline__ void epilogue_tile(const QkvParams &p, uint32_t taddr
     const size_t cache_row = (size_t)p.slot[frame] * p.P + cell;
     const bool park = which == 1 && p.with_norm;       // k under the norm: fp32, finished by the second kernel
     const float *gain = which == 0 ? p.gain_q : p.gain_k;
+    const float2 *t_row = p.t_tab + (size_t)frame * kNt, *h_row = p.h_tab + (size_t)y * kNh, *w_row = p.w_tab + (size_t)x * kNh;
     float ssq = 0.f;
-#pragma unroll 1
-    for (int ch = 0; ch < kTileN / 32; ++ch) {
+#pragma unroll
+    for (int ch = 0; ch < 4; ++ch) {
         uint32_t r[32];
-        tmem_ld_32x32b_x32(taddr + 32 * ch, r);
+        tmem_ld_32x32b_x32(taddr + 128 * half + 32 * ch, r);
         tmem_wait_ld();
         const int cw = cw0 + 32 * ch;                  // first feature of this 32-wide piece
-        const int head = cw / p.head_dim, d0 = cw % p.head_dim;
+        const int head = cw / D;
+        const int d0 = (32 * ch) % D;                  // cw0 is a multiple of 128 and D divides 128
         float v[32];
 #pragma unroll
-        for (int i = 0; i < 32; ++i) {
-            v[i] = __uint_as_float(r[i]);
-            if (p.bias) v[i] += __ldg(p.bias + n0 + 32 * ch + i);
+        for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
+        if (p.bias) {
+            const float4 *bp = reinterpret_cast<const float4 *>(p.bias + n0 + 128 * half + 32 * ch);
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+                const float4 bb = __ldg(bp + i);
+                v[4 * i] += bb.x; v[4 * i + 1] += bb.y; v[4 * i + 2] += bb.z; v[4 * i + 3] += bb.w;
+            }
         }
         if (which < 2) {
 #pragma unroll
             for (int i = 0; i < 32; ++i) ssq = fmaf(v[i], v[i], ssq);
             if (p.with_norm) {
+                const float4 *gp = reinterpret_cast<const float4 *>(gain + cw);
 #pragma unroll
-                for (int i = 0; i < 32; ++i) v[i] *= __ldg(gain + cw + i);
+                for (int i = 0; i < 8; ++i) {
+                    const float4 gg = __ldg(gp + i);
+                    v[4 * i] *= gg.x; v[4 * i + 1] *= gg.y; v[4 * i + 2] *= gg.z; v[4 * i + 3] *= gg.w;
+                }
             }
 #pragma unroll
             for (int i = 0; i < 16; ++i) {
-                const int j = d0 / 2 + i;              // rotation pair inside the head row
-                const float2 *src;
-                if (j < p.n_t)             src = p.t_tab + (size_t)frame * p.n_t + j;
-                else if (j < p.n_t + p.n_h) src = p.h_tab + (size_t)y * p.n_h + (j - p.n_t);
-                else                        src = p.w_tab + (size_t)x * p.n_h + (j - p.n_t - p.n_h);
-                const float2 cs = __ldg(src);
+                const int j = d0 / 2 + i;              // rotation pair inside the head row (compile time)
+                const float2 cs = j < kNt ? __ldg(t_row + j) : j < kNt + kNh ? __ldg(h_row + (j - kNt)) : __ldg(w_row + (j - kNt - kNh));
                 const float a = v[2 * i], b = v[2 * i + 1];
                 v[2 * i] = fmaf(a, cs.x, -(b * cs.y));
                 v[2 * i + 1] = fmaf(a, cs.y, b * cs.x);
@@ -103,8 +115,8 @@ __device__ __forceinline__ void epilogue_tile(const QkvParams &p, uint32_t taddr
             for (int i = 0; i < 8; ++i) dst[i] = make_float4(v[4 * i], v[4 * i + 1], v[4 * i + 2], v[4 * i + 3]);
         } else {
             ll_bf16 *dst;
-            if (which == 0) dst = p.q_out + ((size_t)token * p.heads + head) * p.head_dim + d0;
-            else            dst = (which == 1 ? p.kcache : p.vcache) + ((size_t)head * p.rows_per_head + cache_row) * p.head_dim + d0;
+            if (which == 0) dst = p.q_out + ((size_t)token * p.heads + head) * D + d0;
+            else            dst = (which == 1 ? p.kcache : p.vcache) + ((size_t)head * p.rows_per_head + cache_row) * D + d0;
             uint32_t o[16];
 #pragma unroll
             for (int i = 0; i < 16; ++i) o[i] = cvt_bf16x2(v[2 * i], v[2 * i + 1]);
@@ -113,10 +125,10 @@ __device__ __forceinline__ void epilogue_tile(const QkvParams &p, uint32_t taddr
                 reinterpret_cast<uint4 *>(dst)[i] = make_uint4(o[4 * i], o[4 * i + 1], o[4 * i + 2], o[4 * i + 3]);
         }
     }
-    if (live && p.with_norm && which < 2)
-        p.ssq[((size_t)which * p.n_tokens + token) * (HD / kTileN) + cw0 / kTileN] = ssq;
+    return ssq;
 }
 
+template <int D>
 __global__ void __launch_bounds__(kGemmThreads, 1)
 qkv_gemm_kernel(const __grid_constant__ QkvParams p, const __grid_constant__ CUtensorMap xmap,
                 const __grid_constant__ CUtensorMap wmap)
@@ -132,7 +144,7 @@ qkv_gemm_kernel(const __grid_constant__ QkvParams p, const __grid_constant__ CUt
     const int lane = threadIdx.x & 31;
 
     if (threadIdx.x == 0) {
-        for (int i = 0; i < kGemmBars; ++i) mbar_init(bar(i), (i >= kAccEmpty) ? 4u : 1u);   // four epilogue warps free a buffer
+        for (int i = 0; i < kGemmBars; ++i) mbar_init(bar(i), (i >= kAccEmpty) ? 8u : 1u);   // eight epilogue warps free a buffer
         *abort_flag = (*reinterpret_cast<volatile uint32_t *>(p.status) != kStatusOk) ? 2 : 0;
         fence_mbar_init();
     }
@@ -200,18 +212,25 @@ qkv_gemm_kernel(const __grid_constant__ QkvParams p, const __grid_constant__ CUt
             }
         }
     } else if (warp >= 4) {
-        // ---- epilogue: thread = one token row of the tile ----
-        const int q4 = warp & 3;
+        // ---- epilogue: thread = one token row of one half (128 features) of the tile ----
+        const int q4 = warp & 3, half = (warp - 4) >> 2;
         uint32_t t = 0;
         for (int tile = blockIdx.x; tile < n_tiles; tile += gridDim.x, ++t) {
             const uint32_t buf = t & 1u;
             const int m0 = (tile / p.n_tiles) * kTileM, n0 = (tile % p.n_tiles) * kTileN;
             if (!__all_sync(0xffffffffu, wait(kAccFull + buf, t >> 1, (int)t))) goto done;
             tc_fence_after_sync();
-            epilogue_tile(p, tmem + buf * kTileN + ((uint32_t)(32 * q4) << 16), m0 + 32 * q4 + lane, n0);
+            const int token = m0 + 32 * q4 + lane;
+            const float ssq = epilogue_half<D>(p, tmem + buf * kTileN + ((uint32_t)(32 * q4) << 16), token, n0, half);
             tc_fence_before_sync();
             __syncwarp();
             if (lane == 0) mbar_arrive(bar(kAccEmpty + buf));
+            // the half's part of the row's sum of squares: one slot per token and 128 features
+            const int HD = p.heads * D;
+            if (p.with_norm && n0 < 2 * HD && token < p.n_tokens) {
+                const int which = n0 / HD;
+                p.ssq[((size_t)which * p.n_tokens + token) * (HD / 128) + (n0 - which * HD) / 128 + half] = ssq;
+            }
         }
     }
 done:
@@ -229,28 +248,27 @@ done:
     }
 }
 
-// The norm's second step: every token's row factors from the per-tile sums of squares (summed
-// in tile order), q's to q_row_scale, k's applied to the parked fp32 rows, which are rounded
-// once to bf16 into the cache rows.  One thread per 8 features of a token's k row.
-__global__ void __launch_bounds__(256)
+// The norm's second step, one thread block per token: the row factors from the sums of squares
+// per 128 features (added in feature order), q's to q_row_scale, k's applied to the parked fp32
+// row, which is rounded once to bf16 into the cache row.  One thread per 8 features.
+__global__ void __launch_bounds__(1024)
 qkv_finish_kernel(const __grid_constant__ QkvParams p)
 {
+    __shared__ float r_sh[2];
     const int HD = p.heads * p.head_dim;
-    const int vecs = HD / 8, tiles = HD / kTileN;
-    const long long gid = (long long)blockIdx.x * blockDim.x + threadIdx.x;
-    const int vec = (int)(gid % vecs);
-    const long long token = gid / vecs;
-    if (token >= p.n_tokens) return;
-    float sq = 0.f, sk = 0.f;
-    for (int t = 0; t < tiles; ++t) {
-        sq += p.ssq[(size_t)token * tiles + t];
-        sk += p.ssq[((size_t)p.n_tokens + token) * tiles + t];
+    const int tiles = HD / 128;
+    const int token = blockIdx.x;
+    if (threadIdx.x < 2) {
+        const float *src = p.ssq + ((size_t)threadIdx.x * p.n_tokens + token) * tiles;
+        float sum = 0.f;
+        for (int t = 0; t < tiles; ++t) sum += src[t];
+        r_sh[threadIdx.x] = 1.f / sqrtf(fmaf(sum, 1.f / (float)HD, p.eps));
     }
-    const float inv_n = 1.f / (float)HD;
-    const float rq = 1.f / sqrtf(fmaf(sq, inv_n, p.eps)), rk = 1.f / sqrtf(fmaf(sk, inv_n, p.eps));
-    if (vec == 0) p.q_row_scale[token] = rq;
-    const int f0 = vec * 8, head = f0 / p.head_dim, d0 = f0 % p.head_dim;
-    const int frame = (int)(token / p.P), cell = (int)(token % p.P);
+    __syncthreads();
+    const float rk = r_sh[1];
+    if (threadIdx.x == 0) p.q_row_scale[token] = r_sh[0];
+    const int f0 = threadIdx.x * 8, head = f0 / p.head_dim, d0 = f0 % p.head_dim;
+    const int frame = token / p.P, cell = token % p.P;
     const size_t cache_row = (size_t)p.slot[frame] * p.P + cell;
     const float4 *src = reinterpret_cast<const float4 *>(p.k_park + (size_t)token * HD + f0);
     const float4 a = src[0], b = src[1];
@@ -264,22 +282,19 @@ qkv_finish_kernel(const __grid_constant__ QkvParams p)
 cudaError_t launch_qkv_gemm(const QkvParams &p, const CUtensorMap &xmap, const CUtensorMap &wmap, int sm_count,
                             cudaStream_t stream)
 {
-    static bool prepared = false;                      // the attribute is per function, not per device state we track
-    cudaError_t e;
-    if (!prepared) {
-        e = cudaFuncSetAttribute(qkv_gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kGemmSmem);
-        if (e != cudaSuccess) return e;
-        prepared = true;
-    }
+    cudaError_t e = p.head_dim == 128
+        ? cudaFuncSetAttribute(qkv_gemm_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, kGemmSmem)
+        : cudaFuncSetAttribute(qkv_gemm_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, kGemmSmem);
+    if (e != cudaSuccess) return e;
     const int n_tiles = p.m_tiles * p.n_tiles;
     if (n_tiles <= 0) return cudaSuccess;
     const int grid = n_tiles < sm_count ? n_tiles : sm_count;
-    qkv_gemm_kernel<<<grid, kGemmThreads, kGemmSmem, stream>>>(p, xmap, wmap);
+    if (p.head_dim == 128) qkv_gemm_kernel<128><<<grid, kGemmThreads, kGemmSmem, stream>>>(p, xmap, wmap);
+    else                   qkv_gemm_kernel<64><<<grid, kGemmThreads, kGemmSmem, stream>>>(p, xmap, wmap);
     count_launch();
     e = cudaGetLastError();
     if (e != cudaSuccess || !p.with_norm) return e;
-    const long long threads = (long long)p.n_tokens * (p.heads * p.head_dim / 8);
-    qkv_finish_kernel<<<(unsigned)((threads + 255) / 256), 256, 0, stream>>>(p);
+    qkv_finish_kernel<<<(unsigned)p.n_tokens, p.heads * p.head_dim / 8, 0, stream>>>(p);
     count_launch();
     return cudaGetLastError();
 }

@@ -45,7 +45,8 @@ enum {
     LL_ERR_UNSUPPORTED_SHAPE = -3,  /* shape outside what the kernels were built for */
     LL_ERR_NO_STORAGE = -4,         /* compute call before ll_cache_bind_storage */
     LL_ERR_CUDA = -5,               /* a CUDA runtime/driver call failed */
-    LL_ERR_DEVICE_TIMEOUT = -6      /* a kernel gave up on a bounded wait (see ll_cache_device_status) */
+    LL_ERR_DEVICE_TIMEOUT = -6,     /* a kernel gave up on a bounded wait (see ll_cache_device_status) */
+    LL_ERR_DEVICE_CHECK = -7        /* a kernel's own bounds check, or a guard band of a debug handle, tripped */
 };
 
 #define LL_MAX_SLOTS 64             /* sink_frames + window_frames <= LL_MAX_SLOTS */
@@ -372,7 +373,13 @@ int ll_cache_set_dry_run(ll_cache *cache, int on);
  * LL_ERR_DEVICE_TIMEOUT if a kernel abandoned a bounded wait (its outputs are
  * then invalid); ll_last_error() names the role and barrier.  On a time-out
  * the call also zeroes the arrival counters of the split-column merge, which
- * the abandoned launch left mid-count, so the handle can be used again. */
+ * the abandoned launch left mid-count, so the handle can be used again.
+ * LL_ERR_DEVICE_CHECK: an append kernel was handed a storage slot outside the
+ * layer and refused to write (it never is with the slot rule above; the check
+ * costs one comparison), or - for a handle created while the environment
+ * variable LL_DEBUG was set to something other than 0 - one of the two 4 KB
+ * guard bands that such a handle keeps in front of and behind its K/V region
+ * no longer holds its pattern (ll_cache_storage_bytes accounts for the bands). */
 int ll_cache_device_status(ll_cache *cache, ll_stream stream);
 
 /* Kernel launches made by this process through the library so far. */

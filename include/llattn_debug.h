@@ -79,6 +79,11 @@ int ll_debug_attn_plan_batched(const ll_attn_item *items, int n_items, int sm_co
 int ll_debug_aux_layout(const ll_cache *cache, size_t *status_offset, size_t *status_bytes,
                         size_t *counters_offset, size_t *counters_bytes);
 
+/* Where the guard bands of a handle created under LL_DEBUG sit inside its storage (byte
+ * offsets) and how long each is.  Lets a test overwrite one from the host and see
+ * ll_cache_device_status report it.  LL_ERR_INVALID_ARG for a handle without bands. */
+int ll_debug_guard_layout(const ll_cache *cache, size_t *front_offset, size_t *back_offset, size_t *bytes);
+
 #ifdef __cplusplus
 }
 #endif

@@ -20,6 +20,7 @@ LL_ERR_UNSUPPORTED_SHAPE = -3
 LL_ERR_NO_STORAGE = -4
 LL_ERR_CUDA = -5
 LL_ERR_DEVICE_TIMEOUT = -6
+LL_ERR_DEVICE_CHECK = -7
 LL_MAX_SLOTS = 64
 LL_KV_BF16, LL_KV_E4M3 = 0, 1
 LL_MAX_RANGES = 4
@@ -132,6 +133,7 @@ SIGNATURES = {
     "ll_debug_attn_plan": (C.c_int, [C.c_void_p, C.c_int, C.c_int, C.c_int, C.POINTER(ll_attn_plan)]),
     "ll_debug_attn_plan_batched": (C.c_int, [C.POINTER(ll_attn_item), C.c_int, C.c_int, C.POINTER(ll_attn_plan)]),
     "ll_debug_aux_layout": (C.c_int, [C.c_void_p] + [C.POINTER(C.c_size_t)] * 4),
+    "ll_debug_guard_layout": (C.c_int, [C.c_void_p] + [C.POINTER(C.c_size_t)] * 3),
     "ll_launch_count": (C.c_int64, []),
     "ll_last_error": (C.c_char_p, []),
     "ll_version": (C.c_char_p, []),
@@ -344,6 +346,13 @@ def ll_debug_aux_layout(h):
     """(status_offset, status_bytes, counters_offset, counters_bytes) inside the bound storage."""
     v = [C.c_size_t() for _ in range(4)]
     _check(lib().ll_debug_aux_layout(h, *[C.byref(x) for x in v]))
+    return tuple(x.value for x in v)
+
+
+def ll_debug_guard_layout(h):
+    """(front_offset, back_offset, bytes) of the guard bands of a handle created under LL_DEBUG."""
+    v = [C.c_size_t() for _ in range(3)]
+    _check(lib().ll_debug_guard_layout(h, *[C.byref(x) for x in v]))
     return tuple(x.value for x in v)
 
 

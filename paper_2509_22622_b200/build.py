@@ -59,7 +59,7 @@ def build(force: bool = False, verbose: bool = False) -> str:
         raise RuntimeError("nvcc failed")
     tmp = LIB + ".tmp%d" % os.getpid()
     subprocess.check_call([_nvcc(), "-shared", "-o", tmp] + objs +
-                          ["-gencode", "arch=compute_100a,code=sm_100a", "-Xcompiler", "-fPIC"])
+                          ["-gencode", "arch=compute_100a,code=sm_100a", "-Xcompiler", "-fPIC", "-ldl"])
     os.replace(tmp, LIB)
     return LIB
 

@@ -5,11 +5,33 @@
 #include <cmath>
 #include <cstdarg>
 #include <cstdio>
+#include <cstdlib>
 #include <cstring>
+
+#include <nvtx3/nvToolsExt.h>
 
 #include "ll_internal.h"
 
 namespace {
+
+// NVTX range around a compute call (the kernels it enqueues show up under it in a timeline),
+// only when the environment variable LL_NVTX is set to something other than 0.
+bool nvtx_on()
+{
+    static const bool on = [] { const char *e = getenv("LL_NVTX"); return e && e[0] && e[0] != '0'; }();
+    return on;
+}
+struct Range {
+    bool on;
+    Range(const char *what, int layer, long long frame) : on(nvtx_on())
+    {
+        if (!on) return;
+        char buf[96];
+        snprintf(buf, sizeof buf, "%s layer %d frame %lld", what, layer, frame);
+        nvtxRangePushA(buf);
+    }
+    ~Range() { if (on) nvtxRangePop(); }
+};
 
 thread_local std::string g_err;
 std::atomic<int64_t> g_launches{0};
@@ -92,6 +114,9 @@ const float *layer_scales(const ll_cache *c, int layer, int which)
     return reinterpret_cast<const float *>(c->storage + c->off_scales) + ((size_t)layer * 2 + which) * c->H;
 }
 
+constexpr size_t kGuardBytes = 4096;
+constexpr int kGuardByte = 0xA5;
+
 // Offsets of the aux block's parts and the size of a stored K (or V) matrix set.
 void compute_layout(ll_cache *c)
 {
@@ -112,6 +137,13 @@ void compute_layout(ll_cache *c)
         c->off_scales = end;
         c->off_stage = align_up(c->off_scales + (size_t)c->L * 2 * c->H * sizeof(float), 1024);
         end = align_up(c->off_stage + 2 * c->kv_bytes, 1024);
+    }
+    c->off_guard0 = c->off_guard1 = 0;
+    if (c->debug) {
+        // a band of a fixed pattern right in front of the K/V region (and one behind it, see
+        // ll_cache_storage_bytes): a kernel that writes outside the layers' rows trips one
+        c->off_guard0 = end;
+        end += kGuardBytes;
     }
     c->aux_bytes = end;
 }
@@ -218,6 +250,8 @@ int fill_rope_params(ll_cache *c, int layer, const ll_bf16 *q, const ll_bf16 *k,
     p->heads = c->H; p->P = c->P; p->grid_w = gw;
     p->n_t = n_t; p->n_h = n_h;
     for (int i = 0; i < n_frames; ++i) p->slot[i] = slot_of(c, frame_start + i);
+    p->status = reinterpret_cast<uint32_t *>(c->storage + c->off_status);
+    p->n_slots = c->n_slots;
     return LL_OK;
 }
 
@@ -498,6 +532,7 @@ int check_decode_item(ll_cache *c, int layer, const ll_bf16 *q_roped, int64_t q_
 int attn_entry(ll_cache *c, int layer, const ll_bf16 *q_roped, int64_t q_frame_start, int n_q_frames,
                ll_bf16 *out, float *lse_out, ll_stream stream, bool simt, const float *q_scale = nullptr)
 {
+    Range range("ll_sink_window_attn", layer, (long long)q_frame_start);
     int s = check_decode_item(c, layer, q_roped, q_frame_start, n_q_frames, out, lse_out);
     if (s != LL_OK) return s;
     if (simt && c->kv_format != LL_KV_BF16) return fail(LL_ERR_UNSUPPORTED_SHAPE, "the triage kernel reads bf16 caches only");
@@ -556,6 +591,8 @@ int ll_cache_create(int layers, int heads, int head_dim, int tokens_per_frame, i
     for (auto &l : c->layers)
         for (int s = 0; s < LL_MAX_SLOTS; ++s) l.slot_frame[s] = -1;
     c->scales.assign((size_t)layers * 2 * heads, 1.f);
+    const char *dbg = getenv("LL_DEBUG");
+    c->debug = dbg && dbg[0] && dbg[0] != '0';
     compute_layout(c);
     *out = c;
     return LL_OK;
@@ -566,7 +603,7 @@ void ll_cache_destroy(ll_cache *cache) { delete cache; }
 size_t ll_cache_storage_bytes(const ll_cache *c)
 {
     if (!c) return 0;
-    return c->aux_bytes + (size_t)c->L * 2 * c->kv_store_bytes;
+    return c->aux_bytes + (size_t)c->L * 2 * c->kv_store_bytes + (c->debug ? kGuardBytes : 0);
 }
 
 int ll_cache_bind_storage(ll_cache *c, void *dev, size_t bytes, ll_stream stream)
@@ -578,6 +615,13 @@ int ll_cache_bind_storage(ll_cache *c, void *dev, size_t bytes, ll_stream stream
     if (c->dry_run) return fail(LL_ERR_INVALID_ARG, "handle is in bookkeeping-only mode");
     cudaError_t e = cudaMemsetAsync(dev, 0, ll_cache_storage_bytes(c), (cudaStream_t)stream);
     if (e != cudaSuccess) return cuda_fail(e, "cudaMemsetAsync(storage)");
+    if (c->debug) {
+        c->off_guard1 = c->aux_bytes + (size_t)c->L * 2 * c->kv_store_bytes;
+        e = cudaMemsetAsync(static_cast<char *>(dev) + c->off_guard0, kGuardByte, kGuardBytes, (cudaStream_t)stream);
+        if (e == cudaSuccess)
+            e = cudaMemsetAsync(static_cast<char *>(dev) + c->off_guard1, kGuardByte, kGuardBytes, (cudaStream_t)stream);
+        if (e != cudaSuccess) return cuda_fail(e, "cudaMemsetAsync(guard bands)");
+    }
     cudaPointerAttributes attr;
     int sms = 0;
     e = cudaPointerGetAttributes(&attr, dev);
@@ -660,6 +704,7 @@ int append_entry(ll_cache *c, int layer, const ll_bf16 *q, const ll_bf16 *k, con
                  int64_t frame_start, int n_frames, int grid_h, int grid_w, float rope_theta,
                  ll_bf16 *q_out, ll_stream stream)
 {
+    Range range(with_norm ? "ll_norm_rope_append_kv" : "ll_rope_append_kv", layer, (long long)frame_start);
     if (!layer_ok(c, layer)) return fail(LL_ERR_INVALID_ARG, "bad cache handle or layer %d", layer);
     if (grid_h <= 0 || grid_w <= 0 || (int64_t)grid_h * grid_w != c->P)
         return fail(LL_ERR_INVALID_ARG, "grid %dx%d does not give %d tokens per frame", grid_h, grid_w, c->P);
@@ -755,6 +800,7 @@ int ll_qkv_proj_append(ll_cache *c, int layer, const ll_bf16 *x, int d_model, co
     if (grid_h <= 0 || grid_w <= 0 || (int64_t)grid_h * grid_w != c->P)
         return fail(LL_ERR_INVALID_ARG, "grid %dx%d does not give %d tokens per frame", grid_h, grid_w, c->P);
     if (!(rope_theta > 0.f)) return fail(LL_ERR_INVALID_ARG, "rope_theta must be positive");
+    Range range("ll_qkv_proj_append", layer, (long long)frame_start);
     if (d_model < 64 || d_model % 8) return fail(LL_ERR_UNSUPPORTED_SHAPE, "d_model must be a multiple of 8, at least 64");
     if ((c->H * c->D) % 256 || c->H * c->D > 8192)
         return fail(LL_ERR_UNSUPPORTED_SHAPE, "heads * head_dim must be a multiple of 256, at most 8192");
@@ -825,6 +871,7 @@ int ll_qkv_proj_append(ll_cache *c, int layer, const ll_bf16 *x, int d_model, co
 
 int ll_sink_window_attn_batched(const ll_attn_item *items, int n_items, ll_stream stream)
 {
+    Range range("ll_sink_window_attn_batched items", n_items, 0);
     if (!items || n_items < 1) return fail(LL_ERR_INVALID_ARG, "no items");
     if (n_items > LL_MAX_BATCH) return fail(LL_ERR_UNSUPPORTED_SHAPE, "more than %d items", LL_MAX_BATCH);
     static_assert(LL_MAX_BATCH == ll::kMaxItems, "header and kernel disagree on the batch limit");
@@ -867,6 +914,7 @@ int ll_recache(ll_cache *c, int layer, const ll_bf16 *q, const ll_bf16 *k, const
     if (!(rope_theta > 0.f)) return fail(LL_ERR_INVALID_ARG, "rope_theta must be positive");
     ll::LayerState &st = c->layers[layer];
     const int64_t r0 = std::max<int64_t>(c->S, st.end - c->W);
+    Range range("ll_recache", layer, (long long)r0);
     const int64_t resident = std::max<int64_t>(0, st.end - r0);
     if (n_frames != resident)
         return fail(LL_ERR_BAD_POSITION, "n_frames %d != resident window frames %lld", n_frames, (long long)resident);
@@ -904,6 +952,7 @@ int ll_recache(ll_cache *c, int layer, const ll_bf16 *q, const ll_bf16 *k, const
 int ll_cross_attn(ll_cache *c, const ll_bf16 *q, int64_t n_q, const ll_bf16 *k, const ll_bf16 *v, int64_t n_k,
                   ll_bf16 *out, float *lse_out, ll_stream stream)
 {
+    Range range("ll_cross_attn keys", (int)n_k, 0);
     if (!c) return fail(LL_ERR_INVALID_ARG, "null handle");
     if (n_q <= 0 || n_k <= 0) return fail(LL_ERR_INVALID_ARG, "n_q and n_k must be positive");
     if (n_q > (1ll << 30) || n_k > (1ll << 30)) return fail(LL_ERR_UNSUPPORTED_SHAPE, "more than 2^30 queries or keys");
@@ -933,6 +982,7 @@ int ll_clip_append_attn(ll_cache *c, int layer, const ll_bf16 *q, const ll_bf16 
     if (grid_h <= 0 || grid_w <= 0 || (int64_t)grid_h * grid_w != c->P)
         return fail(LL_ERR_INVALID_ARG, "grid %dx%d does not give %d tokens per frame", grid_h, grid_w, c->P);
     if (!(rope_theta > 0.f)) return fail(LL_ERR_INVALID_ARG, "rope_theta must be positive");
+    Range range("ll_clip_append_attn", layer, (long long)frame_start);
     if (n_frames <= 0 || n_frames % c->C)
         return fail(LL_ERR_BAD_POSITION, "n_frames %d is not a positive multiple of chunk_frames %d", n_frames, c->C);
     const int n_groups = n_frames / c->C;
@@ -1091,6 +1141,16 @@ int ll_debug_aux_layout(const ll_cache *c, size_t *status_offset, size_t *status
     return LL_OK;
 }
 
+int ll_debug_guard_layout(const ll_cache *c, size_t *front_offset, size_t *back_offset, size_t *bytes)
+{
+    if (!c) return fail(LL_ERR_INVALID_ARG, "null handle");
+    if (!c->debug) return fail(LL_ERR_INVALID_ARG, "the handle was not created with LL_DEBUG set");
+    if (front_offset) *front_offset = c->off_guard0;
+    if (back_offset) *back_offset = c->aux_bytes + (size_t)c->L * 2 * c->kv_store_bytes;
+    if (bytes) *bytes = kGuardBytes;
+    return LL_OK;
+}
+
 int ll_cache_reset(ll_cache *c)
 {
     if (!c) return fail(LL_ERR_INVALID_ARG, "null handle");
@@ -1164,6 +1224,16 @@ int ll_cache_device_status(ll_cache *c, ll_stream stream)
     uint32_t w[ll::kStatusWords];
     e = cudaMemcpy(w, c->storage + c->off_status, sizeof w, cudaMemcpyDeviceToHost);
     if (e != cudaSuccess) return cuda_fail(e, "cudaMemcpy(status)");
+    if (w[0] == ll::kStatusOk && c->debug) {
+        static unsigned char band[2 * kGuardBytes];
+        e = cudaMemcpy(band, c->storage + c->off_guard0, kGuardBytes, cudaMemcpyDeviceToHost);
+        if (e == cudaSuccess) e = cudaMemcpy(band + kGuardBytes, c->storage + c->off_guard1, kGuardBytes, cudaMemcpyDeviceToHost);
+        if (e != cudaSuccess) return cuda_fail(e, "cudaMemcpy(guard bands)");
+        for (size_t i = 0; i < 2 * kGuardBytes; ++i)
+            if (band[i] != kGuardByte)
+                return fail(LL_ERR_DEVICE_CHECK, "guard band %s the K/V region overwritten at byte %zu",
+                            i < kGuardBytes ? "in front of" : "behind", i % kGuardBytes);
+    }
     if (w[0] == ll::kStatusOk) return LL_OK;
     // A CTA that gave up, and every CTA that then skipped its work, never made its arrival on
     // the split-column counters, so the counters of that launch are left mid-count: clear them
@@ -1171,6 +1241,9 @@ int ll_cache_device_status(ll_cache *c, ll_stream stream)
     e = cudaMemset(c->storage + c->off_status, 0, sizeof w);
     if (e == cudaSuccess) e = cudaMemset(c->storage + c->off_counters, 0, ll::counters_bytes());
     if (e != cudaSuccess) return cuda_fail(e, "cudaMemset(status, counters)");
+    if (w[0] == ll::kStatusBadRow)
+        return fail(LL_ERR_DEVICE_CHECK, "an append kernel refused storage slot %u of the call's frame %u (block %u)",
+                    w[1], w[2], w[4]);
     return fail(LL_ERR_DEVICE_TIMEOUT,
                 "a kernel gave up on a bounded wait: code %u role %u barrier %u iteration %u block (%u,%u,%u)",
                 w[0], w[1], w[2], w[3], w[4], w[5], w[6]);

@@ -27,7 +27,22 @@ constexpr int kSlabs = 16;            // 16-row warp slabs in a work column (2 t
 enum StatusCode : uint32_t {
     kStatusOk = 0,
     kStatusTimeout = 1,
+    kStatusBadRow = 2,                // an append kernel was handed a storage slot outside the layer
 };
+
+#ifdef __CUDACC__
+// First come, first served: the record stays until the host has read it.
+__device__ __forceinline__ void record_status(uint32_t *status, uint32_t code, uint32_t a, uint32_t b)
+{
+    if (atomicCAS(status, 0u, code) == 0u) {
+        status[1] = a;
+        status[2] = b;
+        status[3] = 0;
+        status[4] = blockIdx.x; status[5] = blockIdx.y; status[6] = blockIdx.z;
+        __threadfence();
+    }
+}
+#endif
 
 struct LayerState {
     int64_t end = 0;
@@ -121,6 +136,8 @@ struct RopeAppendParams {
     int n_tokens, heads, P, grid_w;
     int n_t, n_h;                     // pairs of the t and h bands (w band takes the rest)
     int slot[LL_MAX_SLOTS];           // storage slot of the call's i-th frame
+    uint32_t *status;                 // aux status words
+    int n_slots;                      // S + W: a slot outside [0, n_slots) is refused by the kernel
 };
 
 // QKV projection with norm, rotation and append in its epilogue (qkv_gemm.cu).
@@ -182,6 +199,8 @@ struct ll_cache {
     int64_t rows;                     // (S+W)*P cache rows per head
     std::vector<ll::LayerState> layers;
     bool dry_run = false;
+    bool debug = false;               // LL_DEBUG=1 at create time: guard bands around the K/V region
+    size_t off_guard0 = 0, off_guard1 = 0;
 
     char *storage = nullptr;
     size_t storage_bytes = 0;

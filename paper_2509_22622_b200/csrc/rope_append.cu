@@ -73,6 +73,10 @@ rope_append_kernel(const __grid_constant__ RopeAppendParams p)
     const int frame = (int)(token / p.P);
     const int cell = (int)(token % p.P);
     const int y = cell / p.grid_w, x = cell % p.grid_w;
+    if ((unsigned)p.slot[frame] >= (unsigned)p.n_slots) {         // never with the host's slot rule: refuse, report
+        record_status(p.status, kStatusBadRow, (uint32_t)p.slot[frame], (uint32_t)frame);
+        return;
+    }
 
     float2 cs[4];
 #pragma unroll
@@ -138,6 +142,10 @@ rope_append_e4m3_kernel(const __grid_constant__ RopeAppendParams p)
     const int frame = (int)(token / p.P);
     const int cell = (int)(token % p.P);
     const int y = cell / p.grid_w, x = cell % p.grid_w;
+    if ((unsigned)p.slot[frame] >= (unsigned)p.n_slots) {         // never with the host's slot rule: refuse, report
+        record_status(p.status, kStatusBadRow, (uint32_t)p.slot[frame], (uint32_t)frame);
+        return;
+    }
     float2 cs[4];
 #pragma unroll
     for (int u = 0; u < 4; ++u) {
@@ -268,6 +276,10 @@ norm_rope_append_kernel(const __grid_constant__ RopeAppendParams p, const float 
     const int frame = (int)(token / p.P);
     const int cell = (int)(token % p.P);
     const int y = cell / p.grid_w, x = cell % p.grid_w;
+    if ((unsigned)p.slot[frame] >= (unsigned)p.n_slots) {         // never with the host's slot rule: refuse, report
+        record_status(p.status, kStatusBadRow, (uint32_t)p.slot[frame], (uint32_t)frame);
+        return;
+    }
     const size_t in_base = (size_t)token * row_vecs * 8;
     const bool with_q = p.q_out != nullptr;
 

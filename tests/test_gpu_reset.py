@@ -159,3 +159,49 @@ def test_replayed_append_after_the_tables_moved(oracle_mod):
     want_q = synth.f32_to_bf16_bits(oracle_mod.rope(F64(q2), 900, wl.grid_h, wl.grid_w, wl.rope_theta).astype(np.float32))
     assert ulp_distance(bits(s_qout), want_q).max() <= 1
     cache.close()
+
+
+def test_debug_handle_guard_bands_and_nvtx_ranges(oracle_mod, monkeypatch):
+    """A handle created under LL_DEBUG keeps a 4 KB band of a fixed pattern in front of and
+    behind its K/V region: a stream with wrap-around, a recache and a clip leave both intact
+    (no kernel writes outside the layers' rows), and a band overwritten from the host is
+    reported.  The calls run inside NVTX ranges (LL_NVTX) without changing any result."""
+    monkeypatch.setenv("LL_DEBUG", "1")
+    monkeypatch.setenv("LL_NVTX", "1")
+    wl = synth.Workload("debug", 2, 2, 128, 7, 19, 1, 1, 4, n_chunks=7, seed=55)
+    plain_bytes = None
+    monkeypatch.delenv("LL_DEBUG")
+    h = B.ll_cache_create(*wl.cache_args)
+    plain_bytes = B.ll_cache_storage_bytes(h)
+    B.ll_cache_destroy(h)
+    monkeypatch.setenv("LL_DEBUG", "1")
+    cache = B.Cache(*wl.cache_args)
+    front, back, nbytes = B.ll_debug_guard_layout(cache.h)
+    assert B.ll_cache_storage_bytes(cache.h) == plain_bytes + 2 * nbytes and back + nbytes == plain_bytes + 2 * nbytes
+    orc = oracle_mod.Oracle(*wl.cache_args)
+    C = wl.chunk_frames
+    for layer in (0, 1):                                   # layer 0 touches the front band's neighbour rows, layer 1 the back's
+        for chunk in range(wl.n_chunks):
+            q, k, v = synth.chunk_qkv(wl, chunk, layer=layer)
+            dq = dev(q)
+            q_out, out = torch.empty_like(dq), torch.empty_like(dq)
+            cache.rope_append_kv(layer, dq, dev(k), dev(v), chunk * C, wl.grid_h, wl.grid_w, wl.rope_theta, q_out)
+            cache.sink_window_attn(layer, q_out, chunk * C, out)
+            orc.append(layer, F64(k), F64(v), chunk * C, wl.grid_h, wl.grid_w, wl.rope_theta)
+        cache.check_device()
+        want, _ = orc.attn(layer, orc.rope_q(F64(q), (wl.n_chunks - 1) * C, wl.grid_h, wl.grid_w, wl.rope_theta),
+                           (wl.n_chunks - 1) * C)
+        check_attn(f64(out), want)
+        n = wl.window_frames
+        rq, rk, rv = (dev(t) for t in synth.chunk_qkv(wl, 99, layer=layer, n_frames=n))
+        cache.recache(layer, rq, rk, rv, n, wl.grid_h, wl.grid_w, wl.rope_theta, torch.empty_like(rq), torch.empty_like(rq))
+        cache.check_device()
+    band = cache.storage[back:back + nbytes]
+    assert bool((band == 0xA5).all())
+    band[17] = 0
+    with pytest.raises(B.LLError) as e:
+        cache.check_device()
+    assert e.value.code == B.LL_ERR_DEVICE_CHECK and "behind" in str(e.value) and "byte 17" in str(e.value)
+    band[17] = 0xA5
+    cache.check_device()
+    cache.close()

@@ -86,6 +86,9 @@ def lib():
             L.llo_clip.argtypes = [C.c_void_p, C.c_int] + [C.POINTER(C.c_double)] * 3 + \
                                   [C.c_int64, C.c_int, C.c_int, C.c_int, C.c_int, C.c_double,
                                    C.POINTER(C.c_int64), C.c_int64] + [C.POINTER(C.c_double)] * 3
+            L.llo_clip_backward.argtypes = [C.c_void_p, C.c_int, C.POINTER(C.c_double), C.POINTER(C.c_double),
+                                            C.c_int64, C.c_int, C.c_int, C.c_int, C.c_int, C.c_double] + \
+                                           [C.POINTER(C.c_double)] * 6
             L.llo_rms_norm.argtypes = [C.POINTER(C.c_double), C.POINTER(C.c_double), C.c_double, C.c_int64, C.c_int,
                                        C.POINTER(C.c_double)]
             L.llo_dense_attn.argtypes = [C.POINTER(C.c_double)] * 3 + [C.c_int64, C.c_int64, C.c_int, C.c_int,
@@ -313,6 +316,22 @@ class Oracle:
         if st != OK:
             raise OracleError(st, "clip")
         return qr, out, lse
+
+    def clip_backward(self, layer, q, d_out, frame_start, n_frames, window, gh, gw, theta=10000.0):
+        """Gradients of a scalar loss through the clip step that was just run (the cache is as
+        ``clip`` left it): q is the clip's unrotated query tensor, d_out the loss gradient with
+        respect to the clip's attention output.  Returns (dq, dk, dv, mag_q, mag_k, mag_v), all
+        [n_frames*P, H, D]: gradients with respect to the q, k, v handed to ``clip`` and the
+        sums of absolute values of the terms each element adds up."""
+        q, g = _f64(q), _f64(d_out)
+        if q.shape != (n_frames * gh * gw, self.H, self.D) or g.shape != q.shape:
+            raise OracleError(ERR_ARG, "clip_backward shape")
+        outs = [np.empty_like(q) for _ in range(6)]
+        st = lib().llo_clip_backward(self._h, layer, _dp(q), _dp(g), frame_start, n_frames, window, gh, gw, theta,
+                                     *[_dp(a) for a in outs])
+        if st != OK:
+            raise OracleError(st, "clip_backward")
+        return tuple(outs)
 
     def visible_window(self, fq: int, fk: int, window: int) -> bool:
         return bool(lib().llo_visible_window(self._h, fq, fk, window))

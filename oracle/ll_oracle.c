@@ -528,6 +528,175 @@ int llo_clip(llo *o, int layer, const double *q, const double *k, const double *
     return st;
 }
 
+/* ---- step: gradients of the clip step (Sec. 3.3, "Consistency between Training and Inference":
+ * the clip's T frames carry gradients, the sink and the preceding context are detached;
+ * Algorithm 1 back-propagates the loss of the newest clip only) ------------------------------- */
+
+/* The inverse of rope_row: rotate every pair by minus its angle (the rotation is orthogonal,
+ * so the gradient with respect to the unrotated row is the rotated gradient turned back). */
+static void rope_row_back(const double *in, double *out, int D, double theta, int64_t t, int y, int x)
+{
+    int n_t, n_h, n_w;
+    llo_rope_split(D, &n_t, &n_h, &n_w);
+    for (int j = 0; j < D / 2; ++j) {
+        double pos; int i, n_a;
+        if (j < n_t)            { pos = (double)t; i = j;             n_a = n_t; }
+        else if (j < n_t + n_h) { pos = (double)y; i = j - n_t;       n_a = n_h; }
+        else                    { pos = (double)x; i = j - n_t - n_h; n_a = n_w; }
+        double ang = pos * pow(theta, -(double)i / (double)n_a);
+        double c = cos(ang), s = sin(ang);
+        double a = in[2 * j], b = in[2 * j + 1];
+        out[2 * j]     = a * c + b * s;
+        out[2 * j + 1] = -a * s + b * c;
+    }
+}
+
+/* Given the cache as llo_clip left it, the clip's unrotated queries q and the gradient d_out of
+ * a scalar loss with respect to the clip's attention output, the gradients with respect to the
+ * clip's q, k and v as they were handed to llo_clip (before the rotation), all [n_frames*P, H, D].
+ * With s_ij = q_i.k_j / sqrt(D) over the keys j visible to row i, p = softmax(s), o_i = sum p_ij v_j:
+ *   delta_i = d_out_i . o_i,  dP_ij = d_out_i . v_j,  dS_ij = p_ij (dP_ij - delta_i),
+ *   dq_i = sum_j dS_ij k_j / sqrt(D),  dk_j = sum_i dS_ij q_i / sqrt(D),  dv_j = sum_i p_ij d_out_i,
+ * (q, k after rotation), dk and dv only for keys that are frames of the clip, then dq and dk
+ * turned back through the rotation.  mag_* (nullable, same shapes) receive the sums of the
+ * absolute values of the terms each gradient element adds up (dq, dk: in the rotated frame,
+ * summed over the element's rotation pair): the scale of its rounding error. */
+int llo_clip_backward(const llo *o, int layer, const double *q, const double *d_out,
+                      int64_t frame_start, int n_frames, int window, int gh, int gw, double theta,
+                      double *dq, double *dk, double *dv, double *mag_q, double *mag_k, double *mag_v)
+{
+    if (!o || layer < 0 || layer >= o->L || !q || !d_out || !dq || !dk || !dv) return LLO_ERR_ARG;
+    if (gh * gw != o->P || n_frames <= 0 || n_frames % o->C) return LLO_ERR_ARG;
+    if (frame_start + n_frames != o->end[layer]) return LLO_ERR_POSITION;
+    const int H = o->H, D = o->D, P = o->P;
+    const int64_t nq = (int64_t)n_frames * P;
+    const size_t re = row_elems(o);
+    const double scale = 1.0 / sqrt((double)D);
+    const int32_t *sf = o->slot_frame + (size_t)layer * slots(o);
+    const double *K = o->K + (size_t)layer * layer_elems(o);
+    const double *V = o->V + (size_t)layer * layer_elems(o);
+    double *qr = (double *)malloc(sizeof(double) * (size_t)nq * re);
+    double *lse = (double *)malloc(sizeof(double) * (size_t)nq * H);
+    double *delta = (double *)malloc(sizeof(double) * (size_t)nq * H);
+    double *dq_r = (double *)calloc((size_t)nq * re, sizeof(double));      /* gradients in the rotated frame */
+    double *dk_r = (double *)calloc((size_t)nq * re, sizeof(double));
+    double *mq = (double *)calloc((size_t)nq * re, sizeof(double));
+    double *mk = (double *)calloc((size_t)nq * re, sizeof(double));
+    if (!qr || !lse || !delta || !dq_r || !dk_r || !mq || !mk) return LLO_ERR_ARG;
+    llo_rope(q, qr, nq, H, D, frame_start, gh, gw, theta, o->faithful);
+    memset(dv, 0, sizeof(double) * (size_t)nq * re);
+    if (mag_v) memset(mag_v, 0, sizeof(double) * (size_t)nq * re);
+    int status = LLO_OK;
+
+    /* pass 1, per query row: softmax statistics, delta, dq */
+#pragma omp parallel for schedule(dynamic, 1)
+    for (int64_t r = 0; r < nq; ++r) {
+        int64_t fq = frame_start + r / P;
+        int64_t hi = (fq / o->C + 1) * o->C;
+        for (int h = 0; h < H; ++h) {
+            const double *qv = qr + ((size_t)r * H + h) * D;
+            const double *go = d_out + ((size_t)r * H + h) * D;
+            /* scores over the visible keys */
+            double m = -INFINITY, denom = 0.0;
+            for (int pass = 0; pass < 2; ++pass)
+                for (int64_t fk = 0; fk < hi; ++fk) {
+                    if (!visible_in_window(o, fq, fk, 0, window)) continue;
+                    int slot = llo_slot_of(o, fk);
+                    if (sf[slot] != (int32_t)fk) { status = LLO_ERR_NOT_RESIDENT; continue; }
+                    for (int n = 0; n < P; ++n) {
+                        const double *kv = K + (((size_t)slot * P + n) * H + h) * D;
+                        double dot = 0.0;
+                        for (int d = 0; d < D; ++d) dot += qv[d] * kv[d];
+                        dot *= scale;
+                        if (pass == 0) { if (dot > m) m = dot; } else denom += exp(dot - m);
+                    }
+                }
+            double l = m + log(denom);
+            lse[(size_t)r * H + h] = l;
+            /* o_i and delta_i */
+            double dl = 0.0;
+            double *ov = (double *)calloc((size_t)D, sizeof(double));
+            for (int64_t fk = 0; fk < hi; ++fk) {
+                if (!visible_in_window(o, fq, fk, 0, window)) continue;
+                int slot = llo_slot_of(o, fk);
+                for (int n = 0; n < P; ++n) {
+                    const double *kv = K + (((size_t)slot * P + n) * H + h) * D;
+                    const double *vv = V + (((size_t)slot * P + n) * H + h) * D;
+                    double dot = 0.0;
+                    for (int d = 0; d < D; ++d) dot += qv[d] * kv[d];
+                    double p = exp(dot * scale - l);
+                    for (int d = 0; d < D; ++d) ov[d] += p * vv[d];
+                }
+            }
+            for (int d = 0; d < D; ++d) dl += go[d] * ov[d];
+            free(ov);
+            delta[(size_t)r * H + h] = dl;
+            /* dq_i */
+            double *gq = dq_r + ((size_t)r * H + h) * D, *gm = mq + ((size_t)r * H + h) * D;
+            for (int64_t fk = 0; fk < hi; ++fk) {
+                if (!visible_in_window(o, fq, fk, 0, window)) continue;
+                int slot = llo_slot_of(o, fk);
+                for (int n = 0; n < P; ++n) {
+                    const double *kv = K + (((size_t)slot * P + n) * H + h) * D;
+                    const double *vv = V + (((size_t)slot * P + n) * H + h) * D;
+                    double dot = 0.0, dp = 0.0;
+                    for (int d = 0; d < D; ++d) { dot += qv[d] * kv[d]; dp += go[d] * vv[d]; }
+                    double p = exp(dot * scale - l);
+                    double ds = p * (dp - dl) * scale;
+                    for (int d = 0; d < D; ++d) { gq[d] += ds * kv[d]; gm[d] += fabs(ds * kv[d]); }
+                }
+            }
+        }
+    }
+
+    /* pass 2, per key row of the clip: dk_j and dv_j over the query rows that see it */
+#pragma omp parallel for schedule(dynamic, 1)
+    for (int64_t j = 0; j < nq; ++j) {
+        int64_t fk = frame_start + j / P;
+        int slot = llo_slot_of(o, fk);
+        int n = (int)(j % P);
+        for (int h = 0; h < H; ++h) {
+            const double *kv = K + (((size_t)slot * P + n) * H + h) * D;
+            const double *vv = V + (((size_t)slot * P + n) * H + h) * D;
+            double *gk = dk_r + ((size_t)j * H + h) * D, *gkm = mk + ((size_t)j * H + h) * D;
+            double *gv = dv + ((size_t)j * H + h) * D;
+            double *gvm = mag_v ? mag_v + ((size_t)j * H + h) * D : NULL;
+            for (int64_t r = 0; r < nq; ++r) {
+                int64_t fq = frame_start + r / P;
+                if (!visible_in_window(o, fq, fk, 0, window)) continue;
+                const double *qv = qr + ((size_t)r * H + h) * D;
+                const double *go = d_out + ((size_t)r * H + h) * D;
+                double dot = 0.0, dp = 0.0;
+                for (int d = 0; d < D; ++d) { dot += qv[d] * kv[d]; dp += go[d] * vv[d]; }
+                double p = exp(dot * scale - lse[(size_t)r * H + h]);
+                double ds = p * (dp - delta[(size_t)r * H + h]) * scale;
+                for (int d = 0; d < D; ++d) {
+                    gk[d] += ds * qv[d]; gkm[d] += fabs(ds * qv[d]);
+                    gv[d] += p * go[d];
+                    if (gvm) gvm[d] += fabs(p * go[d]);
+                }
+            }
+        }
+    }
+
+    /* back through the rotation */
+    for (int64_t r = 0; r < nq; ++r) {
+        int64_t t = frame_start + r / P;
+        int y = (int)((r % P) / gw), x = (int)((r % P) % gw);
+        for (int h = 0; h < H; ++h) {
+            size_t off = ((size_t)r * H + h) * D;
+            rope_row_back(dq_r + off, dq + off, D, theta, t, y, x);
+            rope_row_back(dk_r + off, dk + off, D, theta, t, y, x);
+            for (int d = 0; d < D; d += 2) {
+                if (mag_q) mag_q[off + d] = mag_q[off + d + 1] = mq[off + d] + mq[off + d + 1];
+                if (mag_k) mag_k[off + d] = mag_k[off + d + 1] = mk[off + d] + mk[off + d + 1];
+            }
+        }
+    }
+    free(qr); free(lse); free(delta); free(dq_r); free(dk_r); free(mq); free(mk);
+    return status;
+}
+
 /* ---- step: RMS norm of q and k rows (upstream of the rotation) ---------------- */
 
 /* y[t][e] = x[t][e] / sqrt(mean_e(x[t][e]^2) + eps) * gain[e], e over the token's

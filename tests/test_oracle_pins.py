@@ -771,3 +771,64 @@ def test_qkv_projection_equals_the_written_out_sum_and_splits_q_k_v(oracle_mod):
     eye = np.eye(dm)
     q, k, v = oracle_mod.qkv_proj(x, np.concatenate([eye, 2 * eye, -eye]))
     assert np.array_equal(q, x) and np.array_equal(k, 2 * x) and np.array_equal(v, -x)
+
+
+# ---------------------------------------------------------------------------
+# gradients of the clip step
+# ---------------------------------------------------------------------------
+
+def _clip_loss(oracle_mod, shape, ctx, q, k, v, G, window):
+    """sum(out * G) of a clip run on a fresh cache holding the context frames."""
+    H, D, gh, gw, C, S, W = shape
+    orc = oracle_mod.Oracle(1, H, D, gh * gw, C, S, W)
+    for f, (ck, cv) in enumerate(ctx):
+        orc.append(0, ck, cv, f * C, gh, gw)
+    n_frames = q.shape[0] // (gh * gw)
+    _, out, _ = orc.clip(0, q, k, v, len(ctx) * C, n_frames, window, gh, gw)
+    return float((out * G).sum()), orc
+
+
+def test_clip_backward_equals_central_finite_differences(oracle_mod):
+    """Every element of dq, dk, dv against (L(x + e) - L(x - e)) / 2e of the pinned forward clip,
+    L = sum(out * G): sink + context tail + earlier clip chunks all in play, window shorter than
+    the clip, gradients through the rotation."""
+    H, D, gh, gw, C, S, W = 2, 8, 1, 2, 1, 1, 5
+    shape = (H, D, gh, gw, C, S, W)
+    P, T, window = gh * gw, 3, 2
+    rng = np.random.default_rng(11)
+    ctx = [(rng.standard_normal((C * P, H, D)), rng.standard_normal((C * P, H, D))) for _ in range(2)]
+    q, k, v = (rng.standard_normal((T * P, H, D)) for _ in range(3))
+    G = rng.standard_normal((T * P, H, D))
+    _, orc = _clip_loss(oracle_mod, shape, ctx, q, k, v, G, window)
+    dq, dk, dv, mq, mk, mv = orc.clip_backward(0, q, G, 2 * C, T, window, gh, gw)
+    eps = 1e-5
+    for name, x, g in (("q", q, dq), ("k", k, dk), ("v", v, dv)):
+        fd = np.zeros_like(x)
+        for idx in np.ndindex(x.shape):
+            xp, xm = x.copy(), x.copy()
+            xp[idx] += eps
+            xm[idx] -= eps
+            args_p = dict(q=q, k=k, v=v); args_p[name] = xp
+            args_m = dict(q=q, k=k, v=v); args_m[name] = xm
+            fd[idx] = (_clip_loss(oracle_mod, shape, ctx, args_p["q"], args_p["k"], args_p["v"], G, window)[0] -
+                       _clip_loss(oracle_mod, shape, ctx, args_m["q"], args_m["k"], args_m["v"], G, window)[0]) / (2 * eps)
+        assert np.abs(fd - g).max() < 1e-7, (name, np.abs(fd - g).max())
+        assert np.abs(g).max() > 1e-3                         # not trivially zero
+    # the magnitudes bound the gradients they belong to (rotation pairs share one bound)
+    assert (np.abs(dv) <= mv + 1e-12).all()
+    pair = lambda a: np.repeat(np.abs(a).reshape(T * P, H, D // 2, 2).sum(axis=3), 2, axis=2).reshape(a.shape)
+    assert (pair(dq) <= 2 * mq + 1e-12).all() and (pair(dk) <= 2 * mk + 1e-12).all()
+
+
+def test_clip_backward_closed_forms(oracle_mod):
+    """One visible key per query (one-token frames, no sink, window of one frame): o_i = v_i, so
+    dv = d_out and dq = dk = 0.  And d_out = 0 gives zero gradients."""
+    H, D = 2, 8
+    orc = oracle_mod.Oracle(1, H, D, 1, 1, 0, 4)
+    rng = np.random.default_rng(12)
+    q, k, v, G = (rng.standard_normal((3, H, D)) for _ in range(4))
+    orc.clip(0, q, k, v, 0, 3, 1, 1, 1)
+    dq, dk, dv, *_ = orc.clip_backward(0, q, G, 0, 3, 1, 1, 1)
+    assert np.abs(dv - G).max() < 1e-14 and np.abs(dq).max() < 1e-14 and np.abs(dk).max() < 1e-14
+    dq, dk, dv, *_ = orc.clip_backward(0, q, 0 * G, 0, 3, 1, 1, 1)
+    assert not dq.any() and not dk.any() and not dv.any()

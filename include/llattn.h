@@ -291,6 +291,31 @@ int ll_clip_append_attn(ll_cache *cache, int layer, const ll_bf16 *q, const ll_b
                         int attn_window_frames, int grid_h, int grid_w, float rope_theta,
                         ll_bf16 *q_out, ll_bf16 *out, float *lse_out, ll_stream stream);
 
+/* Backward of ll_clip_append_attn: gradients of a scalar loss through the clip step (Sec. 3.3
+ * "Consistency between Training and Inference": the clip's T frames carry gradients, the sink
+ * and the preceding context are detached; Algorithm 1 back-propagates the newest clip's loss).
+ * Call it while the cache is as the forward left it (frame_start + n_frames == end; same
+ * attn_window_frames, grid and rope_theta).
+ *   q_roped  the forward's q_out; out, lse: the forward's outputs (lse is required here);
+ *   d_out    gradient of the loss with respect to out, bf16 [n_frames*tokens_per_frame, heads, head_dim]
+ *   dq, dk, dv  bf16, same shape: gradients with respect to the q, k, v that were handed to the
+ *            forward (BEFORE the rotation: dq and dk are turned back through it); dk, dv cover
+ *            the clip's own keys only.
+ *   workspace  device, 256-byte aligned, >= ll_clip_backward_workspace_bytes (one float per query
+ *            row and head), caller-owned.
+ * With s_ij the scaled scores over the keys visible to row i and p = softmax(s):
+ *   dv_j = sum_i p_ij d_out_i;  dS_ij = p_ij (d_out_i.v_j - d_out_i.out_i);
+ *   dq_i = sum_j dS_ij k_j / sqrt(D);  dk_j = sum_i dS_ij q_i / sqrt(D).
+ * P and dS are rounded to bf16 for the tensor-core products (fp32 accumulation); every element is
+ * accumulated by one thread block in one order, so the result is run-to-run deterministic.  bf16
+ * caches only.  State is not changed. */
+size_t ll_clip_backward_workspace_bytes(const ll_cache *cache, int n_frames);
+int ll_clip_attn_backward(ll_cache *cache, int layer, const ll_bf16 *q_roped, const ll_bf16 *out,
+                          const ll_bf16 *d_out, const float *lse, int64_t frame_start, int n_frames,
+                          int attn_window_frames, int grid_h, int grid_w, float rope_theta,
+                          ll_bf16 *dq, ll_bf16 *dk, ll_bf16 *dv, void *workspace, size_t workspace_bytes,
+                          ll_stream stream);
+
 /* KV-recache (Sec. 3.1; Sec. 3.3 last paragraph: only the most recent W frames
  * are rebuilt; the sink is left alone).  q, k, v hold fresh activations for the
  * resident window frames [r0, end), r0 = max(S, end - W), oldest first.

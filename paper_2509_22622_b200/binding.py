@@ -116,6 +116,10 @@ SIGNATURES = {
     "ll_clip_append_attn": (C.c_int, [C.c_void_p, C.c_int, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int64, C.c_int,
                                       C.c_int, C.c_int, C.c_int, C.c_float, C.c_void_p, C.c_void_p, C.c_void_p,
                                       C.c_void_p]),
+    "ll_clip_backward_workspace_bytes": (C.c_size_t, [C.c_void_p, C.c_int]),
+    "ll_clip_attn_backward": (C.c_int, [C.c_void_p, C.c_int, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int64, C.c_int,
+                                        C.c_int, C.c_int, C.c_int, C.c_float, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p,
+                                        C.c_size_t, C.c_void_p]),
     "ll_recache": (C.c_int, [C.c_void_p, C.c_int, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int, C.c_int,
                              C.c_int, C.c_float, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]),
     "ll_rope_q_static": (C.c_int, [C.c_void_p, C.c_void_p, C.c_int, C.c_int, C.c_int64, C.c_int, C.c_int, C.c_int,
@@ -278,6 +282,17 @@ def ll_clip_append_attn(h, layer, q, k, v, frame_start, n_frames, attn_window_fr
     _check(lib().ll_clip_append_attn(h, layer, _ptr(q), _ptr(k), _ptr(v), frame_start, n_frames, attn_window_frames,
                                      grid_h, grid_w, rope_theta, _ptr(q_out), _ptr(out), _ptr(lse_out),
                                      _stream(stream)))
+
+
+def ll_clip_backward_workspace_bytes(h, n_frames) -> int:
+    return lib().ll_clip_backward_workspace_bytes(h, n_frames)
+
+
+def ll_clip_attn_backward(h, layer, q_roped, out, d_out, lse, frame_start, n_frames, attn_window_frames, grid_h, grid_w,
+                          rope_theta, dq, dk, dv, workspace, stream=None):
+    _check(lib().ll_clip_attn_backward(h, layer, _ptr(q_roped), _ptr(out), _ptr(d_out), _ptr(lse), frame_start, n_frames,
+                                       attn_window_frames, grid_h, grid_w, rope_theta, _ptr(dq), _ptr(dk), _ptr(dv),
+                                       _ptr(workspace), workspace.numel() * workspace.element_size(), _stream(stream)))
 
 
 def ll_recache(h, layer, q, k, v, n_frames, grid_h, grid_w, rope_theta, q_out, out, lse_out=None, stream=None):

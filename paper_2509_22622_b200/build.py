@@ -9,7 +9,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libllattn.so")
-SOURCES = ["ll_host.cu", "rope_append.cu", "attn_sm100.cu", "attn_simt.cu", "rope_static.cu", "qkv_gemm.cu"]
+SOURCES = ["ll_host.cu", "rope_append.cu", "attn_sm100.cu", "attn_simt.cu", "rope_static.cu", "qkv_gemm.cu", "attn_bwd.cu"]
 HEADERS = ["ll_internal.h", "ptx.cuh", "bounded_wait.cuh", "rope_math.cuh", os.path.join(ROOT, "include", "llattn.h"),
            os.path.join(ROOT, "include", "llattn_debug.h")]
 

@@ -1042,6 +1042,100 @@ int ll_clip_append_attn(ll_cache *c, int layer, const ll_bf16 *q, const ll_bf16 
     return LL_OK;
 }
 
+size_t ll_clip_backward_workspace_bytes(const ll_cache *c, int n_frames)
+{
+    if (!c || n_frames <= 0) return 0;
+    return align_up((size_t)c->H * n_frames * c->P * sizeof(float), 256);
+}
+
+int ll_clip_attn_backward(ll_cache *c, int layer, const ll_bf16 *q_roped, const ll_bf16 *out, const ll_bf16 *d_out,
+                          const float *lse, int64_t frame_start, int n_frames, int attn_window_frames, int grid_h,
+                          int grid_w, float rope_theta, ll_bf16 *dq, ll_bf16 *dk, ll_bf16 *dv, void *workspace,
+                          size_t workspace_bytes, ll_stream stream)
+{
+    Range range("ll_clip_attn_backward", layer, (long long)frame_start);
+    if (!layer_ok(c, layer)) return fail(LL_ERR_INVALID_ARG, "bad cache handle or layer %d", layer);
+    if (grid_h <= 0 || grid_w <= 0 || (int64_t)grid_h * grid_w != c->P)
+        return fail(LL_ERR_INVALID_ARG, "grid %dx%d does not give %d tokens per frame", grid_h, grid_w, c->P);
+    if (!(rope_theta > 0.f)) return fail(LL_ERR_INVALID_ARG, "rope_theta must be positive");
+    if (c->kv_format != LL_KV_BF16) return fail(LL_ERR_UNSUPPORTED_SHAPE, "the backward pass is built for bf16 caches only");
+    if (n_frames <= 0 || n_frames % c->C)
+        return fail(LL_ERR_BAD_POSITION, "n_frames %d is not a positive multiple of chunk_frames %d", n_frames, c->C);
+    const int n_groups = n_frames / c->C;
+    if (n_groups > ll::kMaxGroups) return fail(LL_ERR_UNSUPPORTED_SHAPE, "more than %d chunks in a clip", ll::kMaxGroups);
+    if (attn_window_frames < c->C || attn_window_frames % c->C)
+        return fail(LL_ERR_INVALID_ARG, "attn_window_frames %d is not a positive multiple of chunk_frames", attn_window_frames);
+    if ((int64_t)attn_window_frames + n_frames - c->C > c->W)
+        return fail(LL_ERR_UNSUPPORTED_SHAPE, "the ring (%d frames) cannot have held this clip's windows", c->W);
+    ll::LayerState &st = c->layers[layer];
+    if (frame_start < 0 || frame_start + n_frames != st.end)
+        return fail(LL_ERR_BAD_POSITION, "the clip [%lld, %lld) is not the newest %d frames of the stream (end %lld)",
+                    (long long)frame_start, (long long)frame_start + n_frames, n_frames, (long long)st.end);
+    if ((int64_t)n_frames * c->P > INT32_MAX / 2) return fail(LL_ERR_UNSUPPORTED_SHAPE, "clip too long");
+    if (c->dry_run) return LL_OK;
+    if (!q_roped || !out || !d_out || !lse || !dq || !dk || !dv || !workspace)
+        return fail(LL_ERR_INVALID_ARG, "null tensor or workspace");
+    if (!aligned16(q_roped) || !aligned16(out) || !aligned16(d_out) || !aligned16(lse) || !aligned16(dq) || !aligned16(dk) ||
+        !aligned16(dv) || (reinterpret_cast<uintptr_t>(workspace) & 255u))
+        return fail(LL_ERR_INVALID_ARG, "pointers must be 16-byte aligned (workspace: 256)");
+    if (workspace_bytes < ll_clip_backward_workspace_bytes(c, n_frames))
+        return fail(LL_ERR_INVALID_ARG, "workspace smaller than ll_clip_backward_workspace_bytes");
+    int s = need_storage(c);
+    if (s != LL_OK) return s;
+    // the forward's query groups and key runs
+    AttnCall call{c, layer, q_roped, nullptr, nullptr, n_groups, {}, 0, {}};
+    for (int g = 0; g < n_groups; ++g) {
+        call.group_frame_start[g] = frame_start + (int64_t)g * c->C;
+        call.group_lo_floor[g] = call.group_frame_start[g] + c->C - attn_window_frames;
+    }
+    ll::AttnParams ap;
+    s = build_attn_params(&call, 1, &ap);
+    if (s != LL_OK) return s;
+    s = ensure_tables(c, frame_start, frame_start + n_frames, grid_h, grid_w, rope_theta, (cudaStream_t)stream);
+    if (s != LL_OK) return s;
+    ll::RopeAppendParams rp;
+    fill_rope_params(c, layer, nullptr, nullptr, nullptr, nullptr, frame_start, n_frames, grid_w, &rp);
+    ll::BwdParams p;
+    memset(&p, 0, sizeof p);
+    p.n_groups = n_groups; p.heads = c->H; p.head_dim = c->D; p.nq_total = n_frames * c->P;
+    p.scale = (float)(1.0 / std::sqrt((double)c->D));
+    p.scale_log2 = ap.scale_log2;
+    p.out = out; p.d_out = d_out; p.lse = lse; p.delta = static_cast<float *>(workspace);
+    p.dq = dq; p.dk = dk; p.dv = dv;
+    p.status = reinterpret_cast<uint32_t *>(c->storage + c->off_status);
+    p.P = c->P; p.grid_w = grid_w; p.n_t = rp.n_t; p.n_h = rp.n_h;
+    p.t_tab = rp.t_tab; p.h_tab = rp.h_tab; p.w_tab = rp.w_tab;
+    p.rows_per_head = c->rows;
+    for (int g = 0; g < n_groups; ++g) {
+        p.g[g] = ap.g[g];
+        p.n_qtiles += (ap.g[g].q_rows + 127) / 128;
+    }
+    // where the clip's frames sit: contiguous slots make runs of cache rows
+    for (int sl = 0; sl < LL_MAX_SLOTS; ++sl) p.slot_clip_frame[sl] = -1;
+    for (int i = 0; i < n_frames; ++i) p.slot_clip_frame[slot_of(c, frame_start + i)] = i;
+    for (int sl = 0; sl < c->n_slots;) {
+        if (p.slot_clip_frame[sl] < 0) { ++sl; continue; }
+        int e = sl;
+        while (e < c->n_slots && p.slot_clip_frame[e] >= 0) ++e;
+        if (p.n_kruns >= 4) return fail(LL_ERR_UNSUPPORTED_SHAPE, "the clip's frames sit in more than 4 runs of slots");
+        p.krun_start[p.n_kruns] = sl * c->P;
+        p.krun_len[p.n_kruns] = (e - sl) * c->P;
+        p.n_ktiles += (p.krun_len[p.n_kruns] + 127) / 128;
+        ++p.n_kruns;
+        sl = e;
+    }
+    ll::BwdMaps maps;
+    memset(&maps, 0, sizeof maps);
+    s = token_major_map(c, &maps.q, q_roped, (uint64_t)p.nq_total);
+    if (s == LL_OK) s = token_major_map(c, &maps.d_out, d_out, (uint64_t)p.nq_total);
+    if (s != LL_OK) return s;
+    maps.k = c->kmap[layer];
+    maps.v = c->vmap[layer];
+    cudaError_t e = ll::launch_attn_backward(p, maps, (cudaStream_t)stream);
+    if (e != cudaSuccess) return cuda_fail(e, "clip backward kernels");
+    return LL_OK;
+}
+
 namespace {
 void copy_plan(const ll::AttnParams &p, ll_attn_plan *out)
 {

@@ -162,6 +162,30 @@ struct QkvParams {
 cudaError_t launch_qkv_gemm(const QkvParams &p, const CUtensorMap &xmap, const CUtensorMap &wmap, int sm_count,
                             cudaStream_t stream);
 
+// Backward of the clip step (attn_bwd.cu): the forward's query groups and key runs, plus where
+// the clip's own rows sit in the cache.
+struct BwdParams {
+    int n_groups, heads, head_dim, nq_total;
+    float scale;                      // 1 / sqrt(D)
+    float scale_log2;                 // log2(e) / sqrt(D)
+    const ll_bf16 *out, *d_out;       // [nq_total, H, D]
+    const float *lse;                 // [H, nq_total], natural log (the forward's)
+    float *delta;                     // [H, nq_total] workspace: sum_d d_out * out
+    ll_bf16 *dq, *dk, *dv;            // [nq_total, H, D]
+    uint32_t *status;
+    int P, grid_w, n_t, n_h;
+    const float2 *t_tab, *h_tab, *w_tab;   // t_tab at the clip's first frame
+    int64_t rows_per_head;
+    int n_kruns;                      // runs of cache rows that hold the clip's frames
+    int krun_start[4], krun_len[4];
+    int n_ktiles;                     // 128-row tiles over those runs
+    int n_qtiles;                     // 128-row query tiles over all groups
+    int slot_clip_frame[LL_MAX_SLOTS];     // index of the clip frame a slot holds, -1: not the clip's
+    AttnGroup g[kMaxGroups];
+};
+struct BwdMaps { CUtensorMap q, d_out, k, v; };
+cudaError_t launch_attn_backward(const BwdParams &p, const BwdMaps &maps, cudaStream_t stream);
+
 // kernel launchers (each returns the cudaError of the launch)
 cudaError_t launch_rope_tables(float2 *t_tab, int64_t t_base, int n_t_frames, int n_t,
                                float2 *h_tab, int grid_h, float2 *w_tab, int grid_w, int n_hw,

@@ -504,15 +504,29 @@ def run_ours(args):
             big.rope_append_kv(0, None, k, v, chunk * C, wl.grid_h, wl.grid_w, wl.rope_theta)
         cq, ck, cv = (torch.cat([dev_sets[i % N_INPUT_SETS][j] for i in range(clip_chunks)]) for j in range(3))
         cq_out, c_out = torch.empty_like(cq), torch.empty_like(cq)
+        c_lse = torch.empty(H, T * P, device="cuda", dtype=torch.float32)
         pos = [n_fill * C]
 
         def clip():
             big.clip_append_attn(0, cq, ck, cv, pos[0], T, wl.window_frames, wl.grid_h, wl.grid_w, wl.rope_theta,
-                                 cq_out, c_out)
+                                 cq_out, c_out, c_lse)
             pos[0] += T
         ms = median_ms(clip)
         others["clip_21_frames"] = {"ms": ms, "tflops_attention_over_append_plus_attention":
                                     clip_chunks * attn_flops(wl) / ms / 1e9}
+        # backward of that clip (gradients for the clip's q, k, v; sink and context detached)
+        d_out = torch.randn_like(cq)
+        dq_g, dk_g, dv_g = (torch.empty_like(cq) for _ in range(3))
+        bws = torch.empty(B.ll_clip_backward_workspace_bytes(big.h, T) + 256, dtype=torch.uint8, device="cuda")
+        bws = bws[(-bws.data_ptr()) % 256:]
+        ms = median_ms(lambda: B.ll_clip_attn_backward(big.h, 0, cq_out, c_out, d_out, c_lse, pos[0] - T, T, wl.window_frames,
+                                                       wl.grid_h, wl.grid_w, wl.rope_theta, dq_g, dk_g, dv_g, bws), reps=5)
+        all_f = clip_chunks * (wl.sink_frames + wl.window_frames)
+        own_f = sum(min((g + 1) * C, wl.window_frames) for g in range(clip_chunks))
+        bwd_flops = 2.0 * nq * P * D * H * (3 * all_f + 2 * own_f)      # S, dP, dQ over all keys; dK, dV over the clip's
+        others["clip_21_frames_backward"] = {"ms": ms, "tflops_algorithmic": bwd_flops / ms / 1e9,
+                                             "note": "S and dP are formed twice (dq kernel and dk/dv kernel): 7 products "
+                                                     "run where 5 are counted"}
         big.check_device()
         big.close()
         gains = torch.ones(H * D, device="cuda")

@@ -104,3 +104,69 @@ def test_clip_backward_argument_checks():
     assert e.value.code == B.LL_ERR_INVALID_ARG
     cache.check_device()
     cache.close()
+
+
+def test_clip_backward_closed_forms_at_the_benchmark_shape(oracle_mod):
+    """Config-1 layer shape, a 21-frame clip behind 12 frames of context, K = 0: every weight is
+    1/n (n = 12 frames of keys), so the gradients have closed forms that need no oracle run:
+    dq = 0; dv is the same for all tokens of a frame, (1/n) * sum over the chunks that see the
+    frame of the chunk's summed d_out; dk_j = (1/(n sqrt(D))) sum_i (d_out_i.v_j - d_out_i.o_i) q_i
+    over the rows i that see j (checked on sampled key rows, in the rotated frame)."""
+    base = synth.CONFIGS[1]
+    C, P, H, D, S, Wa = base.chunk_frames, base.tokens_per_frame, base.heads, base.head_dim, base.sink_frames, base.window_frames
+    clip_chunks, ctx = 7, 4
+    T = clip_chunks * C
+    cache = B.Cache(1, H, D, P, C, S, Wa + T - C)
+    rng = np.random.default_rng(91)
+    zeros = torch.zeros(C * P, H, D, device="cuda", dtype=torch.bfloat16)
+    v_ctx = []
+    for chunk in range(ctx):
+        v = synth.normal_bf16(rng, (C * P, H, D))
+        v_ctx.append(F64(v))
+        cache.rope_append_kv(0, None, zeros, dev(v), chunk * C, base.grid_h, base.grid_w, base.rope_theta)
+    q = synth.normal_bf16(rng, (T * P, H, D))
+    v = synth.normal_bf16(rng, (T * P, H, D))
+    g = synth.normal_bf16(rng, (T * P, H, D))
+    dq_in, dv_in, dg = dev(q), dev(v), dev(g)
+    k0 = torch.zeros_like(dq_in)
+    q_out, out = torch.empty_like(dq_in), torch.empty_like(dq_in)
+    lse = torch.empty(H, T * P, device="cuda", dtype=torch.float32)
+    fs = ctx * C
+    cache.clip_append_attn(0, dq_in, k0, dv_in, fs, T, Wa, base.grid_h, base.grid_w, base.rope_theta, q_out, out, lse)
+    ws = torch.empty(B.ll_clip_backward_workspace_bytes(cache.h, T) + 256, dtype=torch.uint8, device="cuda")
+    ws = ws[(-ws.data_ptr()) % 256:]
+    dq, dk, dv = (torch.full_like(dq_in, float("nan")) for _ in range(3))
+    B.ll_clip_attn_backward(cache.h, 0, q_out, out, dg, lse, fs, T, Wa, base.grid_h, base.grid_w, base.rope_theta, dq, dk, dv, ws)
+    cache.check_device()
+    n = (S + Wa) * P
+    assert np.abs(lse.cpu().numpy() - np.log(n)).max() < 1e-3
+    assert float(dq.float().abs().max()) == 0.0
+    # frames (absolute) each clip chunk sees, and the d_out sums per chunk
+    gf, vf, qf = F64(g), F64(v), F64(q)
+    all_v = np.concatenate(v_ctx + [vf]).reshape(ctx * C + T, P, H, D)             # by absolute frame
+    chunk_sum = gf.reshape(clip_chunks, C * P, H, D).sum(axis=1)
+    sees = lambda c_, f: f < fs + (c_ + 1) * C and (f < S or f >= fs + (c_ + 1) * C - Wa)
+    got_dv = f64(dv).reshape(T, P, H, D)
+    for i in range(T):
+        want = sum(chunk_sum[c_] for c_ in range(clip_chunks) if sees(c_, fs + i)) / n
+        err = np.abs(got_dv[i] - want[None])
+        # one bf16 rounding of 1/n, one of the result, fp32 accumulation over up to 14040 rows
+        assert err.max() <= 2.0 ** -7 * np.abs(want).max() + 1e-6, (i, err.max())
+    # dk on sampled key rows, in the rotated frame: rotate the stored gradient forward again
+    o_bar = np.stack([sum(all_v[f].sum(axis=0) for f in range(ctx * C + T) if sees(c_, f)) / n for c_ in range(clip_chunks)])
+    q_rot = oracle_mod.rope(qf, fs, base.grid_h, base.grid_w, base.rope_theta)
+    dk_rot = oracle_mod.rope(f64(dk), fs, base.grid_h, base.grid_w, base.rope_theta)
+    for j in synth.sample_rows(T * P, 24, seed=3, edges=False):
+        fj = fs + j // P
+        want = np.zeros((H, D))
+        mag = np.zeros((H, D))
+        for c_ in range(clip_chunks):
+            if not sees(c_, fj):
+                continue
+            rows = slice(c_ * C * P, (c_ + 1) * C * P)
+            w = (np.einsum("ihd,hd->ih", gf[rows], vf[j]) - np.einsum("ihd,hd->ih", gf[rows], o_bar[c_])) / (n * np.sqrt(D))
+            want += np.einsum("ih,ihd->hd", w, q_rot[rows])
+            mag += np.einsum("ih,ihd->hd", np.abs(w), np.abs(q_rot[rows]))
+        err = np.abs(dk_rot[j] - want)
+        assert (err <= 2.0 ** -7 * mag + 2e-5).all(), (j, (err / (2.0 ** -7 * mag + 2e-5)).max())
+    cache.close()

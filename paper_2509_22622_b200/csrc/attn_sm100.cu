@@ -479,7 +479,6 @@ attn_sm100_kernel(const __grid_constant__ AttnParams p, const __grid_constant__ 
                     if (r < s.rows_valid) c_a *= __ldg(q_scale + s.q0 + r);
                     if (r + 8 < s.rows_valid) c_b *= __ldg(q_scale + s.q0 + r + 8);
                 }
-                const uint64_t c2a = pack2(c_a, c_a), c2b = pack2(c_b, c_b);
                 float m_a = -INFINITY, m_b = -INFINITY;
                 uint64_t acc_a = 0ull, acc_b = 0ull;       // two partial sums per row
                 for (int j = s.kt0; j < s.kt1; ++j, kit.next(), ++sc) {
@@ -508,6 +507,7 @@ attn_sm100_kernel(const __grid_constant__ AttnParams p, const __grid_constant__ 
                         uint64_t ts_a = 0ull, ts_b = 0ull;         // the piece's sums, two partials per row
                         {
                             const uint64_t na2 = pack2(-m_a, -m_a), nb2 = pack2(-m_b, -m_b);
+                            const uint64_t c2a = pack2(c_a, c_a), c2b = pack2(c_b, c_b);
                             const PolyRow ra{c_a * (1.f / 128.f), ((float)kPolyLow - m_a) * (1.f / 128.f)};
                             const PolyRow rb{c_b * (1.f / 128.f), ((float)kPolyLow - m_b) * (1.f / 128.f)};
                             // Four 8-key groups at a time, stage by stage, so that the exponentials of a
@@ -618,6 +618,7 @@ attn_sm100_kernel(const __grid_constant__ AttnParams p, const __grid_constant__ 
                             }
                             // the piece again, against the new references
                             const uint64_t na2 = pack2(-m_a, -m_a), nb2 = pack2(-m_b, -m_b);
+                            const uint64_t c2a = pack2(c_a, c_a), c2b = pack2(c_b, c_b);
                             ts_a = ts_b = 0ull;
 #pragma unroll
                             for (int k = 0; k < 8; ++k) {

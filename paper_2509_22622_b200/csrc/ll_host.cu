@@ -1319,7 +1319,8 @@ int ll_cache_device_status(ll_cache *c, ll_stream stream)
     e = cudaMemcpy(w, c->storage + c->off_status, sizeof w, cudaMemcpyDeviceToHost);
     if (e != cudaSuccess) return cuda_fail(e, "cudaMemcpy(status)");
     if (w[0] == ll::kStatusOk && c->debug) {
-        static unsigned char band[2 * kGuardBytes];
+        std::vector<unsigned char> band_buf(2 * kGuardBytes);
+        unsigned char *band = band_buf.data();
         e = cudaMemcpy(band, c->storage + c->off_guard0, kGuardBytes, cudaMemcpyDeviceToHost);
         if (e == cudaSuccess) e = cudaMemcpy(band + kGuardBytes, c->storage + c->off_guard1, kGuardBytes, cudaMemcpyDeviceToHost);
         if (e != cudaSuccess) return cuda_fail(e, "cudaMemcpy(guard bands)");

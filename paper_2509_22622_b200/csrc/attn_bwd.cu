@@ -11,9 +11,10 @@
 //
 // Two kernels instead of one with atomics: every gradient element is accumulated by one CTA in one
 // order, so the result is run-to-run deterministic, at the price of forming S and dP twice.  Both
-// kernels are plain: one warp loads (TMA) and issues the MMAs, four warps (one thread per tile row,
-// the 32x32b TMEM shape) turn S and dP into P and dS in shared memory; a tile pair's steps run one
-// after the other, with only the next operand load in flight.
+// kernels have one warp that loads (TMA) and issues the MMAs and eight compute warps that turn S
+// and dP into P and dS in shared memory (one thread per tile row and 64-key half, the 32x32b TMEM
+// shape).  The dq kernel forms S and dP in two 64-key halves, each with its own warp group, so that
+// the tensor pipe works on one half while the other is in the exponentials.
 #include <cuda_bf16.h>
 
 #include "bounded_wait.cuh"
@@ -26,7 +27,8 @@ namespace {
 
 using namespace ptx;
 
-constexpr int kBwdThreads = 160;                       // four compute warps, one load/issue warp
+constexpr int kBwdThreads = 288;                       // eight compute warps, one load/issue warp
+constexpr int kIssueWarp = 8;
 constexpr int kTile = 128;
 
 __device__ __forceinline__ float as_f(uint32_t u) { return __uint_as_float(u); }
@@ -39,13 +41,20 @@ __device__ __forceinline__ void tmem_ld_32x32b_x32(uint32_t taddr, uint32_t *r)
                  : "memory");
 }
 
+__device__ __forceinline__ void tmem_st_32x32b_x32(uint32_t taddr, const uint32_t *r)
+{
+    asm volatile("tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31, %32};"
+                 ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]), "r"(r[8]), "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15]), "r"(r[16]), "r"(r[17]), "r"(r[18]), "r"(r[19]), "r"(r[20]), "r"(r[21]), "r"(r[22]), "r"(r[23]), "r"(r[24]), "r"(r[25]), "r"(r[26]), "r"(r[27]), "r"(r[28]), "r"(r[29]), "r"(r[30]), "r"(r[31])
+                 : "memory");
+}
+
 __device__ __forceinline__ void st_shared_v4(uint32_t addr, uint32_t a, uint32_t b, uint32_t c, uint32_t d)
 {
     asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(a), "r"(b), "r"(c), "r"(d) : "memory");
 }
 
-// Meeting point of the four compute warps (hardware barrier 1; 0 is __syncthreads).
-__device__ __forceinline__ void compute_sync() { asm volatile("barrier.sync 1, 128;" ::: "memory"); }
+// Meeting point of the eight compute warps (hardware barrier 0 is __syncthreads).
+__device__ __forceinline__ void compute_sync() { asm volatile("barrier.sync 1, 256;" ::: "memory"); }
 
 // delta[h][i] = sum_d d_out[i][h][d] * out[i][h][d]: one warp per (row, head).
 template <int D>
@@ -69,28 +78,43 @@ __global__ void __launch_bounds__(256) bwd_delta_kernel(const __grid_constant__ 
     if (lane == 0) p.delta[(size_t)head * p.nq_total + row] = s;
 }
 
-// One row of a 128 x 128 score tile and of the matching dP tile (TMEM, fp32) to P and/or dS
+// One row of one 64-key half of a 128 x 128 score tile and of the matching dP tile (TMEM, fp32) to P and/or dS
 // (bf16) in 128-byte-swizzled shared-memory tiles laid out [row][key]: two 64-key atoms of
 // 128 rows x 128 bytes, row r's 16-byte chunk k at chunk position k ^ (r % 8).
-//   p = 2^(s * c - lse2), ds = p * (dp - delta); columns whose bit in `valid` is clear, and rows
-//   that are not live, give zeros.
-__device__ __forceinline__ void row_to_p_ds(uint32_t t_s, uint32_t t_dp, int row, bool live, float c, float lse2,
+//   p = 2^(s * c - lse2), ds = p * (dp - delta); columns whose bit in `valid` is clear give
+//   zeros (a row that is not live passes lse2 = +inf, which makes its p zero).  The arithmetic
+//   runs on packed pairs; the per-column mask is only applied to chunks that are not all valid.
+__device__ __forceinline__ void row_to_p_ds(uint32_t t_s, uint32_t t_dp, int row, int half, float c, float lse2,
                                             float delta, const uint32_t (&valid)[4], uint32_t p_tile, uint32_t ds_tile)
 {
+    const uint64_t c2 = pack2(c, c), nl2 = pack2(-lse2, -lse2), nd2 = pack2(-delta, -delta);
 #pragma unroll 1
-    for (int ch = 0; ch < 4; ++ch) {
+    for (int ch = 2 * half; ch < 2 * half + 2; ++ch) {
         uint32_t s[32], dp[32];
         tmem_ld_32x32b_x32(t_s + 32 * ch, s);
         tmem_ld_32x32b_x32(t_dp + 32 * ch, dp);
         tmem_wait_ld();
+        const uint32_t vbits = ch == 0 ? valid[0] : ch == 1 ? valid[1] : ch == 2 ? valid[2] : valid[3];
         uint32_t pw[16], dw[16];
+        if (vbits == 0xffffffffu) {
 #pragma unroll
-        for (int i = 0; i < 16; ++i) {
-            float p0 = ex2(fmaf(as_f(s[2 * i]), c, -lse2)), p1 = ex2(fmaf(as_f(s[2 * i + 1]), c, -lse2));
-            if (!live || !((valid[ch] >> (2 * i)) & 1u)) p0 = 0.f;
-            if (!live || !((valid[ch] >> (2 * i + 1)) & 1u)) p1 = 0.f;
-            pw[i] = cvt_bf16x2(p0, p1);
-            dw[i] = cvt_bf16x2(p0 * (as_f(dp[2 * i]) - delta), p1 * (as_f(dp[2 * i + 1]) - delta));
+            for (int i = 0; i < 16; ++i) {
+                float e0, e1, d0, d1;
+                unpack2(fma2(pack2(as_f(s[2 * i]), as_f(s[2 * i + 1])), c2, nl2), e0, e1);
+                const float p0 = ex2(e0), p1 = ex2(e1);
+                pw[i] = cvt_bf16x2(p0, p1);
+                unpack2(mul2(pack2(p0, p1), add2(pack2(as_f(dp[2 * i]), as_f(dp[2 * i + 1])), nd2)), d0, d1);
+                dw[i] = cvt_bf16x2(d0, d1);
+            }
+        } else {
+#pragma unroll
+            for (int i = 0; i < 16; ++i) {
+                float p0 = ex2(fmaf(as_f(s[2 * i]), c, -lse2)), p1 = ex2(fmaf(as_f(s[2 * i + 1]), c, -lse2));
+                if (!((vbits >> (2 * i)) & 1u)) p0 = 0.f;
+                if (!((vbits >> (2 * i + 1)) & 1u)) p1 = 0.f;
+                pw[i] = cvt_bf16x2(p0, p1);
+                dw[i] = cvt_bf16x2(p0 * (as_f(dp[2 * i]) - delta), p1 * (as_f(dp[2 * i + 1]) - delta));
+            }
         }
         // 32 keys = four 16-byte chunks of this row, in atom ch / 2
         const uint32_t row_off = (uint32_t)(ch >> 1) * (128 * 128) + (uint32_t)row * 128;
@@ -103,16 +127,18 @@ __device__ __forceinline__ void row_to_p_ds(uint32_t t_s, uint32_t t_dp, int row
     }
 }
 
-// 128 rows x D fp32 in TMEM (row = thread), times `mul`, optionally turned back through the
-// rotation of the row's grid position, rounded to bf16 and stored at dst (one head row of D).
+// Half `half` of the D columns of 128 rows x D fp32 in TMEM (row = thread), times `mul`,
+// optionally turned back through the rotation of the row's grid position, rounded to bf16 and
+// stored at dst (one head row of D).
 template <int D, bool kRotateBack>
 __device__ __forceinline__ void store_grad_row(uint32_t taddr, float mul, ll_bf16 *dst, const BwdParams &p, int frame,
-                                               int y, int x, bool live)
+                                               int y, int x, bool live, int half)
 {
     constexpr int kNh = D / 6, kNt = D / 2 - 2 * kNh;
     const float2 *t_row = p.t_tab + (size_t)frame * kNt, *h_row = p.h_tab + (size_t)y * kNh, *w_row = p.w_tab + (size_t)x * kNh;
 #pragma unroll
-    for (int ch = 0; ch < D / 32; ++ch) {
+    for (int c = 0; c < D / 64; ++c) {
+        const int ch = half * (D / 64) + c;
         uint32_t r[32];
         tmem_ld_32x32b_x32(taddr + 32 * ch, r);
         tmem_wait_ld();
@@ -159,19 +185,26 @@ struct BwdCfg {
     static constexpr int kPBytes = 2 * kAtomBytes;               // 128 rows x 128 keys bf16
 };
 
-// MMA helpers: all tiles are 128-byte-swizzled, 128 rows, tile base 1024-byte aligned.
-// K-major operand [rows][64-element atoms]: slice kk (16 elements) of the contraction.
-__device__ __forceinline__ uint64_t desc_kmajor(uint32_t tile, int kk)
+// MMA helpers: all tiles are 128-byte-swizzled, 128 rows, tile base 1024-byte aligned.  The low
+// descriptor word of a tile is formed once; a slice of the contraction adds a constant to it.
+//   K-major operand [rows][64-element atoms]: slice kk = 16 elements of the contraction.
+//   MN-major operand: the tile's rows are the contraction index, its columns the M (or N) index;
+//   slice kk = rows 16 kk .. 16 kk + 15.
+__device__ __forceinline__ uint32_t lo_kmajor(uint32_t tile) { return smem_desc_lo(tile, 16); }
+__device__ __forceinline__ uint32_t lo_mnmajor(uint32_t tile) { return smem_desc_lo(tile, 128 * 128); }
+__host__ __device__ constexpr uint32_t slice_kmajor(int kk) { return (uint32_t)(((kk / 4) * (128 * 128) + (kk % 4) * 32) >> 4); }
+__host__ __device__ constexpr uint32_t slice_mnmajor(int kk) { return (uint32_t)((kk * 2048) >> 4); }
+
+// Slices kBegin .. kEnd - 1 of D (+)= A B; kAMn / kBMn say which operand is MN-major.  The first
+// slice accumulates iff `acc_first`.
+template <int kBegin, int kEnd, bool kAMn, bool kBMn>
+__device__ __forceinline__ void mma_slices(uint32_t d, uint32_t a_lo, uint32_t b_lo, uint32_t idesc, uint32_t acc_first)
 {
     constexpr uint32_t hi = smem_desc_hi_sw128(1024);
-    return smem_desc_join(smem_desc_lo(tile, 16) + (uint32_t)(((kk / 4) * (128 * 128) + (kk % 4) * 32) >> 4), hi);
-}
-// MN-major operand: the tile's rows are the contraction index, its columns the M (or N) index;
-// slice kk = rows 16 kk .. 16 kk + 15.
-__device__ __forceinline__ uint64_t desc_mnmajor(uint32_t tile, int kk)
-{
-    constexpr uint32_t hi = smem_desc_hi_sw128(1024);
-    return smem_desc_join(smem_desc_lo(tile, 128 * 128) + (uint32_t)((kk * 2048) >> 4), hi);
+#pragma unroll
+    for (int kk = kBegin; kk < kEnd; ++kk)
+        mma_ss(d, smem_desc_join(a_lo + (kAMn ? slice_mnmajor(kk) : slice_kmajor(kk)), hi),
+               smem_desc_join(b_lo + (kBMn ? slice_mnmajor(kk) : slice_kmajor(kk)), hi), idesc, kk > kBegin ? 1u : acc_first);
 }
 
 __device__ __forceinline__ void key_mask(int nvalid, uint32_t (&valid)[4])
@@ -181,18 +214,75 @@ __device__ __forceinline__ void key_mask(int nvalid, uint32_t (&valid)[4])
         valid[ch] = nvalid >= 32 * (ch + 1) ? 0xffffffffu : nvalid > 32 * ch ? ((1u << (nvalid - 32 * ch)) - 1u) : 0u;
 }
 
+// This thread's 64 columns of a score row (fp32 words in s) to the weights p = 2^(s c - lse2),
+// in place; columns whose bit in vlo (first 32) / vhi is clear give zero.
+__device__ __forceinline__ void scores_to_weights(uint32_t (&s)[64], float c, float lse2, uint32_t vlo, uint32_t vhi)
+{
+    const uint64_t c2 = pack2(c, c), nl2 = pack2(-lse2, -lse2);
+#pragma unroll
+    for (int i = 0; i < 32; ++i) {
+        float e0, e1;
+        unpack2(fma2(pack2(as_f(s[2 * i]), as_f(s[2 * i + 1])), c2, nl2), e0, e1);
+        s[2 * i] = __float_as_uint(ex2(e0));
+        s[2 * i + 1] = __float_as_uint(ex2(e1));
+    }
+    if ((vlo & vhi) != 0xffffffffu) {
+#pragma unroll
+        for (int i = 0; i < 64; ++i)
+            if (!(((i < 32 ? vlo : vhi) >> (i & 31)) & 1u)) s[i] = 0u;
+    }
+}
+
+// dS = p (dP - delta) of this thread's 64 columns (32-column chunks ch0, ch0 + 1 of tile row
+// `row`), rounded to bf16, into the swizzled [row][key] tile.
+__device__ __forceinline__ void store_ds(const uint32_t (&pw)[64], uint32_t t_dp, int row, int ch0, float delta, uint32_t ds_tile)
+{
+    const uint64_t nd2 = pack2(-delta, -delta);
+#pragma unroll
+    for (int h = 0; h < 2; ++h) {
+        const int ch = ch0 + h;
+        uint32_t dp[32];
+        tmem_ld_32x32b_x32(t_dp + 32 * ch, dp);
+        tmem_wait_ld();
+        uint32_t dw[16];
+#pragma unroll
+        for (int i = 0; i < 16; ++i) {
+            float d0, d1;
+            unpack2(mul2(pack2(as_f(pw[32 * h + 2 * i]), as_f(pw[32 * h + 2 * i + 1])),
+                         add2(pack2(as_f(dp[2 * i]), as_f(dp[2 * i + 1])), nd2)), d0, d1);
+            dw[i] = cvt_bf16x2(d0, d1);
+        }
+        const uint32_t row_off = (uint32_t)(ch >> 1) * (128 * 128) + (uint32_t)row * 128;
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+            const uint32_t chunk = (uint32_t)(((ch & 1) * 4 + k) ^ (row & 7)) << 4;
+            st_shared_v4(ds_tile + row_off + chunk, dw[4 * k], dw[4 * k + 1], dw[4 * k + 2], dw[4 * k + 3]);
+        }
+    }
+}
+
 // ---- dq: one CTA per (128-row query tile, head) ---------------------------------------------
+// The tile's Q and dO rows are the stationary A operands of S = Q K^T and dP = dO V^T: they are
+// written once into tensor memory (bf16, two elements per column), so those products read only
+// K and V from shared memory.  Eight compute warps share a step (thread = tile row x 64-key
+// half).  Per 128-key step j the tensor pipe runs S(j+1) | dQ(j-1) | dP(j) ...: the compute warps
+// take S(j) into registers and release it at once, so S(j+1) is formed while they are in the
+// exponentials; dP(j) is only needed for the last multiply, dS = P (dP - delta), after which
+// dQ(j) and dP(j+1) are issued.  K and V tiles sit in three stages; K is needed until the
+// step's dQ product, V only until its dP.
+//   tensor memory columns: S 0..127, dP 128..255, dQ 256..256+D-1, Q 384.., dO 448..
 template <int D>
 __global__ void __launch_bounds__(kBwdThreads, 1)
 bwd_dq_kernel(const __grid_constant__ BwdParams p, const __grid_constant__ BwdMaps maps)
 {
     using C = BwdCfg<D>;
+    constexpr int kStages = 3;
     extern __shared__ uint8_t smem_raw[];
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     uint8_t *gen = smem_raw + (base - smem_u32(smem_raw));
-    const uint32_t q_s = base, do_s = q_s + C::kTileBytes, k_s = do_s + C::kTileBytes, v_s = k_s + 2 * C::kTileBytes,
-                   ds_s = v_s + 2 * C::kTileBytes, bars = ds_s + C::kPBytes;
-    enum { kQFull = 0, kKvFull = 1, kKvEmpty = 3, kSFull = 5, kDsFull = 6, kDone = 7, kBars = 8 };
+    const uint32_t k_s = base, v_s = k_s + kStages * C::kTileBytes, ds_s = v_s + kStages * C::kTileBytes, bars = ds_s + C::kPBytes;
+    enum { kKFull = 0, kVFull = 3, kKEmpty = 6, kVEmpty = 9, kSFull = 12, kSFree = 13, kDpFull = 14, kDsFull = 15, kDone = 16, kBars = 17 };
+    constexpr int kComputeWarps = 8;
     uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(gen + (bars - base) + kBars * 8);
     volatile int *abort_flag = reinterpret_cast<volatile int *>(tmem_slot + 1);
     auto bar = [&](int i) -> uint32_t { return bars + 8u * (uint32_t)i; };
@@ -206,11 +296,11 @@ bwd_dq_kernel(const __grid_constant__ BwdParams p, const __grid_constant__ BwdMa
     const int n_kt = G.n_kt;
 
     if (threadIdx.x == 0) {
-        for (int i = 0; i < kBars; ++i) mbar_init(bar(i), 1);
+        for (int i = 0; i < kBars; ++i) mbar_init(bar(i), (i == kSFree || i == kDsFull) ? kComputeWarps : 1);
         *abort_flag = (*reinterpret_cast<volatile uint32_t *>(p.status) != kStatusOk) ? 2 : 0;
         fence_mbar_init();
     }
-    if (warp == 4) { tmem_alloc(smem_u32(tmem_slot), 512); tmem_relinquish(); }
+    if (warp == kIssueWarp) { tmem_alloc(smem_u32(tmem_slot), 512); tmem_relinquish(); }
     tc_fence_before_sync();
     __syncthreads();
     tc_fence_after_sync();
@@ -218,71 +308,140 @@ bwd_dq_kernel(const __grid_constant__ BwdParams p, const __grid_constant__ BwdMa
     WaitCtx ctx{abort_flag, p.status, warp};
     auto wait = [&](int bar_id, uint32_t parity, int iter) -> bool { return wait_bar(bar(bar_id), parity & 1u, ctx, bar_id, iter); };
     const bool skip = *abort_flag != 0;
-    const uint32_t t_s = tmem, t_dp = tmem + 128, t_dq = tmem + 256;
+    const uint32_t t_s = tmem, t_dp = tmem + 128, t_dq = tmem + 256, t_q = tmem + 384, t_do = tmem + 448;
+
+    // the tile's Q rows (warps 0-3) and dO rows (warps 4-7) into tensor memory; rows past the
+    // group's end become zeros
+    if (!skip && warp != kIssueWarp) {
+        const int row = threadIdx.x & 127, half = threadIdx.x >> 7;
+        const bool live = row < rows;
+        const uint4 *src = reinterpret_cast<const uint4 *>((half ? p.d_out : p.q) + ((size_t)(q0 + (live ? row : 0)) * p.heads + head) * D);
+        const uint32_t dst = (half ? t_do : t_q) + ((uint32_t)(32 * (warp & 3)) << 16);
+#pragma unroll
+        for (int c = 0; c < D / 64; ++c) {
+            uint32_t w[32];
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+                const uint4 u = live ? __ldg(src + 8 * c + i) : make_uint4(0u, 0u, 0u, 0u);
+                w[4 * i] = u.x; w[4 * i + 1] = u.y; w[4 * i + 2] = u.z; w[4 * i + 3] = u.w;
+            }
+            tmem_st_32x32b_x32(dst + 32 * c, w);
+        }
+        tmem_wait_st();
+    }
+    tc_fence_before_sync();
+    __syncthreads();
+    tc_fence_after_sync();
 
     if (skip) {
-    } else if (warp == 4) {
-        if (lane == 0) [&]() {
+    } else if (warp == kIssueWarp) {
+        // All 32 lanes walk the loop and the waits, so that addresses and descriptors are
+        // warp-uniform values; one elected lane issues the copies, the MMAs and the commits.
+        [&]() {
+            const bool elected = elect_one();
             constexpr uint32_t idesc_s = idesc_bf16_f32(128, 128, 0, 0), idesc_dq = idesc_bf16_f32(128, D, 0, 1);
-            auto load_kv = [&](int j, int row) {
-                const int b = j & 1;
-                mbar_arrive_expect_tx(bar(kKvFull + b), 2 * C::kTileBytes);
-                for (int a = 0; a < D / 64; ++a) {
-                    tma_load_3d(k_s + b * C::kTileBytes + a * C::kAtomBytes, &maps.k, bar(kKvFull + b), a * 64, row, head);
-                    tma_load_3d(v_s + b * C::kTileBytes + a * C::kAtomBytes, &maps.v, bar(kKvFull + b), a * 64, row, head);
+            constexpr uint32_t hi = smem_desc_hi_sw128(1024);
+            RunTiles kt(&G);                                     // walks ahead of the products: tile of the next load
+            int loaded = 0;
+            auto load_kv = [&]() {                               // K and V tiles of step `loaded`
+                const int st = loaded % kStages, row = kt.row();
+                if (elected) {
+                    mbar_arrive_expect_tx(bar(kKFull + st), C::kTileBytes);
+                    for (int a = 0; a < D / 64; ++a)
+                        tma_load_3d(k_s + st * C::kTileBytes + a * C::kAtomBytes, &maps.k, bar(kKFull + st), a * 64, row, head);
+                    mbar_arrive_expect_tx(bar(kVFull + st), C::kTileBytes);
+                    for (int a = 0; a < D / 64; ++a)
+                        tma_load_3d(v_s + st * C::kTileBytes + a * C::kAtomBytes, &maps.v, bar(kVFull + st), a * 64, row, head);
                 }
+                __syncwarp();
+                ++loaded;
+                kt.next();
             };
-            mbar_arrive_expect_tx(bar(kQFull), 2 * C::kTileBytes);
-            for (int a = 0; a < D / 64; ++a) {
-                tma_load_3d(q_s + a * C::kAtomBytes, &maps.q, bar(kQFull), a * 64, head, q0);
-                tma_load_3d(do_s + a * C::kAtomBytes, &maps.d_out, bar(kQFull), a * 64, head, q0);
-            }
-            RunTiles kt(&G);
-            load_kv(0, kt.row());
-            if (!wait(kQFull, 0, 0)) return;
-            for (int j = 0; j < n_kt; ++j) {
-                const int b = j & 1;
-                if (j + 1 < n_kt) {
-                    kt.next();
-                    if (j + 1 >= 2 && !wait(kKvEmpty + ((j + 1) & 1), ((j + 1) >> 1) - 1, j)) return;
-                    load_kv(j + 1, kt.row());
+            auto commit = [&](int bar_id) { if (elected) tc_commit(bar(bar_id)); };
+            const uint32_t k_lo = lo_kmajor(k_s), v_lo = lo_kmajor(v_s), ds_lo = lo_kmajor(ds_s);
+            auto issue_s = [&](int j) -> bool {                  // S(j) = Q K(j)^T
+                const int st = j % kStages;
+                if (!wait(kKFull + st, j / kStages, j)) return false;
+                tc_fence_after_sync();
+                const uint32_t b_lo = k_lo + ((uint32_t)(st * C::kTileBytes) >> 4);
+                if (elected) {
+#pragma unroll
+                    for (int kk = 0; kk < D / 16; ++kk)
+                        mma_ts(t_s, t_q + 8 * kk, smem_desc_join(b_lo + slice_kmajor(kk), hi), idesc_s, kk > 0);
                 }
-                if (!wait(kKvFull + b, j >> 1, j)) return;
+                __syncwarp();
+                commit(kSFull);
+                return true;
+            };
+            auto issue_dp = [&](int j) -> bool {                 // dP(j) = dO V(j)^T
+                const int st = j % kStages;
+                if (!wait(kVFull + st, j / kStages, j)) return false;
                 tc_fence_after_sync();
-                for (int kk = 0; kk < D / 16; ++kk)
-                    mma_ss(t_s, desc_kmajor(q_s, kk), desc_kmajor(k_s + b * C::kTileBytes, kk), idesc_s, kk > 0);
-                for (int kk = 0; kk < D / 16; ++kk)
-                    mma_ss(t_dp, desc_kmajor(do_s, kk), desc_kmajor(v_s + b * C::kTileBytes, kk), idesc_s, kk > 0);
-                tc_commit(bar(kSFull));
-                if (!wait(kDsFull, j, j)) return;
+                const uint32_t b_lo = v_lo + ((uint32_t)(st * C::kTileBytes) >> 4);
+                if (elected) {
+#pragma unroll
+                    for (int kk = 0; kk < D / 16; ++kk)
+                        mma_ts(t_dp, t_do + 8 * kk, smem_desc_join(b_lo + slice_kmajor(kk), hi), idesc_s, kk > 0);
+                }
+                __syncwarp();
+                commit(kDpFull);
+                commit(kVEmpty + st);
+                return true;
+            };
+            for (int i = 0; i < kStages && i < n_kt; ++i) load_kv();
+            if (!issue_s(0) || !issue_dp(0)) return;
+            for (int j = 0; j < n_kt; ++j) {
+                const int st = j % kStages;
+                if (j >= 1 && j + 2 < n_kt) {                    // the stage step j - 1 used takes step j + 2
+                    const int free_st = (j - 1) % kStages;
+                    if (!wait(kVEmpty + free_st, (j - 1) / kStages, j) || !wait(kKEmpty + free_st, (j - 1) / kStages, j)) return;
+                    load_kv();
+                }
+                if (j + 1 < n_kt) {
+                    if (!wait(kSFree, j, j)) return;             // S(j) is in the compute warps' registers
+                    if (!issue_s(j + 1)) return;
+                }
+                if (!wait(kDsFull, j, j)) return;                // dS(j) is in shared memory, dP(j) has been read
                 tc_fence_after_sync();
-                for (int kk = 0; kk < kTile / 16; ++kk)
-                    mma_ss(t_dq, desc_kmajor(ds_s, kk), desc_mnmajor(k_s + b * C::kTileBytes, kk), idesc_dq, (j > 0 || kk > 0) ? 1u : 0u);
-                tc_commit(bar(kKvEmpty + b));
+                const uint32_t k_mn = lo_mnmajor(k_s + st * C::kTileBytes);
+                if (elected) mma_slices<0, 8, false, true>(t_dq, ds_lo, k_mn, idesc_dq, j > 0 ? 1u : 0u);
+                __syncwarp();
+                commit(kKEmpty + st);
+                if (j + 1 < n_kt && !issue_dp(j + 1)) return;
             }
-            tc_commit(bar(kDone));
+            commit(kDone);
         }();
     } else {
         bool alive = true;
         auto wait_c = [&](int bar_id, uint32_t parity, int iter) {
             if (alive && !__all_sync(0xffffffffu, wait(bar_id, parity, iter))) alive = false;
         };
-        const int row = threadIdx.x;                             // tile row = TMEM lane
+        const int row = threadIdx.x & 127, half = threadIdx.x >> 7;      // tile row = TMEM lane; 64-key half
         const bool live = row < rows;
-        const uint32_t lane_off = (uint32_t)(32 * warp) << 16;
+        const uint32_t lane_off = (uint32_t)(32 * (warp & 3)) << 16;
         const size_t stat = (size_t)head * p.nq_total + q0 + (live ? row : 0);
-        const float lse2 = p.lse[stat] * 1.4426950408889634f, delta = p.delta[stat];
+        const float lse2 = live ? p.lse[stat] * 1.4426950408889634f : INFINITY, delta = p.delta[stat];
         RunTiles kt(&G);
         for (int j = 0; j < n_kt; ++j, kt.next()) {
             uint32_t valid[4];
             key_mask(kt.valid(), valid);
             wait_c(kSFull, j, j);
             tc_fence_after_sync();
-            row_to_p_ds(t_s + lane_off, t_dp + lane_off, row, live, p.scale_log2, lse2, delta, valid, 0u, ds_s);
+            uint32_t w[64];
+            tmem_ld_32x32b_x32(t_s + lane_off + 64 * half, w);
+            tmem_ld_32x32b_x32(t_s + lane_off + 64 * half + 32, w + 32);
+            tmem_wait_ld();
+            tc_fence_before_sync();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar(kSFree));
+            scores_to_weights(w, p.scale_log2, lse2, half ? valid[2] : valid[0], half ? valid[3] : valid[1]);
+            wait_c(kDpFull, j, j);
+            tc_fence_after_sync();
+            store_ds(w, t_dp + lane_off, row, 2 * half, delta, ds_s);
             fence_proxy_async_smem();
             tc_fence_before_sync();
-            compute_sync();
-            if (threadIdx.x == 0) mbar_arrive(bar(kDsFull));
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar(kDsFull));
         }
         wait_c(kDone, 0, n_kt);
         tc_fence_after_sync();
@@ -290,7 +449,7 @@ bwd_dq_kernel(const __grid_constant__ BwdParams p, const __grid_constant__ BwdMa
         const int frame = token / p.P, cell = token % p.P;
         if (alive)
             store_grad_row<D, true>(t_dq + lane_off, p.scale, p.dq + ((size_t)token * p.heads + head) * D, p, frame,
-                                    cell / p.grid_w, cell % p.grid_w, live);
+                                    cell / p.grid_w, cell % p.grid_w, live, half);
     }
     tc_fence_before_sync();
     __syncthreads();
@@ -299,7 +458,7 @@ bwd_dq_kernel(const __grid_constant__ BwdParams p, const __grid_constant__ BwdMa
         while (globaltimer_ns() - t0 < 200000ull) __nanosleep(1000);
         __syncthreads();
     }
-    if (warp == 4) { __syncwarp(); tc_fence_after_sync(); tmem_dealloc(tmem, 512); }
+    if (warp == kIssueWarp) { __syncwarp(); tc_fence_after_sync(); tmem_dealloc(tmem, 512); }
 }
 
 
@@ -310,13 +469,43 @@ __device__ __forceinline__ bool group_mask(const AttnGroup &G, int r0, uint32_t 
     bool any = false;
     for (int r = 0; r < G.n_ranges; ++r) {
         const int lo = max(G.k_start[r], r0) - r0, hi = min(G.k_start[r] + G.k_len[r], r0 + kTile) - r0;
-        for (int c = lo; c < hi; ++c) valid[c >> 5] |= 1u << (c & 31);
+#pragma unroll
+        for (int w = 0; w < 4; ++w) {
+            const int a = min(max(lo - 32 * w, 0), 32), b = min(max(hi - 32 * w, 0), 32);
+            if (b > a) valid[w] |= (b == 32 ? 0xffffffffu : (1u << b) - 1u) & ~((1u << a) - 1u);
+        }
         any |= hi > lo;
     }
     return any;
 }
 
+// Whether any of the 128 cache rows starting at r0 is visible to the group.
+__device__ __forceinline__ bool group_sees(const AttnGroup &G, int r0)
+{
+    bool any = false;
+    for (int r = 0; r < G.n_ranges; ++r)
+        any |= min(G.k_start[r] + G.k_len[r], r0 + kTile) > max(G.k_start[r], r0);
+    return any;
+}
+
+// The (group, 128-row query tile) pairs a key tile takes part in, in order.
+struct QTiles {
+    const BwdParams &p;
+    int r0, g, i;
+    __device__ QTiles(const BwdParams &params, int first_row) : p(params), r0(first_row), g(0), i(-1) { next(); }
+    __device__ bool done() const { return g >= p.n_groups; }
+    __device__ int q_row() const { return p.g[g].q_begin + i * kTile; }
+    __device__ void next()
+    {
+        ++i;
+        while (g < p.n_groups && !(i * kTile < p.g[g].q_rows && group_sees(p.g[g], r0))) { ++g; i = 0; }
+    }
+};
+
 // ---- dk, dv: one CTA per (128-row tile of the clip's cache rows, head) -----------------------
+// K and V of the tile stay in shared memory; per step one query tile's Q and dO come in.  The
+// step's last products are issued dK (reads dS, Q) then dV (reads P, dO), each with a barrier of
+// its own, so the next Q is under way while dV runs and the next S can start before dO is in.
 template <int D>
 __global__ void __launch_bounds__(kBwdThreads, 1)
 bwd_dkdv_kernel(const __grid_constant__ BwdParams p, const __grid_constant__ BwdMaps maps)
@@ -327,11 +516,11 @@ bwd_dkdv_kernel(const __grid_constant__ BwdParams p, const __grid_constant__ Bwd
     uint8_t *gen = smem_raw + (base - smem_u32(smem_raw));
     const uint32_t k_s = base, v_s = k_s + C::kTileBytes, q_s = v_s + C::kTileBytes, do_s = q_s + C::kTileBytes,
                    p_s = do_s + C::kTileBytes, ds_s = p_s + C::kPBytes, bars = ds_s + C::kPBytes;
-    enum { kKvFull = 0, kQdFull = 1, kSFull = 2, kPdsFull = 3, kStepDone = 4, kBars = 5 };
+    enum { kKvFull = 0, kQFull = 1, kDoFull = 2, kSFull = 3, kPdsFull = 4, kQFree = 5, kStepDone = 6, kBars = 7 };
     uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(gen + (bars - base) + kBars * 8);
     volatile int *abort_flag = reinterpret_cast<volatile int *>(tmem_slot + 1);
     auto bar = [&](int i) -> uint32_t { return bars + 8u * (uint32_t)i; };
-    const int warp = __shfl_sync(0xffffffffu, (int)(threadIdx.x >> 5), 0), lane = threadIdx.x & 31;
+    const int warp = __shfl_sync(0xffffffffu, (int)(threadIdx.x >> 5), 0);
     const int head = blockIdx.y;
     // the tile's first cache row and the end of the run it belongs to
     int run = 0, t = blockIdx.x;
@@ -343,7 +532,7 @@ bwd_dkdv_kernel(const __grid_constant__ BwdParams p, const __grid_constant__ Bwd
         *abort_flag = (*reinterpret_cast<volatile uint32_t *>(p.status) != kStatusOk) ? 2 : 0;
         fence_mbar_init();
     }
-    if (warp == 4) { tmem_alloc(smem_u32(tmem_slot), 512); tmem_relinquish(); }
+    if (warp == kIssueWarp) { tmem_alloc(smem_u32(tmem_slot), 512); tmem_relinquish(); }
     tc_fence_before_sync();
     __syncthreads();
     tc_fence_after_sync();
@@ -354,43 +543,65 @@ bwd_dkdv_kernel(const __grid_constant__ BwdParams p, const __grid_constant__ Bwd
     const uint32_t t_s = tmem, t_dp = tmem + 128, t_dk = tmem + 256, t_dv = tmem + 256 + D;
 
     if (skip) {
-    } else if (warp == 4) {
-        if (lane == 0) [&]() {
+    } else if (warp == kIssueWarp) {
+        [&]() {
+            const bool elected = elect_one();                    // all lanes walk the loop; one issues
             constexpr uint32_t idesc_s = idesc_bf16_f32(128, 128, 0, 0), idesc_g = idesc_bf16_f32(128, D, 1, 1);
-            mbar_arrive_expect_tx(bar(kKvFull), 2 * C::kTileBytes);
-            for (int a = 0; a < D / 64; ++a) {
-                tma_load_3d(k_s + a * C::kAtomBytes, &maps.k, bar(kKvFull), a * 64, r0, head);
-                tma_load_3d(v_s + a * C::kAtomBytes, &maps.v, bar(kKvFull), a * 64, r0, head);
+            auto load_q = [&](int q_row) {
+                if (elected) {
+                    mbar_arrive_expect_tx(bar(kQFull), C::kTileBytes);
+                    for (int a = 0; a < D / 64; ++a) tma_load_3d(q_s + a * C::kAtomBytes, &maps.q, bar(kQFull), a * 64, head, q_row);
+                }
+                __syncwarp();
+            };
+            auto load_do = [&](int q_row) {
+                if (elected) {
+                    mbar_arrive_expect_tx(bar(kDoFull), C::kTileBytes);
+                    for (int a = 0; a < D / 64; ++a) tma_load_3d(do_s + a * C::kAtomBytes, &maps.d_out, bar(kDoFull), a * 64, head, q_row);
+                }
+                __syncwarp();
+            };
+            auto commit = [&](int bar_id) { if (elected) tc_commit(bar(bar_id)); };
+            QTiles qt(p, r0);
+            if (qt.done()) return;
+            if (elected) {
+                mbar_arrive_expect_tx(bar(kKvFull), 2 * C::kTileBytes);
+                for (int a = 0; a < D / 64; ++a) {
+                    tma_load_3d(k_s + a * C::kAtomBytes, &maps.k, bar(kKvFull), a * 64, r0, head);
+                    tma_load_3d(v_s + a * C::kAtomBytes, &maps.v, bar(kKvFull), a * 64, r0, head);
+                }
             }
+            __syncwarp();
+            load_q(qt.q_row());
+            load_do(qt.q_row());
             if (!wait(kKvFull, 0, 0)) return;
-            uint32_t step = 0;
-            for (int g = 0; g < p.n_groups; ++g) {
-                const AttnGroup &G = p.g[g];
-                uint32_t valid[4];
-                if (!group_mask(G, r0, valid)) continue;
-                for (int i = 0; i * kTile < G.q_rows; ++i, ++step) {
-                    // the previous step's products have read Q, dO, P and dS
-                    if (step > 0 && !wait(kStepDone, step - 1, (int)step)) return;
-                    mbar_arrive_expect_tx(bar(kQdFull), 2 * C::kTileBytes);
-                    for (int a = 0; a < D / 64; ++a) {
-                        tma_load_3d(q_s + a * C::kAtomBytes, &maps.q, bar(kQdFull), a * 64, head, G.q_begin + i * kTile);
-                        tma_load_3d(do_s + a * C::kAtomBytes, &maps.d_out, bar(kQdFull), a * 64, head, G.q_begin + i * kTile);
-                    }
-                    if (!wait(kQdFull, step, (int)step)) return;
-                    tc_fence_after_sync();
-                    for (int kk = 0; kk < D / 16; ++kk)
-                        mma_ss(t_s, desc_kmajor(q_s, kk), desc_kmajor(k_s, kk), idesc_s, kk > 0);
-                    for (int kk = 0; kk < D / 16; ++kk)
-                        mma_ss(t_dp, desc_kmajor(do_s, kk), desc_kmajor(v_s, kk), idesc_s, kk > 0);
-                    tc_commit(bar(kSFull));
-                    if (!wait(kPdsFull, step, (int)step)) return;
-                    tc_fence_after_sync();
-                    // dV += P^T dO and dK += dS^T Q: the contraction runs over the 128 query rows
-                    for (int kk = 0; kk < kTile / 16; ++kk)
-                        mma_ss(t_dv, desc_mnmajor(p_s, kk), desc_mnmajor(do_s, kk), idesc_g, (step > 0 || kk > 0) ? 1u : 0u);
-                    for (int kk = 0; kk < kTile / 16; ++kk)
-                        mma_ss(t_dk, desc_mnmajor(ds_s, kk), desc_mnmajor(q_s, kk), idesc_g, (step > 0 || kk > 0) ? 1u : 0u);
-                    tc_commit(bar(kStepDone));
+            const uint32_t q_k = lo_kmajor(q_s), k_k = lo_kmajor(k_s), do_k = lo_kmajor(do_s), v_k = lo_kmajor(v_s);
+            const uint32_t ds_mn = lo_mnmajor(ds_s), q_mn = lo_mnmajor(q_s), p_mn = lo_mnmajor(p_s), do_mn = lo_mnmajor(do_s);
+            for (uint32_t step = 0; !qt.done(); ++step) {
+                if (!wait(kQFull, step, (int)step)) return;
+                tc_fence_after_sync();
+                if (elected) mma_slices<0, D / 16, false, false>(t_s, q_k, k_k, idesc_s, 0u);
+                __syncwarp();
+                if (!wait(kDoFull, step, (int)step)) return;
+                tc_fence_after_sync();
+                if (elected) mma_slices<0, D / 16, false, false>(t_dp, do_k, v_k, idesc_s, 0u);
+                __syncwarp();
+                commit(kSFull);
+                if (!wait(kPdsFull, step, (int)step)) return;
+                tc_fence_after_sync();
+                // dK += dS^T Q and dV += P^T dO: the contraction runs over the 128 query rows
+                if (elected) mma_slices<0, kTile / 16, true, true>(t_dk, ds_mn, q_mn, idesc_g, step > 0 ? 1u : 0u);
+                __syncwarp();
+                commit(kQFree);
+                if (elected) mma_slices<0, kTile / 16, true, true>(t_dv, p_mn, do_mn, idesc_g, step > 0 ? 1u : 0u);
+                __syncwarp();
+                commit(kStepDone);
+                qt.next();
+                if (!qt.done()) {
+                    if (!wait(kQFree, step, (int)step)) return;
+                    load_q(qt.q_row());
+                    if (!wait(kStepDone, step, (int)step)) return;
+                    load_do(qt.q_row());
                 }
             }
         }();
@@ -399,8 +610,8 @@ bwd_dkdv_kernel(const __grid_constant__ BwdParams p, const __grid_constant__ Bwd
         auto wait_c = [&](int bar_id, uint32_t parity, int iter) {
             if (alive && !__all_sync(0xffffffffu, wait(bar_id, parity, iter))) alive = false;
         };
-        const int row = threadIdx.x;
-        const uint32_t lane_off = (uint32_t)(32 * warp) << 16;
+        const int row = threadIdx.x & 127, half = threadIdx.x >> 7;
+        const uint32_t lane_off = (uint32_t)(32 * (warp & 3)) << 16;
         uint32_t step = 0;
         for (int g = 0; g < p.n_groups; ++g) {
             const AttnGroup &G = p.g[g];
@@ -409,10 +620,10 @@ bwd_dkdv_kernel(const __grid_constant__ BwdParams p, const __grid_constant__ Bwd
             for (int i = 0; i * kTile < G.q_rows; ++i, ++step) {
                 const bool live = i * kTile + row < G.q_rows;
                 const size_t stat = (size_t)head * p.nq_total + G.q_begin + (live ? i * kTile + row : 0);
-                const float lse2 = p.lse[stat] * 1.4426950408889634f, delta = p.delta[stat];
+                const float lse2 = live ? p.lse[stat] * 1.4426950408889634f : INFINITY, delta = p.delta[stat];
                 wait_c(kSFull, step, (int)step);
                 tc_fence_after_sync();
-                row_to_p_ds(t_s + lane_off, t_dp + lane_off, row, live, p.scale_log2, lse2, delta, valid, p_s, ds_s);
+                row_to_p_ds(t_s + lane_off, t_dp + lane_off, row, half, p.scale_log2, lse2, delta, valid, p_s, ds_s);
                 fence_proxy_async_smem();
                 tc_fence_before_sync();
                 compute_sync();
@@ -429,8 +640,8 @@ bwd_dkdv_kernel(const __grid_constant__ BwdParams p, const __grid_constant__ Bwd
         tc_fence_after_sync();
         if (alive && step > 0) {
             store_grad_row<D, true>(t_dk + lane_off, p.scale, p.dk + (token * p.heads + head) * D, p, live ? cf : 0,
-                                    cell / p.grid_w, cell % p.grid_w, live);
-            store_grad_row<D, false>(t_dv + lane_off, 1.f, p.dv + (token * p.heads + head) * D, p, 0, 0, 0, live);
+                                    cell / p.grid_w, cell % p.grid_w, live, half);
+            store_grad_row<D, false>(t_dv + lane_off, 1.f, p.dv + (token * p.heads + head) * D, p, 0, 0, 0, live, half);
         }
     }
     tc_fence_before_sync();
@@ -440,7 +651,7 @@ bwd_dkdv_kernel(const __grid_constant__ BwdParams p, const __grid_constant__ Bwd
         while (globaltimer_ns() - t0 < 200000ull) __nanosleep(1000);
         __syncthreads();
     }
-    if (warp == 4) { __syncwarp(); tc_fence_after_sync(); tmem_dealloc(tmem, 512); }
+    if (warp == kIssueWarp) { __syncwarp(); tc_fence_after_sync(); tmem_dealloc(tmem, 512); }
 }
 
 }  // namespace

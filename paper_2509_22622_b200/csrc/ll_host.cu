@@ -1100,7 +1100,7 @@ int ll_clip_attn_backward(ll_cache *c, int layer, const ll_bf16 *q_roped, const 
     p.n_groups = n_groups; p.heads = c->H; p.head_dim = c->D; p.nq_total = n_frames * c->P;
     p.scale = (float)(1.0 / std::sqrt((double)c->D));
     p.scale_log2 = ap.scale_log2;
-    p.out = out; p.d_out = d_out; p.lse = lse; p.delta = static_cast<float *>(workspace);
+    p.q = q_roped; p.out = out; p.d_out = d_out; p.lse = lse; p.delta = static_cast<float *>(workspace);
     p.dq = dq; p.dk = dk; p.dv = dv;
     p.status = reinterpret_cast<uint32_t *>(c->storage + c->off_status);
     p.P = c->P; p.grid_w = grid_w; p.n_t = rp.n_t; p.n_h = rp.n_h;

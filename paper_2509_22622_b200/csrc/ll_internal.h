@@ -168,7 +168,7 @@ struct BwdParams {
     int n_groups, heads, head_dim, nq_total;
     float scale;                      // 1 / sqrt(D)
     float scale_log2;                 // log2(e) / sqrt(D)
-    const ll_bf16 *out, *d_out;       // [nq_total, H, D]
+    const ll_bf16 *q, *out, *d_out;   // [nq_total, H, D]; q is the rotated query
     const float *lse;                 // [H, nq_total], natural log (the forward's)
     float *delta;                     // [H, nq_total] workspace: sum_d d_out * out
     ll_bf16 *dq, *dk, *dv;            // [nq_total, H, D]

@@ -11,10 +11,11 @@
 //
 // Two kernels instead of one with atomics: every gradient element is accumulated by one CTA in one
 // order, so the result is run-to-run deterministic, at the price of forming S and dP twice.  Both
-// kernels have one warp that loads (TMA) and issues the MMAs and eight compute warps that turn S
-// and dP into P and dS in shared memory (one thread per tile row and 64-key half, the 32x32b TMEM
-// shape).  The dq kernel forms S and dP in two 64-key halves, each with its own warp group, so that
-// the tensor pipe works on one half while the other is in the exponentials.
+// kernels have one warp that loads (TMA) and issues the MMAs (all its lanes walk the loop so that
+// descriptors are warp-uniform; one elected lane issues) and eight compute warps (one thread per
+// tile row and 64-key half, the 32x32b TMEM shape).  The compute warps take S into registers and
+// release its tensor memory at once, so the next step's S is formed while they are in the
+// exponentials; dP is read only for the last multiply.
 #include <cuda_bf16.h>
 
 #include "bounded_wait.cuh"
@@ -53,9 +54,6 @@ __device__ __forceinline__ void st_shared_v4(uint32_t addr, uint32_t a, uint32_t
     asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(a), "r"(b), "r"(c), "r"(d) : "memory");
 }
 
-// Meeting point of the eight compute warps (hardware barrier 0 is __syncthreads).
-__device__ __forceinline__ void compute_sync() { asm volatile("barrier.sync 1, 256;" ::: "memory"); }
-
 // delta[h][i] = sum_d d_out[i][h][d] * out[i][h][d]: one warp per (row, head).
 template <int D>
 __global__ void __launch_bounds__(256) bwd_delta_kernel(const __grid_constant__ BwdParams p)
@@ -76,55 +74,6 @@ __global__ void __launch_bounds__(256) bwd_delta_kernel(const __grid_constant__ 
 #pragma unroll
     for (int m = 16; m > 0; m >>= 1) s += __shfl_xor_sync(0xffffffffu, s, m);
     if (lane == 0) p.delta[(size_t)head * p.nq_total + row] = s;
-}
-
-// One row of one 64-key half of a 128 x 128 score tile and of the matching dP tile (TMEM, fp32) to P and/or dS
-// (bf16) in 128-byte-swizzled shared-memory tiles laid out [row][key]: two 64-key atoms of
-// 128 rows x 128 bytes, row r's 16-byte chunk k at chunk position k ^ (r % 8).
-//   p = 2^(s * c - lse2), ds = p * (dp - delta); columns whose bit in `valid` is clear give
-//   zeros (a row that is not live passes lse2 = +inf, which makes its p zero).  The arithmetic
-//   runs on packed pairs; the per-column mask is only applied to chunks that are not all valid.
-__device__ __forceinline__ void row_to_p_ds(uint32_t t_s, uint32_t t_dp, int row, int half, float c, float lse2,
-                                            float delta, const uint32_t (&valid)[4], uint32_t p_tile, uint32_t ds_tile)
-{
-    const uint64_t c2 = pack2(c, c), nl2 = pack2(-lse2, -lse2), nd2 = pack2(-delta, -delta);
-#pragma unroll 1
-    for (int ch = 2 * half; ch < 2 * half + 2; ++ch) {
-        uint32_t s[32], dp[32];
-        tmem_ld_32x32b_x32(t_s + 32 * ch, s);
-        tmem_ld_32x32b_x32(t_dp + 32 * ch, dp);
-        tmem_wait_ld();
-        const uint32_t vbits = ch == 0 ? valid[0] : ch == 1 ? valid[1] : ch == 2 ? valid[2] : valid[3];
-        uint32_t pw[16], dw[16];
-        if (vbits == 0xffffffffu) {
-#pragma unroll
-            for (int i = 0; i < 16; ++i) {
-                float e0, e1, d0, d1;
-                unpack2(fma2(pack2(as_f(s[2 * i]), as_f(s[2 * i + 1])), c2, nl2), e0, e1);
-                const float p0 = ex2(e0), p1 = ex2(e1);
-                pw[i] = cvt_bf16x2(p0, p1);
-                unpack2(mul2(pack2(p0, p1), add2(pack2(as_f(dp[2 * i]), as_f(dp[2 * i + 1])), nd2)), d0, d1);
-                dw[i] = cvt_bf16x2(d0, d1);
-            }
-        } else {
-#pragma unroll
-            for (int i = 0; i < 16; ++i) {
-                float p0 = ex2(fmaf(as_f(s[2 * i]), c, -lse2)), p1 = ex2(fmaf(as_f(s[2 * i + 1]), c, -lse2));
-                if (!((vbits >> (2 * i)) & 1u)) p0 = 0.f;
-                if (!((vbits >> (2 * i + 1)) & 1u)) p1 = 0.f;
-                pw[i] = cvt_bf16x2(p0, p1);
-                dw[i] = cvt_bf16x2(p0 * (as_f(dp[2 * i]) - delta), p1 * (as_f(dp[2 * i + 1]) - delta));
-            }
-        }
-        // 32 keys = four 16-byte chunks of this row, in atom ch / 2
-        const uint32_t row_off = (uint32_t)(ch >> 1) * (128 * 128) + (uint32_t)row * 128;
-#pragma unroll
-        for (int k = 0; k < 4; ++k) {
-            const uint32_t chunk = (uint32_t)(((ch & 1) * 4 + k) ^ (row & 7)) << 4;
-            if (p_tile) st_shared_v4(p_tile + row_off + chunk, pw[4 * k], pw[4 * k + 1], pw[4 * k + 2], pw[4 * k + 3]);
-            st_shared_v4(ds_tile + row_off + chunk, dw[4 * k], dw[4 * k + 1], dw[4 * k + 2], dw[4 * k + 3]);
-        }
-    }
 }
 
 // Half `half` of the D columns of 128 rows x D fp32 in TMEM (row = thread), times `mul`,
@@ -234,8 +183,10 @@ __device__ __forceinline__ void scores_to_weights(uint32_t (&s)[64], float c, fl
 }
 
 // dS = p (dP - delta) of this thread's 64 columns (32-column chunks ch0, ch0 + 1 of tile row
-// `row`), rounded to bf16, into the swizzled [row][key] tile.
-__device__ __forceinline__ void store_ds(const uint32_t (&pw)[64], uint32_t t_dp, int row, int ch0, float delta, uint32_t ds_tile)
+// `row`), rounded to bf16, into the swizzled [row][key] tile; the weights themselves too when
+// p_tile is not 0.
+__device__ __forceinline__ void store_ds(const uint32_t (&pw)[64], uint32_t t_dp, int row, int ch0, float delta, uint32_t p_tile,
+                                         uint32_t ds_tile)
 {
     const uint64_t nd2 = pack2(-delta, -delta);
 #pragma unroll
@@ -257,6 +208,11 @@ __device__ __forceinline__ void store_ds(const uint32_t (&pw)[64], uint32_t t_dp
         for (int k = 0; k < 4; ++k) {
             const uint32_t chunk = (uint32_t)(((ch & 1) * 4 + k) ^ (row & 7)) << 4;
             st_shared_v4(ds_tile + row_off + chunk, dw[4 * k], dw[4 * k + 1], dw[4 * k + 2], dw[4 * k + 3]);
+            if (p_tile) {
+                const int b = 32 * h + 8 * k;
+                st_shared_v4(p_tile + row_off + chunk, cvt_bf16x2(as_f(pw[b]), as_f(pw[b + 1])), cvt_bf16x2(as_f(pw[b + 2]), as_f(pw[b + 3])),
+                             cvt_bf16x2(as_f(pw[b + 4]), as_f(pw[b + 5])), cvt_bf16x2(as_f(pw[b + 6]), as_f(pw[b + 7])));
+            }
         }
     }
 }
@@ -437,7 +393,7 @@ bwd_dq_kernel(const __grid_constant__ BwdParams p, const __grid_constant__ BwdMa
             scores_to_weights(w, p.scale_log2, lse2, half ? valid[2] : valid[0], half ? valid[3] : valid[1]);
             wait_c(kDpFull, j, j);
             tc_fence_after_sync();
-            store_ds(w, t_dp + lane_off, row, 2 * half, delta, ds_s);
+            store_ds(w, t_dp + lane_off, row, 2 * half, delta, 0u, ds_s);
             fence_proxy_async_smem();
             tc_fence_before_sync();
             __syncwarp();
@@ -503,9 +459,15 @@ struct QTiles {
 };
 
 // ---- dk, dv: one CTA per (128-row tile of the clip's cache rows, head) -----------------------
-// K and V of the tile stay in shared memory; per step one query tile's Q and dO come in.  The
-// step's last products are issued dK (reads dS, Q) then dV (reads P, dO), each with a barrier of
-// its own, so the next Q is under way while dV runs and the next S can start before dO is in.
+// K and V of the tile stay in shared memory; per step j one query tile's Q and dO stream in.
+// The tensor pipe runs, per step,  S(j+1) | dV(j) | dK(j) | dP(j+1):  the eight compute warps
+// take S(j) into registers and release it at once, so S(j+1) is formed while they are in the
+// exponentials; dP(j) is only needed for dS = P (dP - delta), after which P and dS go to shared
+// memory as the MN-major A operands of dV += P^T dO and dK += dS^T Q.
+// Shared memory has room for three streamed tiles beside K, V, P and dS, so Q is loaded twice:
+//   slot j % 2:  Q(j) for S(j), then (once S(j) is done) dO(j) for dP(j) and dV(j), then Q(j+2)
+//   slot C:      Q(j) for dK(j), then Q(j+1)
+// which gives every load about one step of lead.
 template <int D>
 __global__ void __launch_bounds__(kBwdThreads, 1)
 bwd_dkdv_kernel(const __grid_constant__ BwdParams p, const __grid_constant__ BwdMaps maps)
@@ -514,13 +476,14 @@ bwd_dkdv_kernel(const __grid_constant__ BwdParams p, const __grid_constant__ Bwd
     extern __shared__ uint8_t smem_raw[];
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     uint8_t *gen = smem_raw + (base - smem_u32(smem_raw));
-    const uint32_t k_s = base, v_s = k_s + C::kTileBytes, q_s = v_s + C::kTileBytes, do_s = q_s + C::kTileBytes,
-                   p_s = do_s + C::kTileBytes, ds_s = p_s + C::kPBytes, bars = ds_s + C::kPBytes;
-    enum { kKvFull = 0, kQFull = 1, kDoFull = 2, kSFull = 3, kPdsFull = 4, kQFree = 5, kStepDone = 6, kBars = 7 };
+    const uint32_t k_s = base, v_s = k_s + C::kTileBytes, slot_s = v_s + C::kTileBytes, c_s = slot_s + 2 * C::kTileBytes,
+                   p_s = c_s + C::kTileBytes, ds_s = p_s + C::kPBytes, bars = ds_s + C::kPBytes;
+    enum { kKvFull = 0, kSlotFull = 1, kCFull = 3, kSFull = 4, kSFree = 5, kDpFull = 6, kDsFull = 7, kSlotFree = 8, kCFree = 10, kBars = 11 };
+    constexpr int kComputeWarps = 8;
     uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(gen + (bars - base) + kBars * 8);
     volatile int *abort_flag = reinterpret_cast<volatile int *>(tmem_slot + 1);
     auto bar = [&](int i) -> uint32_t { return bars + 8u * (uint32_t)i; };
-    const int warp = __shfl_sync(0xffffffffu, (int)(threadIdx.x >> 5), 0);
+    const int warp = __shfl_sync(0xffffffffu, (int)(threadIdx.x >> 5), 0), lane = threadIdx.x & 31;
     const int head = blockIdx.y;
     // the tile's first cache row and the end of the run it belongs to
     int run = 0, t = blockIdx.x;
@@ -528,7 +491,7 @@ bwd_dkdv_kernel(const __grid_constant__ BwdParams p, const __grid_constant__ Bwd
     const int r0 = p.krun_start[run] + t * kTile, run_end = p.krun_start[run] + p.krun_len[run];
 
     if (threadIdx.x == 0) {
-        for (int i = 0; i < kBars; ++i) mbar_init(bar(i), 1);
+        for (int i = 0; i < kBars; ++i) mbar_init(bar(i), (i == kSFree || i == kDsFull) ? kComputeWarps : 1);
         *abort_flag = (*reinterpret_cast<volatile uint32_t *>(p.status) != kStatusOk) ? 2 : 0;
         fence_mbar_init();
     }
@@ -547,23 +510,19 @@ bwd_dkdv_kernel(const __grid_constant__ BwdParams p, const __grid_constant__ Bwd
         [&]() {
             const bool elected = elect_one();                    // all lanes walk the loop; one issues
             constexpr uint32_t idesc_s = idesc_bf16_f32(128, 128, 0, 0), idesc_g = idesc_bf16_f32(128, D, 1, 1);
-            auto load_q = [&](int q_row) {
+            auto load_tile = [&](uint32_t dst, const CUtensorMap *map, int bar_id, int q_row) {
                 if (elected) {
-                    mbar_arrive_expect_tx(bar(kQFull), C::kTileBytes);
-                    for (int a = 0; a < D / 64; ++a) tma_load_3d(q_s + a * C::kAtomBytes, &maps.q, bar(kQFull), a * 64, head, q_row);
-                }
-                __syncwarp();
-            };
-            auto load_do = [&](int q_row) {
-                if (elected) {
-                    mbar_arrive_expect_tx(bar(kDoFull), C::kTileBytes);
-                    for (int a = 0; a < D / 64; ++a) tma_load_3d(do_s + a * C::kAtomBytes, &maps.d_out, bar(kDoFull), a * 64, head, q_row);
+                    mbar_arrive_expect_tx(bar(bar_id), C::kTileBytes);
+                    for (int a = 0; a < D / 64; ++a) tma_load_3d(dst + a * C::kAtomBytes, map, bar(bar_id), a * 64, head, q_row);
                 }
                 __syncwarp();
             };
             auto commit = [&](int bar_id) { if (elected) tc_commit(bar(bar_id)); };
+            // first rows of the query tiles of steps j, j + 1, j + 2 (-1: no such step)
             QTiles qt(p, r0);
-            if (qt.done()) return;
+            auto take = [&]() -> int { if (qt.done()) return -1; const int r = qt.q_row(); qt.next(); return r; };
+            int row_j = take(), row_j1 = take(), row_j2 = take();
+            if (row_j < 0) return;
             if (elected) {
                 mbar_arrive_expect_tx(bar(kKvFull), 2 * C::kTileBytes);
                 for (int a = 0; a < D / 64; ++a) {
@@ -572,37 +531,64 @@ bwd_dkdv_kernel(const __grid_constant__ BwdParams p, const __grid_constant__ Bwd
                 }
             }
             __syncwarp();
-            load_q(qt.q_row());
-            load_do(qt.q_row());
-            if (!wait(kKvFull, 0, 0)) return;
-            const uint32_t q_k = lo_kmajor(q_s), k_k = lo_kmajor(k_s), do_k = lo_kmajor(do_s), v_k = lo_kmajor(v_s);
-            const uint32_t ds_mn = lo_mnmajor(ds_s), q_mn = lo_mnmajor(q_s), p_mn = lo_mnmajor(p_s), do_mn = lo_mnmajor(do_s);
-            for (uint32_t step = 0; !qt.done(); ++step) {
-                if (!wait(kQFull, step, (int)step)) return;
+            load_tile(slot_s, &maps.q, kSlotFull + 0, row_j);
+            if (row_j1 >= 0) load_tile(slot_s + C::kTileBytes, &maps.q, kSlotFull + 1, row_j1);
+            load_tile(c_s, &maps.q, kCFull, row_j);
+            const uint32_t k_k = lo_kmajor(k_s), v_k = lo_kmajor(v_s), p_mn = lo_mnmajor(p_s), ds_mn = lo_mnmajor(ds_s), c_mn = lo_mnmajor(c_s);
+            // a slot's fills alternate Q (for S) and dO: waits see parity 0 for Q, 1 for dO
+            auto issue_s = [&](int j) -> bool {
+                const int sl = j & 1;
+                if (!wait(kSlotFull + sl, 0, j)) return false;
                 tc_fence_after_sync();
-                if (elected) mma_slices<0, D / 16, false, false>(t_s, q_k, k_k, idesc_s, 0u);
-                __syncwarp();
-                if (!wait(kDoFull, step, (int)step)) return;
-                tc_fence_after_sync();
-                if (elected) mma_slices<0, D / 16, false, false>(t_dp, do_k, v_k, idesc_s, 0u);
+                if (elected) mma_slices<0, D / 16, false, false>(t_s, lo_kmajor(slot_s + sl * C::kTileBytes), k_k, idesc_s, 0u);
                 __syncwarp();
                 commit(kSFull);
-                if (!wait(kPdsFull, step, (int)step)) return;
+                return true;
+            };
+            auto issue_dp = [&](int j) -> bool {
+                const int sl = j & 1;
+                if (!wait(kSlotFull + sl, 1, j)) return false;
                 tc_fence_after_sync();
-                // dK += dS^T Q and dV += P^T dO: the contraction runs over the 128 query rows
-                if (elected) mma_slices<0, kTile / 16, true, true>(t_dk, ds_mn, q_mn, idesc_g, step > 0 ? 1u : 0u);
+                if (elected) mma_slices<0, D / 16, false, false>(t_dp, lo_kmajor(slot_s + sl * C::kTileBytes), v_k, idesc_s, 0u);
                 __syncwarp();
-                commit(kQFree);
-                if (elected) mma_slices<0, kTile / 16, true, true>(t_dv, p_mn, do_mn, idesc_g, step > 0 ? 1u : 0u);
-                __syncwarp();
-                commit(kStepDone);
-                qt.next();
-                if (!qt.done()) {
-                    if (!wait(kQFree, step, (int)step)) return;
-                    load_q(qt.q_row());
-                    if (!wait(kStepDone, step, (int)step)) return;
-                    load_do(qt.q_row());
+                commit(kDpFull);
+                return true;
+            };
+            if (!wait(kKvFull, 0, 0)) return;
+            if (!issue_s(0)) return;
+            if (!wait(kSFull, 0, 0)) return;                     // S(0) has read Q(0): its slot takes dO(0)
+            load_tile(slot_s, &maps.d_out, kSlotFull + 0, row_j);
+            if (!issue_dp(0)) return;
+            for (int j = 0;; ++j) {
+                const int sl = j & 1;
+                if (row_j1 >= 0) {
+                    if (!wait(kSFree, j, j)) return;             // S(j) is in the compute warps' registers
+                    if (!issue_s(j + 1)) return;
+                    if (!wait(kSFull, j + 1, j)) return;         // S(j+1) has read Q(j+1): its slot takes dO(j+1)
+                    load_tile(slot_s + (sl ^ 1) * C::kTileBytes, &maps.d_out, kSlotFull + (sl ^ 1), row_j1);
                 }
+                if (!wait(kDsFull, j, j)) return;                // P(j) and dS(j) are in shared memory, dP(j) has been read
+                tc_fence_after_sync();
+                // dV += P^T dO and dK += dS^T Q: the contraction runs over the 128 query rows
+                if (elected) mma_slices<0, kTile / 16, true, true>(t_dv, p_mn, lo_mnmajor(slot_s + sl * C::kTileBytes), idesc_g, j > 0 ? 1u : 0u);
+                __syncwarp();
+                commit(kSlotFree + sl);
+                if (!wait(kCFull, j, j)) return;
+                tc_fence_after_sync();
+                if (elected) mma_slices<0, kTile / 16, true, true>(t_dk, ds_mn, c_mn, idesc_g, j > 0 ? 1u : 0u);
+                __syncwarp();
+                commit(kCFree);
+                if (row_j1 < 0) break;
+                if (!issue_dp(j + 1)) return;
+                if (row_j2 >= 0) {                               // dV(j) has read dO(j): its slot takes Q(j+2)
+                    if (!wait(kSlotFree + sl, j >> 1, j)) return;
+                    load_tile(slot_s + sl * C::kTileBytes, &maps.q, kSlotFull + sl, row_j2);
+                }
+                if (!wait(kCFree, j, j)) return;                 // dK(j) has read Q(j)
+                load_tile(c_s, &maps.q, kCFull, row_j1);
+                row_j = row_j1;
+                row_j1 = row_j2;
+                row_j2 = take();
             }
         }();
     } else {
@@ -623,11 +609,22 @@ bwd_dkdv_kernel(const __grid_constant__ BwdParams p, const __grid_constant__ Bwd
                 const float lse2 = live ? p.lse[stat] * 1.4426950408889634f : INFINITY, delta = p.delta[stat];
                 wait_c(kSFull, step, (int)step);
                 tc_fence_after_sync();
-                row_to_p_ds(t_s + lane_off, t_dp + lane_off, row, half, p.scale_log2, lse2, delta, valid, p_s, ds_s);
+                uint32_t w[64];
+                tmem_ld_32x32b_x32(t_s + lane_off + 64 * half, w);
+                tmem_ld_32x32b_x32(t_s + lane_off + 64 * half + 32, w + 32);
+                tmem_wait_ld();
+                tc_fence_before_sync();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(bar(kSFree));
+                scores_to_weights(w, p.scale_log2, lse2, half ? valid[2] : valid[0], half ? valid[3] : valid[1]);
+                wait_c(kDpFull, step, (int)step);
+                if (step > 0) wait_c(kCFree, step - 1, (int)step);       // the last step's products have read P and dS
+                tc_fence_after_sync();
+                store_ds(w, t_dp + lane_off, row, 2 * half, delta, p_s, ds_s);
                 fence_proxy_async_smem();
                 tc_fence_before_sync();
-                compute_sync();
-                if (threadIdx.x == 0) mbar_arrive(bar(kPdsFull));
+                __syncwarp();
+                if (lane == 0) mbar_arrive(bar(kDsFull));
             }
         }
         // this thread's key row: stored only if it is one of the clip's rows inside this run
@@ -636,7 +633,7 @@ bwd_dkdv_kernel(const __grid_constant__ BwdParams p, const __grid_constant__ Bwd
         const int cf = (r < run_end && slot < LL_MAX_SLOTS) ? p.slot_clip_frame[slot] : -1;
         const bool live = cf >= 0;
         const size_t token = live ? (size_t)cf * p.P + cell : 0;
-        if (step > 0) wait_c(kStepDone, step - 1, (int)step);
+        if (step > 0) wait_c(kCFree, step - 1, (int)step);
         tc_fence_after_sync();
         if (alive && step > 0) {
             store_grad_row<D, true>(t_dk + lane_off, p.scale, p.dk + (token * p.heads + head) * D, p, live ? cf : 0,
@@ -660,7 +657,7 @@ cudaError_t launch_attn_backward(const BwdParams &p, const BwdMaps &maps, cudaSt
 {
     const int D = p.head_dim;
     const size_t tile = (size_t)128 * D * 2, ptile = 2 * 128 * 128;
-    const int smem_dq = (int)(6 * tile + ptile + 2048), smem_kv = (int)(4 * tile + 2 * ptile + 2048);
+    const int smem_dq = (int)(6 * tile + ptile + 2048), smem_kv = (int)(5 * tile + 2 * ptile + 2048);
     cudaError_t e;
     if (D == 128) {
         e = cudaFuncSetAttribute(bwd_dq_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_dq);

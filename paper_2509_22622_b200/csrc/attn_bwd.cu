@@ -19,6 +19,7 @@
 #include <cuda_bf16.h>
 
 #include "bounded_wait.cuh"
+#include "exp2_poly.cuh"
 #include "ll_internal.h"
 #include "ptx.cuh"
 
@@ -31,8 +32,6 @@ using namespace ptx;
 constexpr int kBwdThreads = 288;                       // eight compute warps, one load/issue warp
 constexpr int kIssueWarp = 8;
 constexpr int kTile = 128;
-
-__device__ __forceinline__ float as_f(uint32_t u) { return __uint_as_float(u); }
 
 __device__ __forceinline__ void tmem_ld_32x32b_x32(uint32_t taddr, uint32_t *r)
 {
@@ -164,16 +163,19 @@ __device__ __forceinline__ void key_mask(int nvalid, uint32_t (&valid)[4])
 }
 
 // This thread's 64 columns of a score row (fp32 words in s) to the weights p = 2^(s c - lse2),
-// in place; columns whose bit in vlo (first 32) / vhi is clear give zero.
+// in place; columns whose bit in vlo (first 32) / vhi is clear give zero.  (Moving a quarter or
+// a half of the exponentials to the FMA-pipe polynomial of the forward kernel made the pass
+// slower, 8.46 and 8.59 ms against 8.35 ms at the 21-frame clip, so all of them stay on the
+// special-function unit.)
 __device__ __forceinline__ void scores_to_weights(uint32_t (&s)[64], float c, float lse2, uint32_t vlo, uint32_t vhi)
 {
     const uint64_t c2 = pack2(c, c), nl2 = pack2(-lse2, -lse2);
 #pragma unroll
     for (int i = 0; i < 32; ++i) {
         float e0, e1;
-        unpack2(fma2(pack2(as_f(s[2 * i]), as_f(s[2 * i + 1])), c2, nl2), e0, e1);
-        s[2 * i] = __float_as_uint(ex2(e0));
-        s[2 * i + 1] = __float_as_uint(ex2(e1));
+        unpack2(exp2_sfu2(fma2(pack2(as_f(s[2 * i]), as_f(s[2 * i + 1])), c2, nl2)), e0, e1);
+        s[2 * i] = __float_as_uint(e0);
+        s[2 * i + 1] = __float_as_uint(e1);
     }
     if ((vlo & vhi) != 0xffffffffu) {
 #pragma unroll
@@ -376,7 +378,7 @@ bwd_dq_kernel(const __grid_constant__ BwdParams p, const __grid_constant__ BwdMa
         const bool live = row < rows;
         const uint32_t lane_off = (uint32_t)(32 * (warp & 3)) << 16;
         const size_t stat = (size_t)head * p.nq_total + q0 + (live ? row : 0);
-        const float lse2 = live ? p.lse[stat] * 1.4426950408889634f : INFINITY, delta = p.delta[stat];
+        const float lse2 = p.lse[stat] * 1.4426950408889634f, delta = p.delta[stat];
         RunTiles kt(&G);
         for (int j = 0; j < n_kt; ++j, kt.next()) {
             uint32_t valid[4];
@@ -390,7 +392,7 @@ bwd_dq_kernel(const __grid_constant__ BwdParams p, const __grid_constant__ BwdMa
             tc_fence_before_sync();
             __syncwarp();
             if (lane == 0) mbar_arrive(bar(kSFree));
-            scores_to_weights(w, p.scale_log2, lse2, half ? valid[2] : valid[0], half ? valid[3] : valid[1]);
+            scores_to_weights(w, p.scale_log2, lse2, live ? (half ? valid[2] : valid[0]) : 0u, live ? (half ? valid[3] : valid[1]) : 0u);
             wait_c(kDpFull, j, j);
             tc_fence_after_sync();
             store_ds(w, t_dp + lane_off, row, 2 * half, delta, 0u, ds_s);
@@ -606,7 +608,7 @@ bwd_dkdv_kernel(const __grid_constant__ BwdParams p, const __grid_constant__ Bwd
             for (int i = 0; i * kTile < G.q_rows; ++i, ++step) {
                 const bool live = i * kTile + row < G.q_rows;
                 const size_t stat = (size_t)head * p.nq_total + G.q_begin + (live ? i * kTile + row : 0);
-                const float lse2 = live ? p.lse[stat] * 1.4426950408889634f : INFINITY, delta = p.delta[stat];
+                const float lse2 = p.lse[stat] * 1.4426950408889634f, delta = p.delta[stat];
                 wait_c(kSFull, step, (int)step);
                 tc_fence_after_sync();
                 uint32_t w[64];
@@ -616,7 +618,7 @@ bwd_dkdv_kernel(const __grid_constant__ BwdParams p, const __grid_constant__ Bwd
                 tc_fence_before_sync();
                 __syncwarp();
                 if (lane == 0) mbar_arrive(bar(kSFree));
-                scores_to_weights(w, p.scale_log2, lse2, half ? valid[2] : valid[0], half ? valid[3] : valid[1]);
+                scores_to_weights(w, p.scale_log2, lse2, live ? (half ? valid[2] : valid[0]) : 0u, live ? (half ? valid[3] : valid[1]) : 0u);
                 wait_c(kDpFull, step, (int)step);
                 if (step > 0) wait_c(kCFree, step - 1, (int)step);       // the last step's products have read P and dS
                 tc_fence_after_sync();

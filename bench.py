@@ -596,8 +596,19 @@ def run_ours(args):
         n_prompt = 512
         pk = torch.randn(n_prompt, H, D, device="cuda").bfloat16()
         pv = torch.randn(n_prompt, H, D, device="cuda").bfloat16()
-        ms = median_ms(lambda: cache.cross_attn(q, pk, pv, out))
-        others["cross_attn_512_keys"] = {"us": ms * 1e3, "tflops": 4.0 * nq * n_prompt * D * H / ms / 1e9}
+        ms_call = median_ms(lambda: cache.cross_attn(q, pk, pv, out))
+        # the launch is shorter than a call's host time: ten calls in a captured graph give the device time
+        cache.cross_attn(q, pk, pv, out)
+        torch.cuda.synchronize()
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph):
+            for _ in range(10):
+                cache.cross_attn(q, pk, pv, out)
+        ms = median_ms(graph.replay) / 10
+        cache.check_device()
+        others["cross_attn_512_keys"] = {"us": ms * 1e3, "tflops": 4.0 * nq * n_prompt * D * H / ms / 1e9,
+                                         "us_one_call_between_events": ms_call * 1e3,
+                                         "how": "ten launches in a captured CUDA graph, replayed"}
         cache.check_device()
 
     loop_vals = [in_loop["ms_total"], in_loop["attn_ms_per_launch_second_half"]] if in_loop else [0.0, 0.0]

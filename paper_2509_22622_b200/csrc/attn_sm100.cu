@@ -34,8 +34,9 @@
 //   warps hold the tile in registers, so the MMA warp issues QK of step j+1 while
 //   the softmax of step j is still running, and the softmax warps find the next S
 //   waiting.  The tensor pipe then sees, per lane and step, PV(first half), QK(next),
-//   PV(second half), whenever their inputs arrive.  A share of the exponentials is
-//   evaluated with a cubic on the FMA pipe instead of the special-function unit.
+//   PV(second half), whenever their inputs arrive.  A share of the exponentials can be
+//   evaluated with a cubic on the FMA pipe instead of the special-function unit
+//   (kPolyMask; measured best at none).
 //
 // TMEM columns: S_0 | S_1 | O_0 | O_1 (fp32).  The visible keys are a short list of
 // contiguous cache-row runs (sink, ring, wrapped ring); softmax does not care about
@@ -76,8 +77,11 @@ constexpr int kSoftmaxRegs = 104;
 constexpr int kProducerRegs = 64;
 static_assert(kSoftmaxWarps * kSoftmaxRegs + (kThreads / 32 - kSoftmaxWarps) * kProducerRegs <= (kThreads / 32) * kLaunchRegs,
               "setmaxnreg targets exceed the CTA's register allocation");
-// 8-key groups (bit k of 16 per 128-key tile) whose exponentials use the cubic
-constexpr uint32_t kPolyMask = 0x8888u;
+// 8-key groups (bit k of 16 per 128-key tile) whose exponentials use the cubic.  None: with
+// the kernel as it stands the special-function unit is not what a step waits for, and the
+// cubic's ten instructions per pair cost time and power (0.4027 ms against 0.4047 ms with one
+// group in four, 0.4218 ms with two; 0.4664 / 0.4715 / 0.4915 ms in a long loop at the power cap).
+constexpr uint32_t kPolyMask = 0x0000u;
 
 template <int D>
 struct Cfg {

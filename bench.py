@@ -606,6 +606,23 @@ def run_ours(args):
                 cache.cross_attn(q, pk, pv, out)
         ms = median_ms(graph.replay) / 10
         cache.check_device()
+        # the same grid and width with 24 heads of 64: twice the exponentials per flop
+        H64, D64 = 2 * H, D // 2
+        c64 = B.Cache(2, H64, D64, P, C, wl.sink_frames, wl.window_frames, device="cuda:%d" % local_rank)
+        q64 = torch.randn(nq, H64, D64, device="cuda").bfloat16()
+        k64, v64 = torch.randn_like(q64), torch.randn_like(q64)
+        qr64, out64 = torch.empty_like(q64), torch.empty_like(q64)
+        for l in range(2):
+            for chunk in range(n_fill):
+                c64.rope_append_kv(l, q64, k64, v64, chunk * C, wl.grid_h, wl.grid_w, wl.rope_theta, qr64)
+
+        def att64():
+            lay[0] ^= 1
+            c64.sink_window_attn(lay[0], qr64, (n_fill - 1) * C, out64)
+        ms64 = median_ms(att64)
+        c64.check_device()
+        c64.close()
+        others["head_dim_64_24_heads"] = {"ms": ms64, "tflops": attn_flops(wl) / ms64 / 1e9}
         others["cross_attn_512_keys"] = {"us": ms * 1e3, "tflops": 4.0 * nq * n_prompt * D * H / ms / 1e9,
                                          "us_one_call_between_events": ms_call * 1e3,
                                          "how": "ten launches in a captured CUDA graph, replayed"}

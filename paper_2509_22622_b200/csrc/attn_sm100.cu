@@ -36,7 +36,7 @@
 //   waiting.  The tensor pipe then sees, per lane and step, PV(first half), QK(next),
 //   PV(second half), whenever their inputs arrive.  A share of the exponentials can be
 //   evaluated with a cubic on the FMA pipe instead of the special-function unit
-//   (kPolyMask; measured best at none).
+//   (kPolyMask: none at head_dim 128, a quarter at head_dim 64, as measured).
 //
 // TMEM columns: S_0 | S_1 | O_0 | O_1 (fp32).  The visible keys are a short list of
 // contiguous cache-row runs (sink, ring, wrapped ring); softmax does not care about
@@ -77,11 +77,14 @@ constexpr int kSoftmaxRegs = 104;
 constexpr int kProducerRegs = 64;
 static_assert(kSoftmaxWarps * kSoftmaxRegs + (kThreads / 32 - kSoftmaxWarps) * kProducerRegs <= (kThreads / 32) * kLaunchRegs,
               "setmaxnreg targets exceed the CTA's register allocation");
-// 8-key groups (bit k of 16 per 128-key tile) whose exponentials use the cubic.  None: with
-// the kernel as it stands the special-function unit is not what a step waits for, and the
-// cubic's ten instructions per pair cost time and power (0.4027 ms against 0.4047 ms with one
-// group in four, 0.4218 ms with two; 0.4664 / 0.4715 / 0.4915 ms in a long loop at the power cap).
-constexpr uint32_t kPolyMask = 0x0000u;
+// 8-key groups (bit k of 16 per 128-key tile) whose exponentials use the cubic instead of the
+// special-function unit.  head_dim 128: none - the special-function unit is not what a step
+// waits for, and the cubic's ten instructions per pair cost time and power (0.4027 ms against
+// 0.4047 ms with one group in four, 0.4218 ms with two; 0.4664 / 0.4715 / 0.4915 ms in a long
+// loop at the power cap).  head_dim 64 has twice the exponentials per flop and is bound by
+// them: one group in four (0.681 ms against 0.726 ms with none, 0.684 / 0.683 ms with one in
+// eight / three in eight, 24 heads on the same grid).
+template <int D> constexpr uint32_t kPolyMask = D == 64 ? 0x8888u : 0x0000u;
 
 template <int D>
 struct Cfg {
@@ -480,7 +483,7 @@ attn_sm100_kernel(const __grid_constant__ AttnParams p, const __grid_constant__ 
 #pragma unroll
                                 for (int kk = 0; kk < 4; ++kk) {
                                     const int k = 4 * g + kk;
-                                    if (!((kPolyMask >> (8 * piece + k)) & 1u)) {
+                                    if (!((kPolyMask<D> >> (8 * piece + k)) & 1u)) {
                                         xa[kk] = fma2(pack2(as_f(v[4 * k]), as_f(v[4 * k + 1])), c2a, na2);
                                         xb[kk] = fma2(pack2(as_f(v[4 * k + 2]), as_f(v[4 * k + 3])), c2b, nb2);
                                     }
@@ -488,7 +491,7 @@ attn_sm100_kernel(const __grid_constant__ AttnParams p, const __grid_constant__ 
 #pragma unroll
                                 for (int kk = 0; kk < 4; ++kk) {
                                     const int k = 4 * g + kk;
-                                    if ((kPolyMask >> (8 * piece + k)) & 1u) {
+                                    if ((kPolyMask<D> >> (8 * piece + k)) & 1u) {
                                         xa[kk] = exp2_poly2(as_f(v[4 * k]), as_f(v[4 * k + 1]), ra);
                                         xb[kk] = exp2_poly2(as_f(v[4 * k + 2]), as_f(v[4 * k + 3]), rb);
                                     } else {

@@ -199,7 +199,7 @@ int ll_norm_rope_append_kv(ll_cache *cache, int layer, const ll_bf16 *q, const l
  * ll_qkv_proj_workspace_bytes (4 bytes per k element of a chunk plus a table of partial
  * sums), caller-owned, free again when the call's kernels have run.  Without the norm
  * q_row_scale and workspace may be NULL.
- * heads*head_dim must be a multiple of 256; bf16 caches only; positions, state and errors
+ * heads*head_dim must be a multiple of 256 or of 192; bf16 caches only; positions, state and errors
  * as ll_rope_append_kv. */
 size_t ll_qkv_proj_workspace_bytes(const ll_cache *cache);
 int ll_qkv_proj_append(ll_cache *cache, int layer, const ll_bf16 *x, int d_model, const ll_bf16 *w_qkv,

@@ -788,7 +788,7 @@ size_t ll_qkv_proj_workspace_bytes(const ll_cache *c)
     if (!c) return 0;
     const size_t tokens = (size_t)c->C * c->P, hd = (size_t)c->H * c->D;
     // parked fp32 k rows, then the per-tile sums of squares of q and k
-    return align_up(tokens * hd * sizeof(float), 256) + align_up(2 * tokens * ((hd + 127) / 128) * sizeof(float), 256);
+    return align_up(tokens * hd * sizeof(float), 256) + align_up(2 * tokens * ((hd + 95) / 96) * sizeof(float), 256);
 }
 
 int ll_qkv_proj_append(ll_cache *c, int layer, const ll_bf16 *x, int d_model, const ll_bf16 *w_qkv, const float *bias,
@@ -802,8 +802,8 @@ int ll_qkv_proj_append(ll_cache *c, int layer, const ll_bf16 *x, int d_model, co
     if (!(rope_theta > 0.f)) return fail(LL_ERR_INVALID_ARG, "rope_theta must be positive");
     Range range("ll_qkv_proj_append", layer, (long long)frame_start);
     if (d_model < 64 || d_model % 8) return fail(LL_ERR_UNSUPPORTED_SHAPE, "d_model must be a multiple of 8, at least 64");
-    if ((c->H * c->D) % 256 || c->H * c->D > 8192)
-        return fail(LL_ERR_UNSUPPORTED_SHAPE, "heads * head_dim must be a multiple of 256, at most 8192");
+    if (((c->H * c->D) % 256 && (c->H * c->D) % 192) || c->H * c->D > 8192)
+        return fail(LL_ERR_UNSUPPORTED_SHAPE, "heads * head_dim must be a multiple of 256 or of 192, at most 8192");
     if (c->kv_format != LL_KV_BF16) return fail(LL_ERR_UNSUPPORTED_SHAPE, "the fused projection is built for bf16 caches only");
     const bool with_norm = gain_q || gain_k;
     if (with_norm && (!gain_q || !gain_k || !(eps >= 0.f))) return fail(LL_ERR_INVALID_ARG, "both gains and eps >= 0 are needed for the norm");
@@ -831,7 +831,19 @@ int ll_qkv_proj_append(ll_cache *c, int layer, const ll_bf16 *x, int d_model, co
         ll::QkvParams p;
         memset(&p, 0, sizeof p);
         p.n_tokens = n_frames * c->P; p.d_model = d_model; p.heads = c->H; p.head_dim = c->D;
-        p.m_tiles = (p.n_tokens + 127) / 128; p.n_tiles = 3 * c->H * c->D / 256;
+        p.m_tiles = (p.n_tokens + 127) / 128;
+        {
+            // tile width: the one whose last round of tiles leaves the SMs less idle
+            const int hd = c->H * c->D, sms = c->sm_count > 0 ? c->sm_count : 148;
+            long long best = -1;
+            for (int tn : {256, 192}) {
+                if (hd % tn) continue;
+                const long long tiles = (long long)p.m_tiles * (3 * hd / tn), cost = (tiles + sms - 1) / sms * tn;
+                if (best < 0 || cost < best) { best = cost; p.tile_n = tn; }
+            }
+            p.n_tiles = 3 * hd / p.tile_n;
+            p.ssq_slots = 2 * hd / p.tile_n;
+        }
         p.P = c->P; p.grid_w = grid_w; p.n_t = rp.n_t; p.n_h = rp.n_h;
         p.with_norm = with_norm ? 1 : 0; p.eps = eps;
         p.bias = bias; p.gain_q = gain_q; p.gain_k = gain_k;
@@ -849,7 +861,7 @@ int ll_qkv_proj_append(ll_cache *c, int layer, const ll_bf16 *x, int d_model, co
                        (uint64_t)p.n_tokens * d_model * 2, 128, 1);
         if (s != LL_OK) return s;
         s = encode_map(&wmap, w_qkv, (uint64_t)d_model, (uint64_t)3 * c->H * c->D, 1, (uint64_t)d_model * 2,
-                       (uint64_t)3 * c->H * c->D * d_model * 2, 256, 1);
+                       (uint64_t)3 * c->H * c->D * d_model * 2, (uint32_t)p.tile_n, 1);
         if (s != LL_OK) return s;
         cudaError_t e = ll::launch_qkv_gemm(p, xmap, wmap, c->sm_count > 0 ? c->sm_count : 148, (cudaStream_t)stream);
         if (e != cudaSuccess) return cuda_fail(e, "qkv projection kernel");

@@ -143,7 +143,8 @@ struct RopeAppendParams {
 // QKV projection with norm, rotation and append in its epilogue (qkv_gemm.cu).
 struct QkvParams {
     int n_tokens, d_model, heads, head_dim;
-    int m_tiles, n_tiles;             // tiles of 128 tokens x 256 output features
+    int m_tiles, n_tiles;             // tiles of 128 tokens x tile_n output features
+    int tile_n, ssq_slots;            // 256 or 192; 2 * H*D / tile_n slots of the sum of squares per token
     int P, grid_w, n_t, n_h;
     int with_norm;
     float eps;
@@ -155,7 +156,7 @@ struct QkvParams {
     ll_bf16 *kcache, *vcache;         // layer base, [H][rows][D]
     int64_t rows_per_head;
     float *k_park;                    // [n_tokens, H*D] fp32 (with_norm): rotated k without its row factor
-    float *ssq;                       // [2][n_tokens][H*D/128] (with_norm): sums of squares per 128 features, q then k
+    float *ssq;                       // [2][n_tokens][ssq_slots] (with_norm): sums of squares per half tile, q then k
     uint32_t *status;
     int slot[LL_MAX_SLOTS];
 };

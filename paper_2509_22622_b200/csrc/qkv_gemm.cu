@@ -5,16 +5,18 @@
 //   q, k: optional RMS norm over the token's whole row of H*D elements with a learned gain,
 //         then the 3-D rotation;  rotated q -> q_out, rotated k and raw v -> the cache rows.
 //
-// The GEMM is a persistent tcgen05 kernel: CTA tile 128 tokens x 256 output features (two
-// heads of 128, or four of 64), K blocks of 64 through a 4-stage TMA ring, accumulators
-// double-buffered in TMEM (2 x 256 columns) so that the epilogue of a tile runs under the
-// main loop of the next.  Warp 0 (one lane): TMA producer.  Warp 1 (one elected lane): MMA
-// issuer.  Warps 4-7: epilogue, one thread per token row (the 32x32b TMEM shape).
+// The GEMM is a persistent tcgen05 kernel: CTA tile 128 tokens x TN output features, TN = 256
+// or 192 (whichever leaves the SMs less idle in the last round of tiles: 3*H*D / TN tiles per
+// 128 tokens over the SM count), K blocks of 64 through a TMA ring of 4 (TN 256) or 5 (TN 192)
+// stages, accumulators double-buffered in TMEM (2 x TN columns) so that the epilogue of a tile
+// runs under the main loop of the next.  Warp 0 (one lane): TMA producer.  Warp 1 (one elected
+// lane): MMA issuer.  Warps 4-11: epilogue, one thread per token row and half of the tile's
+// features (the 32x32b TMEM shape).
 //
 // The norm needs the sum of squares of a token's whole q (or k) row, which is spread over
 // H*D/256 tiles that run on different SMs at different times.  The factor is one scalar per
 // token and everything after it is linear, so a tile stores rotate(gain * y) without it and
-// leaves its part of the sum of squares in a table (one slot per token and 128 features: no atomics,
+// leaves its part of the sum of squares in a table (one slot per token and half tile: no atomics,
 // the sum is taken in a fixed order).  For q the scalar then travels with q_out to the
 // attention call as a per-row softmax scale; for k a small second kernel applies it: the
 // epilogue parks the un-normalised rotated k rows in fp32 in the caller's workspace and the
@@ -32,14 +34,19 @@ namespace {
 using namespace ptx;
 
 constexpr int kGemmThreads = 384;                      // TMA, MMA, two idle warps, eight epilogue warps
-constexpr int kTileM = 128, kTileN = 256, kBlockK = 64;
-constexpr int kGemmStages = 4;
+constexpr int kTileM = 128, kBlockK = 64;
 constexpr int kABytes = kTileM * kBlockK * 2;          // 16 KB
-constexpr int kBBytes = kTileN * kBlockK * 2;          // 32 KB
-constexpr int kStageBytes = kABytes + kBBytes;
-constexpr int kGemmSmem = kGemmStages * kStageBytes + 1024 /*barriers*/ + 1024 /*alignment*/;
 
-enum GBar { kFull = 0, kEmpty = kGemmStages, kAccFull = 2 * kGemmStages, kAccEmpty = 2 * kGemmStages + 2, kGemmBars = 2 * kGemmStages + 4 };
+template <int TN>
+struct GemmCfg {
+    static_assert(TN == 256 || TN == 192, "tile widths built");
+    static constexpr int kStages = TN == 256 ? 4 : 5;
+    static constexpr int kBBytes = TN * kBlockK * 2;   // 32 KB or 24 KB
+    static constexpr int kStageBytes = kABytes + kBBytes;
+    static constexpr int kSmem = kStages * kStageBytes + 1024 /*barriers*/ + 1024 /*alignment*/;
+    // barrier indices
+    static constexpr int kFull = 0, kEmpty = kStages, kAccFull = 2 * kStages, kAccEmpty = 2 * kStages + 2, kBars = 2 * kStages + 4;
+};
 
 __device__ __forceinline__ void tmem_ld_32x32b_x32(uint32_t taddr, uint32_t *r)
 {
@@ -49,90 +56,126 @@ __device__ __forceinline__ void tmem_ld_32x32b_x32(uint32_t taddr, uint32_t *r)
                  : "memory");
 }
 
-// One token row of half a 128 x 256 accumulator tile (128 features: `half` 0 or 1): bias, sum
-// of squares, gain, rotation, stores.  D is a template parameter and the 32-feature pieces are
-// unrolled, so which band (t, h or w) a rotation pair belongs to is known at compile time and
-// the piece's (cos, sin) pairs come from three row pointers at fixed offsets.
-template <int D>
-__device__ __forceinline__ float epilogue_half(const QkvParams &p, uint32_t taddr, int token, int n0, int half)
+// What an epilogue thread knows about its token row.
+struct EpiRow {
+    int which;                         // 0 q, 1 k, 2 v (a tile never straddles them)
+    int token, HD;
+    bool live, park;                   // park: k under the norm, fp32, finished by the second kernel
+    size_t cache_row;
+    const float *gain;
+    const float2 *t_row, *h_row, *w_row;
+};
+
+// 32 features of one token row (first feature cw inside q, k or v, n inside the 3*H*D outputs;
+// kD0 = cw % D, so which band - t, h or w - a rotation pair belongs to is known at compile time
+// and its (cos, sin) comes from one of three row pointers at a fixed offset): bias, sum of
+// squares, gain, rotation, stores.
+template <int D, int kD0>
+__device__ __forceinline__ void epilogue_piece(const QkvParams &p, const EpiRow &e, uint32_t taddr, int n, int cw, float &ssq)
 {
     constexpr int kNh = D / 6, kNt = D / 2 - 2 * kNh;  // pairs of the h (= w) and t bands
-    const int HD = p.heads * D;
-    const int which = n0 / HD;                         // 0 q, 1 k, 2 v (a tile never straddles them)
-    const int cw0 = n0 - which * HD + 128 * half;      // this half's first feature inside q, k or v
-    const bool live = token < p.n_tokens;
-    const int tok = live ? token : 0;
-    const int frame = tok / p.P, cell = tok % p.P;
-    const int y = cell / p.grid_w, x = cell % p.grid_w;
-    const size_t cache_row = (size_t)p.slot[frame] * p.P + cell;
-    const bool park = which == 1 && p.with_norm;       // k under the norm: fp32, finished by the second kernel
-    const float *gain = which == 0 ? p.gain_q : p.gain_k;
-    const float2 *t_row = p.t_tab + (size_t)frame * kNt, *h_row = p.h_tab + (size_t)y * kNh, *w_row = p.w_tab + (size_t)x * kNh;
-    float ssq = 0.f;
+    uint32_t r[32];
+    tmem_ld_32x32b_x32(taddr, r);
+    tmem_wait_ld();
+    const int head = cw / D;
+    float v[32];
 #pragma unroll
-    for (int ch = 0; ch < 4; ++ch) {
-        uint32_t r[32];
-        tmem_ld_32x32b_x32(taddr + 128 * half + 32 * ch, r);
-        tmem_wait_ld();
-        const int cw = cw0 + 32 * ch;                  // first feature of this 32-wide piece
-        const int head = cw / D;
-        const int d0 = (32 * ch) % D;                  // cw0 is a multiple of 128 and D divides 128
-        float v[32];
+    for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
+    if (p.bias) {
+        const float4 *bp = reinterpret_cast<const float4 *>(p.bias + n);
 #pragma unroll
-        for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
-        if (p.bias) {
-            const float4 *bp = reinterpret_cast<const float4 *>(p.bias + n0 + 128 * half + 32 * ch);
+        for (int i = 0; i < 8; ++i) {
+            const float4 bb = __ldg(bp + i);
+            v[4 * i] += bb.x; v[4 * i + 1] += bb.y; v[4 * i + 2] += bb.z; v[4 * i + 3] += bb.w;
+        }
+    }
+    if (e.which < 2) {
+#pragma unroll
+        for (int i = 0; i < 32; ++i) ssq = fmaf(v[i], v[i], ssq);
+        if (p.with_norm) {
+            const float4 *gp = reinterpret_cast<const float4 *>(e.gain + cw);
 #pragma unroll
             for (int i = 0; i < 8; ++i) {
-                const float4 bb = __ldg(bp + i);
-                v[4 * i] += bb.x; v[4 * i + 1] += bb.y; v[4 * i + 2] += bb.z; v[4 * i + 3] += bb.w;
+                const float4 gg = __ldg(gp + i);
+                v[4 * i] *= gg.x; v[4 * i + 1] *= gg.y; v[4 * i + 2] *= gg.z; v[4 * i + 3] *= gg.w;
             }
         }
-        if (which < 2) {
 #pragma unroll
-            for (int i = 0; i < 32; ++i) ssq = fmaf(v[i], v[i], ssq);
-            if (p.with_norm) {
-                const float4 *gp = reinterpret_cast<const float4 *>(gain + cw);
-#pragma unroll
-                for (int i = 0; i < 8; ++i) {
-                    const float4 gg = __ldg(gp + i);
-                    v[4 * i] *= gg.x; v[4 * i + 1] *= gg.y; v[4 * i + 2] *= gg.z; v[4 * i + 3] *= gg.w;
-                }
-            }
-#pragma unroll
-            for (int i = 0; i < 16; ++i) {
-                const int j = d0 / 2 + i;              // rotation pair inside the head row (compile time)
-                const float2 cs = j < kNt ? __ldg(t_row + j) : j < kNt + kNh ? __ldg(h_row + (j - kNt)) : __ldg(w_row + (j - kNt - kNh));
-                const float a = v[2 * i], b = v[2 * i + 1];
-                v[2 * i] = fmaf(a, cs.x, -(b * cs.y));
-                v[2 * i + 1] = fmaf(a, cs.y, b * cs.x);
-            }
+        for (int i = 0; i < 16; ++i) {
+            constexpr int j0 = kD0 / 2;
+            const int j = j0 + i;                      // rotation pair inside the head row (compile time)
+            const float2 cs = j < kNt ? __ldg(e.t_row + j) : j < kNt + kNh ? __ldg(e.h_row + (j - kNt)) : __ldg(e.w_row + (j - kNt - kNh));
+            const float a = v[2 * i], b = v[2 * i + 1];
+            v[2 * i] = fmaf(a, cs.x, -(b * cs.y));
+            v[2 * i + 1] = fmaf(a, cs.y, b * cs.x);
         }
-        if (!live) continue;
-        if (park) {
-            float4 *dst = reinterpret_cast<float4 *>(p.k_park + (size_t)token * HD + cw);
+    }
+    if (!e.live) return;
+    if (e.park) {
+        float4 *dst = reinterpret_cast<float4 *>(p.k_park + (size_t)e.token * e.HD + cw);
 #pragma unroll
-            for (int i = 0; i < 8; ++i) dst[i] = make_float4(v[4 * i], v[4 * i + 1], v[4 * i + 2], v[4 * i + 3]);
-        } else {
-            ll_bf16 *dst;
-            if (which == 0) dst = p.q_out + ((size_t)token * p.heads + head) * D + d0;
-            else            dst = (which == 1 ? p.kcache : p.vcache) + ((size_t)head * p.rows_per_head + cache_row) * D + d0;
-            uint32_t o[16];
+        for (int i = 0; i < 8; ++i) dst[i] = make_float4(v[4 * i], v[4 * i + 1], v[4 * i + 2], v[4 * i + 3]);
+    } else {
+        ll_bf16 *dst;
+        if (e.which == 0) dst = p.q_out + ((size_t)e.token * p.heads + head) * D + kD0;
+        else              dst = (e.which == 1 ? p.kcache : p.vcache) + ((size_t)head * p.rows_per_head + e.cache_row) * D + kD0;
+        uint32_t o[16];
 #pragma unroll
-            for (int i = 0; i < 16; ++i) o[i] = cvt_bf16x2(v[2 * i], v[2 * i + 1]);
+        for (int i = 0; i < 16; ++i) o[i] = cvt_bf16x2(v[2 * i], v[2 * i + 1]);
 #pragma unroll
-            for (int i = 0; i < 4; ++i)
-                reinterpret_cast<uint4 *>(dst)[i] = make_uint4(o[4 * i], o[4 * i + 1], o[4 * i + 2], o[4 * i + 3]);
+        for (int i = 0; i < 4; ++i)
+            reinterpret_cast<uint4 *>(dst)[i] = make_uint4(o[4 * i], o[4 * i + 1], o[4 * i + 2], o[4 * i + 3]);
+    }
+}
+
+// One token row of half a 128 x TN accumulator tile (TN / 2 features: `half` 0 or 1), 32
+// features at a time; returns the half's sum of squares.
+template <int D, int TN>
+__device__ __forceinline__ float epilogue_half(const QkvParams &p, uint32_t taddr, int token, int n0, int half)
+{
+    constexpr int kNh = D / 6, kNt = D / 2 - 2 * kNh;
+    constexpr int kHalf = TN / 2;
+    EpiRow e;
+    e.HD = p.heads * D;
+    e.which = n0 / e.HD;
+    e.live = token < p.n_tokens;
+    e.token = token;
+    const int tok = e.live ? token : 0;
+    const int frame = tok / p.P, cell = tok % p.P;
+    e.cache_row = (size_t)p.slot[frame] * p.P + cell;
+    e.park = e.which == 1 && p.with_norm;
+    e.gain = e.which == 0 ? p.gain_q : p.gain_k;
+    e.t_row = p.t_tab + (size_t)frame * kNt;
+    e.h_row = p.h_tab + (size_t)(cell / p.grid_w) * kNh;
+    e.w_row = p.w_tab + (size_t)(cell % p.grid_w) * kNh;
+    const int cw0 = n0 - e.which * e.HD + kHalf * half;    // this half's first feature inside q, k or v
+    float ssq = 0.f;
+#pragma unroll 1
+    for (int ch = 0; ch < kHalf / 32; ++ch) {
+        const int cw = cw0 + 32 * ch, n = n0 + kHalf * half + 32 * ch;
+        const uint32_t t = taddr + kHalf * half + 32 * ch;
+        switch (cw % D) {                                  // the same for the whole warp
+        case 0: epilogue_piece<D, 0>(p, e, t, n, cw, ssq); break;
+        case 32: epilogue_piece<D, 32>(p, e, t, n, cw, ssq); break;
+        default:
+            if constexpr (D == 128) {
+                if (cw % D == 64) epilogue_piece<D, 64>(p, e, t, n, cw, ssq);
+                else              epilogue_piece<D, 96>(p, e, t, n, cw, ssq);
+            }
+            break;
         }
     }
     return ssq;
 }
 
-template <int D>
+template <int D, int TN>
 __global__ void __launch_bounds__(kGemmThreads, 1)
 qkv_gemm_kernel(const __grid_constant__ QkvParams p, const __grid_constant__ CUtensorMap xmap,
                 const __grid_constant__ CUtensorMap wmap)
 {
+    using G = GemmCfg<TN>;
+    constexpr int kGemmStages = G::kStages, kStageBytes = G::kStageBytes, kTileN = TN, kGemmBars = G::kBars;
+    constexpr int kFull = G::kFull, kEmpty = G::kEmpty, kAccFull = G::kAccFull, kAccEmpty = G::kAccEmpty;
     extern __shared__ uint8_t smem_raw[];
     const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     uint8_t *smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));
@@ -221,15 +264,15 @@ qkv_gemm_kernel(const __grid_constant__ QkvParams p, const __grid_constant__ CUt
             if (!__all_sync(0xffffffffu, wait(kAccFull + buf, t >> 1, (int)t))) goto done;
             tc_fence_after_sync();
             const int token = m0 + 32 * q4 + lane;
-            const float ssq = epilogue_half<D>(p, tmem + buf * kTileN + ((uint32_t)(32 * q4) << 16), token, n0, half);
+            const float ssq = epilogue_half<D, TN>(p, tmem + buf * kTileN + ((uint32_t)(32 * q4) << 16), token, n0, half);
             tc_fence_before_sync();
             __syncwarp();
             if (lane == 0) mbar_arrive(bar(kAccEmpty + buf));
-            // the half's part of the row's sum of squares: one slot per token and 128 features
+            // the half's part of the row's sum of squares: one slot per token and half tile
             const int HD = p.heads * D;
             if (p.with_norm && n0 < 2 * HD && token < p.n_tokens) {
                 const int which = n0 / HD;
-                p.ssq[((size_t)which * p.n_tokens + token) * (HD / 128) + (n0 - which * HD) / 128 + half] = ssq;
+                p.ssq[((size_t)which * p.n_tokens + token) * p.ssq_slots + 2 * ((n0 - which * HD) / kTileN) + half] = ssq;
             }
         }
     }
@@ -249,14 +292,14 @@ done:
 }
 
 // The norm's second step, one thread block per token: the row factors from the sums of squares
-// per 128 features (added in feature order), q's to q_row_scale, k's applied to the parked fp32
+// per half tile (added in feature order), q's to q_row_scale, k's applied to the parked fp32
 // row, which is rounded once to bf16 into the cache row.  One thread per 8 features.
 __global__ void __launch_bounds__(1024)
 qkv_finish_kernel(const __grid_constant__ QkvParams p)
 {
     __shared__ float r_sh[2];
     const int HD = p.heads * p.head_dim;
-    const int tiles = HD / 128;
+    const int tiles = p.ssq_slots;
     const int token = blockIdx.x;
     if (threadIdx.x < 2) {
         const float *src = p.ssq + ((size_t)threadIdx.x * p.n_tokens + token) * tiles;
@@ -282,17 +325,23 @@ qkv_finish_kernel(const __grid_constant__ QkvParams p)
 cudaError_t launch_qkv_gemm(const QkvParams &p, const CUtensorMap &xmap, const CUtensorMap &wmap, int sm_count,
                             cudaStream_t stream)
 {
-    cudaError_t e = p.head_dim == 128
-        ? cudaFuncSetAttribute(qkv_gemm_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, kGemmSmem)
-        : cudaFuncSetAttribute(qkv_gemm_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, kGemmSmem);
-    if (e != cudaSuccess) return e;
     const int n_tiles = p.m_tiles * p.n_tiles;
     if (n_tiles <= 0) return cudaSuccess;
     const int grid = n_tiles < sm_count ? n_tiles : sm_count;
-    if (p.head_dim == 128) qkv_gemm_kernel<128><<<grid, kGemmThreads, kGemmSmem, stream>>>(p, xmap, wmap);
-    else                   qkv_gemm_kernel<64><<<grid, kGemmThreads, kGemmSmem, stream>>>(p, xmap, wmap);
+    cudaError_t e = cudaErrorInvalidValue;
+#define LL_GEMM_CASE(DD, TT)                                                                                                  \
+    if (p.head_dim == DD && p.tile_n == TT) {                                                                                  \
+        e = cudaFuncSetAttribute(qkv_gemm_kernel<DD, TT>, cudaFuncAttributeMaxDynamicSharedMemorySize, GemmCfg<TT>::kSmem);   \
+        if (e != cudaSuccess) return e;                                                                                        \
+        qkv_gemm_kernel<DD, TT><<<grid, kGemmThreads, GemmCfg<TT>::kSmem, stream>>>(p, xmap, wmap);                            \
+        e = cudaGetLastError();                                                                                                \
+    }
+    LL_GEMM_CASE(128, 256)
+    LL_GEMM_CASE(128, 192)
+    LL_GEMM_CASE(64, 256)
+    LL_GEMM_CASE(64, 192)
+#undef LL_GEMM_CASE
     count_launch();
-    e = cudaGetLastError();
     if (e != cudaSuccess || !p.with_norm) return e;
     qkv_finish_kernel<<<(unsigned)p.n_tokens, p.heads * p.head_dim / 8, 0, stream>>>(p);
     count_launch();

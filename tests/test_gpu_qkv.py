@@ -14,12 +14,14 @@ pytestmark = pytest.mark.gpu
 
 F64 = synth.bf16_bits_to_f64
 
-# (workload, d_model): heads * head_dim a multiple of 256; ragged last token tile; a d_model
-# that is not a multiple of the GEMM's 64-wide K block
+# (workload, d_model): heads * head_dim a multiple of 256 or of 192 (the two tile widths, at
+# both head sizes); ragged last token tile; a d_model that is not a multiple of the GEMM's
+# 64-wide K block
 SHAPES = [
     (synth.Workload("qkv_d128", 1, 2, 128, 6, 25, 3, 3, 6, n_chunks=4, seed=71), 192),
     (synth.Workload("qkv_d64", 1, 4, 64, 9, 14, 2, 2, 4, n_chunks=4, seed=72), 136),
-    (synth.Workload("qkv_wide", 1, 6, 128, 5, 13, 2, 2, 4, n_chunks=3, seed=73), 320),
+    (synth.Workload("qkv_wide", 1, 6, 128, 5, 13, 2, 2, 4, n_chunks=3, seed=73), 320),      # 768 = 4 x 192: the 192-wide tiles
+    (synth.Workload("qkv_d64_192", 1, 3, 64, 7, 11, 2, 2, 4, n_chunks=3, seed=74), 200),     # 192 = 3 heads of 64 in one tile
 ]
 
 
@@ -163,7 +165,7 @@ def test_projection_at_the_benchmark_shape(oracle_mod):
 
 
 def test_projection_argument_checks():
-    wl = synth.Workload("qkv_small", 1, 2, 64, 4, 4, 1, 1, 2, n_chunks=1, seed=0)      # heads*head_dim = 128
+    wl = synth.Workload("qkv_small", 1, 2, 64, 4, 4, 1, 1, 2, n_chunks=1, seed=0)      # heads*head_dim = 128: neither tile width divides it
     cache = B.Cache(*wl.cache_args)
     x = torch.zeros(16, 64, device="cuda", dtype=torch.bfloat16)
     w = torch.zeros(3 * 128, 64, device="cuda", dtype=torch.bfloat16)

@@ -31,6 +31,8 @@ using namespace ptx;
 
 constexpr int kBwdThreads = 288;                       // eight compute warps, one load/issue warp
 constexpr int kIssueWarp = 8;
+constexpr int kDkdvThreads = 320;                      // the dk/dv kernel adds a load warp
+constexpr int kLoadWarp = 9;
 constexpr int kTile = 128;
 
 __device__ __forceinline__ void tmem_ld_32x32b_x32(uint32_t taddr, uint32_t *r)
@@ -446,17 +448,26 @@ __device__ __forceinline__ bool group_sees(const AttnGroup &G, int r0)
     return any;
 }
 
-// The (group, 128-row query tile) pairs a key tile takes part in, in order.
+// The (group, 128-row query tile) pairs a key tile takes part in, in order.  The group's first row
+// and tile count are kept, so a step inside a group costs an increment.
 struct QTiles {
     const BwdParams &p;
-    int r0, g, i;
-    __device__ QTiles(const BwdParams &params, int first_row) : p(params), r0(first_row), g(0), i(-1) { next(); }
+    int r0, g, i, tiles, q_begin;
+    __device__ QTiles(const BwdParams &params, int first_row) : p(params), r0(first_row), g(-1), i(0), tiles(0), q_begin(0) { next(); }
     __device__ bool done() const { return g >= p.n_groups; }
-    __device__ int q_row() const { return p.g[g].q_begin + i * kTile; }
+    __device__ int q_row() const { return q_begin + i * kTile; }
     __device__ void next()
     {
-        ++i;
-        while (g < p.n_groups && !(i * kTile < p.g[g].q_rows && group_sees(p.g[g], r0))) { ++g; i = 0; }
+        if (++i < tiles) return;
+        i = 0;
+        for (++g; g < p.n_groups; ++g) {
+            const AttnGroup &G = p.g[g];
+            if (G.q_rows > 0 && group_sees(G, r0)) {
+                tiles = (G.q_rows + kTile - 1) / kTile;
+                q_begin = G.q_begin;
+                return;
+            }
+        }
     }
 };
 
@@ -469,9 +480,10 @@ struct QTiles {
 // Shared memory has room for three streamed tiles beside K, V, P and dS, so Q is loaded twice:
 //   slot j % 2:  Q(j) for S(j), then (once S(j) is done) dO(j) for dP(j) and dV(j), then Q(j+2)
 //   slot C:      Q(j) for dK(j), then Q(j+1)
-// which gives every load about one step of lead.
+// which gives every load about one step of lead.  The loads have a warp of their own (warp 9),
+// so that the MMA issuer (warp 8) never sits in a wait for a slot while products could be issued.
 template <int D>
-__global__ void __launch_bounds__(kBwdThreads, 1)
+__global__ void __launch_bounds__(kDkdvThreads, 1)
 bwd_dkdv_kernel(const __grid_constant__ BwdParams p, const __grid_constant__ BwdMaps maps)
 {
     using C = BwdCfg<D>;
@@ -508,10 +520,10 @@ bwd_dkdv_kernel(const __grid_constant__ BwdParams p, const __grid_constant__ Bwd
     const uint32_t t_s = tmem, t_dp = tmem + 128, t_dk = tmem + 256, t_dv = tmem + 256 + D;
 
     if (skip) {
-    } else if (warp == kIssueWarp) {
+    } else if (warp == kLoadWarp) {
+        // ---- loads: all lanes walk the loop, one elected lane issues the copies ----
         [&]() {
-            const bool elected = elect_one();                    // all lanes walk the loop; one issues
-            constexpr uint32_t idesc_s = idesc_bf16_f32(128, 128, 0, 0), idesc_g = idesc_bf16_f32(128, D, 1, 1);
+            const bool elected = elect_one();
             auto load_tile = [&](uint32_t dst, const CUtensorMap *map, int bar_id, int q_row) {
                 if (elected) {
                     mbar_arrive_expect_tx(bar(bar_id), C::kTileBytes);
@@ -519,7 +531,6 @@ bwd_dkdv_kernel(const __grid_constant__ BwdParams p, const __grid_constant__ Bwd
                 }
                 __syncwarp();
             };
-            auto commit = [&](int bar_id) { if (elected) tc_commit(bar(bar_id)); };
             // first rows of the query tiles of steps j, j + 1, j + 2 (-1: no such step)
             QTiles qt(p, r0);
             auto take = [&]() -> int { if (qt.done()) return -1; const int r = qt.q_row(); qt.next(); return r; };
@@ -536,6 +547,32 @@ bwd_dkdv_kernel(const __grid_constant__ BwdParams p, const __grid_constant__ Bwd
             load_tile(slot_s, &maps.q, kSlotFull + 0, row_j);
             if (row_j1 >= 0) load_tile(slot_s + C::kTileBytes, &maps.q, kSlotFull + 1, row_j1);
             load_tile(c_s, &maps.q, kCFull, row_j);
+            if (!wait(kSFull, 0, 0)) return;                     // S(0) has read Q(0): its slot takes dO(0)
+            load_tile(slot_s, &maps.d_out, kSlotFull + 0, row_j);
+            for (int j = 0; row_j1 >= 0; ++j) {
+                const int sl = j & 1;
+                if (!wait(kSFull, j + 1, j)) return;             // S(j+1) has read Q(j+1): its slot takes dO(j+1)
+                load_tile(slot_s + (sl ^ 1) * C::kTileBytes, &maps.d_out, kSlotFull + (sl ^ 1), row_j1);
+                if (row_j2 >= 0) {                               // dV(j) has read dO(j): its slot takes Q(j+2)
+                    if (!wait(kSlotFree + sl, j >> 1, j)) return;
+                    load_tile(slot_s + sl * C::kTileBytes, &maps.q, kSlotFull + sl, row_j2);
+                }
+                if (!wait(kCFree, j, j)) return;                 // dK(j) has read Q(j)
+                load_tile(c_s, &maps.q, kCFull, row_j1);
+                row_j = row_j1;
+                row_j1 = row_j2;
+                row_j2 = take();
+            }
+        }();
+    } else if (warp == kIssueWarp) {
+        // ---- MMA issue: all lanes walk the loop and the waits, one elected lane issues ----
+        [&]() {
+            const bool elected = elect_one();
+            constexpr uint32_t idesc_s = idesc_bf16_f32(128, 128, 0, 0), idesc_g = idesc_bf16_f32(128, D, 1, 1);
+            auto commit = [&](int bar_id) { if (elected) tc_commit(bar(bar_id)); };
+            int n_steps = 0;
+            for (QTiles qt(p, r0); !qt.done(); qt.next()) ++n_steps;
+            if (n_steps == 0) return;
             const uint32_t k_k = lo_kmajor(k_s), v_k = lo_kmajor(v_s), p_mn = lo_mnmajor(p_s), ds_mn = lo_mnmajor(ds_s), c_mn = lo_mnmajor(c_s);
             // a slot's fills alternate Q (for S) and dO: waits see parity 0 for Q, 1 for dO
             auto issue_s = [&](int j) -> bool {
@@ -557,17 +594,13 @@ bwd_dkdv_kernel(const __grid_constant__ BwdParams p, const __grid_constant__ Bwd
                 return true;
             };
             if (!wait(kKvFull, 0, 0)) return;
-            if (!issue_s(0)) return;
-            if (!wait(kSFull, 0, 0)) return;                     // S(0) has read Q(0): its slot takes dO(0)
-            load_tile(slot_s, &maps.d_out, kSlotFull + 0, row_j);
-            if (!issue_dp(0)) return;
-            for (int j = 0;; ++j) {
+            if (!issue_s(0) || !issue_dp(0)) return;
+            for (int j = 0; j < n_steps; ++j) {
                 const int sl = j & 1;
-                if (row_j1 >= 0) {
+                const bool more = j + 1 < n_steps;
+                if (more) {
                     if (!wait(kSFree, j, j)) return;             // S(j) is in the compute warps' registers
                     if (!issue_s(j + 1)) return;
-                    if (!wait(kSFull, j + 1, j)) return;         // S(j+1) has read Q(j+1): its slot takes dO(j+1)
-                    load_tile(slot_s + (sl ^ 1) * C::kTileBytes, &maps.d_out, kSlotFull + (sl ^ 1), row_j1);
                 }
                 if (!wait(kDsFull, j, j)) return;                // P(j) and dS(j) are in shared memory, dP(j) has been read
                 tc_fence_after_sync();
@@ -580,17 +613,7 @@ bwd_dkdv_kernel(const __grid_constant__ BwdParams p, const __grid_constant__ Bwd
                 if (elected) mma_slices<0, kTile / 16, true, true>(t_dk, ds_mn, c_mn, idesc_g, j > 0 ? 1u : 0u);
                 __syncwarp();
                 commit(kCFree);
-                if (row_j1 < 0) break;
-                if (!issue_dp(j + 1)) return;
-                if (row_j2 >= 0) {                               // dV(j) has read dO(j): its slot takes Q(j+2)
-                    if (!wait(kSlotFree + sl, j >> 1, j)) return;
-                    load_tile(slot_s + sl * C::kTileBytes, &maps.q, kSlotFull + sl, row_j2);
-                }
-                if (!wait(kCFree, j, j)) return;                 // dK(j) has read Q(j)
-                load_tile(c_s, &maps.q, kCFull, row_j1);
-                row_j = row_j1;
-                row_j1 = row_j2;
-                row_j2 = take();
+                if (more && !issue_dp(j + 1)) return;
             }
         }();
     } else {
@@ -679,8 +702,8 @@ cudaError_t launch_attn_backward(const BwdParams &p, const BwdMaps &maps, cudaSt
     else          bwd_dq_kernel<64><<<gq, kBwdThreads, smem_dq, stream>>>(p, maps);
     count_launch();
     if ((e = cudaGetLastError()) != cudaSuccess) return e;
-    if (D == 128) bwd_dkdv_kernel<128><<<gk, kBwdThreads, smem_kv, stream>>>(p, maps);
-    else          bwd_dkdv_kernel<64><<<gk, kBwdThreads, smem_kv, stream>>>(p, maps);
+    if (D == 128) bwd_dkdv_kernel<128><<<gk, kDkdvThreads, smem_kv, stream>>>(p, maps);
+    else          bwd_dkdv_kernel<64><<<gk, kDkdvThreads, smem_kv, stream>>>(p, maps);
     count_launch();
     return cudaGetLastError();
 }

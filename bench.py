@@ -582,6 +582,20 @@ def run_ours(args):
         others["kv_e4m3"] = {"append_us": ms_a * 1e3, "attention_ms_incl_expansion": ms_t,
                              "attention_tflops": attn_flops(wl) / ms_t / 1e9,
                              "storage_bytes_30_layers": None, "bf16_storage_bytes_30_layers": None}
+        if args.in_loop_seconds > 0:
+            # the same call back to back for about a second: the figure under the power cap
+            n8 = int(1e3 / ms_t) + 1
+            a8, b8 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            for _ in range(n8 // 2):
+                att8()
+            a8.record(stream)
+            for _ in range(n8 // 2):
+                att8()
+            b8.record(stream)
+            torch.cuda.synchronize()
+            ms_loop8 = a8.elapsed_time(b8) / (n8 // 2)
+            others["kv_e4m3"]["attention_ms_in_a_one_second_loop"] = ms_loop8
+            others["kv_e4m3"]["attention_tflops_in_the_loop"] = attn_flops(wl) / ms_loop8 / 1e9
         h8, h16 = B.ll_cache_create(30, H, D, P, C, wl.sink_frames, wl.window_frames), \
             B.ll_cache_create(30, H, D, P, C, wl.sink_frames, wl.window_frames)
         B.ll_cache_set_kv_format(h8, B.LL_KV_E4M3)
